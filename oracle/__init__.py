@@ -1,0 +1,158 @@
+"""Python access to the CPU checker (``clv_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by the smoke check and by the CPU-baseline
+timing of the benchmark.  The GPU library never imports this package and this package never
+imports the GPU library.
+
+Every wrapper takes and returns numpy arrays; bf16 tensors are ``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "clv_oracle.c")
+_LIB = os.path.join(_HERE, "libclv_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the checker with gcc (plain -O2, OpenMP for the independent outer loops)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_f64_to_bf16.restype = ctypes.c_uint16
+        _lib.orc_f64_to_bf16.argtypes = [ctypes.c_double]
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def threads() -> int:
+    """Number of threads the OpenMP loops use."""
+    v = os.environ.get("OMP_NUM_THREADS")
+    return int(v) if v else (os.cpu_count() or 1)
+
+
+def f64_to_bf16_bits(x: float) -> int:
+    return int(_load().orc_f64_to_bf16(float(x)))
+
+
+def tree_attn(q, k_cache, v_cache, k_tree, v_tree, parent, ctx_len, scale, *,
+              block_table=None, page_size=64, rows=None
+              ) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Tree attention by the definition (Sec. 2.1).
+
+    q [B,N,Hq,D], k_tree/v_tree [B,N,Hkv,D], cache contiguous [B,cap,Hkv,D] or paged
+    [P,page,Hkv,D] with block_table [B,max_pages].  ``rows``: optional int32 [R,3] of (b,i,h)
+    to evaluate; default all.  Returns (out_f64 [R,D], out_bf16_bits [R,D], lse [R], status [B]);
+    with rows=None the first three are reshaped to [B,N,Hq,...].
+    """
+    lib = _load()
+    q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
+    k_tree = _c(k_tree, np.uint16); v_tree = _c(v_tree, np.uint16)
+    parent = _c(parent, np.int32); ctx_len = _c(ctx_len, np.int32)
+    B, N, Hq, D = q.shape
+    Hkv = k_tree.shape[2]
+    paged = block_table is not None
+    if paged:
+        block_table = _c(block_table, np.int32)
+        cap, max_pages = 0, block_table.shape[1]
+        page_size = k_cache.shape[1]
+    else:
+        cap, max_pages = k_cache.shape[1], 0
+    if rows is None:
+        R = B * N * Hq
+        rows_arr = None
+    else:
+        rows_arr = _c(rows, np.int32).reshape(-1, 3)
+        R = rows_arr.shape[0]
+    out = np.empty((R, D), dtype=np.float64)
+    out16 = np.empty((R, D), dtype=np.uint16)
+    lse = np.empty(R, dtype=np.float64)
+    status = np.zeros(B, dtype=np.int32)
+    lib.orc_tree_attn(ctypes.c_int(B), ctypes.c_int(N), ctypes.c_int(Hq), ctypes.c_int(Hkv),
+                      ctypes.c_int(D), _p(q), _p(k_cache), _p(v_cache), ctypes.c_int(int(paged)),
+                      ctypes.c_int(cap), ctypes.c_int(page_size), ctypes.c_int(max_pages),
+                      _p(block_table), _p(k_tree), _p(v_tree), _p(parent), _p(ctx_len),
+                      ctypes.c_double(float(scale)), ctypes.c_int64(R), _p(rows_arr), _p(out),
+                      _p(out16), _p(lse), _p(status))
+    if rows is None:
+        return (out.reshape(B, N, Hq, D), out16.reshape(B, N, Hq, D), lse.reshape(B, N, Hq),
+                status)
+    return out, out16, lse, status
+
+
+def argmax(logits: np.ndarray, vocab: int) -> np.ndarray:
+    """First strict maximum of each row; logits [..., ld] bf16 bits, the first ``vocab`` columns
+    of a row are scanned (Sec. 4.2: temperature 0 = greedy target decoding)."""
+    lib = _load()
+    lg = _c(logits, np.uint16)
+    ld = lg.shape[-1]
+    lead = lg.shape[:-1]
+    R = int(np.prod(lead)) if lead else 1
+    ids = np.empty(R, dtype=np.int32)
+    lib.orc_argmax(ctypes.c_int64(R), ctypes.c_int(vocab), ctypes.c_int64(ld), _p(lg), _p(ids))
+    return ids.reshape(lead)
+
+
+def accept_walk(parent, tokens, ids, path_cap: int):
+    """Greedy acceptance walk; returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
+    status [B])."""
+    lib = _load()
+    parent = _c(parent, np.int32); tokens = _c(tokens, np.int32); ids = _c(ids, np.int32)
+    B, N = parent.shape
+    alen = np.empty(B, dtype=np.int32)
+    aidx = np.empty((B, path_cap), dtype=np.int32)
+    nxt = np.empty(B, dtype=np.int32)
+    status = np.empty(B, dtype=np.int32)
+    lib.orc_accept_walk(ctypes.c_int(B), ctypes.c_int(N), ctypes.c_int(path_cap), _p(parent),
+                        _p(tokens), _p(ids), _p(alen), _p(aidx), _p(nxt), _p(status))
+    return alen, aidx, nxt, status
+
+
+def kv_commit(k_cache, v_cache, k_tree, v_tree, accept_idx, accept_len, ctx_len, *,
+              block_table=None):
+    """Returns (k_cache', v_cache', ctx_len_out, status); the inputs are not modified."""
+    lib = _load()
+    kc = np.array(k_cache, dtype=np.uint16, order="C", copy=True)
+    vc = np.array(v_cache, dtype=np.uint16, order="C", copy=True)
+    k_tree = _c(k_tree, np.uint16); v_tree = _c(v_tree, np.uint16)
+    accept_idx = _c(accept_idx, np.int32); accept_len = _c(accept_len, np.int32)
+    ctx_len = _c(ctx_len, np.int32)
+    B, N, Hkv, D = k_tree.shape
+    path_cap = accept_idx.shape[1]
+    paged = block_table is not None
+    if paged:
+        block_table = _c(block_table, np.int32)
+        cap, max_pages, n_pages, page = 0, block_table.shape[1], kc.shape[0], kc.shape[1]
+    else:
+        cap, max_pages, n_pages, page = kc.shape[1], 0, 0, 64
+    out_len = np.empty(B, dtype=np.int32)
+    status = np.empty(B, dtype=np.int32)
+    lib.orc_kv_commit(ctypes.c_int(B), ctypes.c_int(N), ctypes.c_int(Hkv), ctypes.c_int(D),
+                      ctypes.c_int(path_cap), _p(kc), _p(vc), ctypes.c_int(int(paged)),
+                      ctypes.c_int(cap), ctypes.c_int(page), ctypes.c_int(n_pages),
+                      ctypes.c_int(max_pages), _p(block_table), _p(k_tree), _p(v_tree),
+                      _p(accept_idx), _p(accept_len), _p(ctx_len), _p(out_len), _p(status))
+    return kc, vc, out_len, status

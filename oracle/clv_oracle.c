@@ -1,0 +1,279 @@
+/*
+ * CPU checker for the tree-verification step of Clover-2-style speculative decoding.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the verification
+ * step computes, written from the paper's prose; the GPU library is compared against it.  It
+ * shares no code with the GPU library and must never be called from the product path.
+ *
+ * All floating point is IEEE double.  bf16 inputs arrive as uint16 bit patterns and are widened
+ * exactly.  There is no blocking, tiling or reordering: every function is the definition itself
+ * written as nested loops (OpenMP only distributes independent outer iterations).
+ *
+ * What each function follows:
+ *   orc_tree_attn     - Sec. 2.1 "Speculative Decoding and Tree Attention" and the caption of
+ *                       Fig. 2: ordinary softmax attention whose causal mask is the token
+ *                       tree's topology matrix (a node sees the committed context and its own
+ *                       ancestors, itself included).
+ *   orc_argmax        - Sec. 4.2 (Table 1 note): temperature 0 is greedy decoding of the target.
+ *   orc_accept_walk   - Sec. 2.1 verification phase (the target filters out wrong drafted
+ *                       tokens; the output equals plain decoding) with the greedy rule of the
+ *                       tree-sampling algorithm Sec. 4.1 adopts.
+ *   orc_kv_commit     - derived from the equivalence requirement of Sec. 2.1: after a step the
+ *                       cache holds exactly what plain decoding of the accepted tokens would.
+ *
+ * Pins (tests/test_oracle_*.py): path linearisation, chain == causal prefill, star == independent
+ * decodes, a float64 library attention with an explicit boolean mask, convex-hull and
+ * log-sum-exp identities, mask exactness under perturbation, brute-force path enumeration,
+ * numpy's first-occurrence argmax, and the commit/append equivalence.  No function here is
+ * "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_OK 0
+#define ORC_ERR_TREE 7   /* same numeric meaning as the status values the library documents */
+
+static double bf16_to_f64(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+/* Round a double to the nearest bf16 (ties to even), one rounding step, result as bits. */
+static uint16_t f64_to_bf16(double d) {
+  if (d != d) return 0x7FC0;
+  uint16_t sign = signbit(d) ? 0x8000 : 0;
+  double a = fabs(d);
+  if (a == 0.0) return sign;
+  if (isinf(a)) return sign | 0x7F80;
+  int e;
+  (void)frexp(a, &e); /* a = m * 2^e, m in [0.5,1)  ->  floor(log2 a) = e-1 */
+  int p = e - 1;
+  if (p < -126) p = -126;                /* subnormal range keeps a fixed quantum */
+  double quantum = ldexp(1.0, p - 7);    /* spacing of bf16 values in this binade */
+  double r = nearbyint(a / quantum) * quantum; /* default rounding mode: ties to even */
+  if (r >= ldexp(1.0, 128)) return sign | 0x7F80;
+  float f = (float)r; /* exact: r has at most 8 significant bits */
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  return sign | (uint16_t)(u >> 16);
+}
+
+/* Address of cache row `t` (token position) of sequence b, kv head g. */
+typedef struct {
+  const uint16_t *k, *v;
+  int paged, cap_tokens, page_size, max_pages, n_kv_heads, head_dim;
+  const int32_t *block_table;
+} orc_cache;
+
+static int64_t cache_row_offset(const orc_cache *c, int b, int64_t t, int g) {
+  int64_t row;
+  if (c->paged) {
+    int64_t page = c->block_table[(int64_t)b * c->max_pages + t / c->page_size];
+    row = page * c->page_size + t % c->page_size;
+  } else {
+    row = (int64_t)b * c->cap_tokens + t;
+  }
+  return (row * c->n_kv_heads + g) * c->head_dim;
+}
+
+static int tree_ok(const int32_t *parent, int n, int allow_forest) {
+  for (int i = 0; i < n; ++i) {
+    int p = parent[i];
+    if (i == 0) {
+      if (p != -1) return 0;
+    } else if (p == -1) {
+      if (!allow_forest) return 0;
+    } else if (p < 0 || p >= i) {
+      return 0;
+    }
+  }
+  return 1;
+}
+
+/*
+ * Tree attention.  rows == NULL: every (b, i, h) in that order, n_rows = B*N*Hq.
+ * Otherwise rows holds n_rows triples (b, i, h).  Row r of the outputs belongs to rows[r].
+ * out_f64 [n_rows, D] double; out_bf16 [n_rows, D] bits (may be NULL); lse [n_rows] natural log
+ * (may be NULL).  status [B]: ORC_ERR_TREE if parent[] of that sequence is malformed (its rows
+ * are then filled with zeros).  Forests (several -1 parents) are allowed here.
+ */
+int orc_tree_attn(int B, int N, int Hq, int Hkv, int D, const uint16_t *q, const uint16_t *kc,
+                  const uint16_t *vc, int paged, int cap_tokens, int page_size, int max_pages,
+                  const int32_t *block_table, const uint16_t *k_tree, const uint16_t *v_tree,
+                  const int32_t *parent, const int32_t *ctx_len, double scale, int64_t n_rows,
+                  const int32_t *rows, double *out_f64, uint16_t *out_bf16, double *lse,
+                  int32_t *status) {
+  orc_cache c = {kc, vc, paged, cap_tokens, page_size, max_pages, Hkv, D, block_table};
+  int G = Hq / Hkv;
+  for (int b = 0; b < B; ++b)
+    status[b] = tree_ok(parent + (int64_t)b * N, N, 1) ? ORC_OK : ORC_ERR_TREE;
+
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t r = 0; r < n_rows; ++r) {
+    int b, i, h;
+    if (rows) {
+      b = rows[3 * r]; i = rows[3 * r + 1]; h = rows[3 * r + 2];
+    } else {
+      b = (int)(r / ((int64_t)N * Hq)); i = (int)((r / Hq) % N); h = (int)(r % Hq);
+    }
+    double *o = out_f64 + r * D;
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    if (status[b] != ORC_OK) {
+      if (out_bf16) for (int d = 0; d < D; ++d) out_bf16[r * D + d] = 0;
+      if (lse) lse[r] = 0.0;
+      continue;
+    }
+    int g = h / G;
+    int64_t L = ctx_len[b];
+    const int32_t *par = parent + (int64_t)b * N;
+    /* row i of the topology matrix: allowed[j] = 1 iff j is i or an ancestor of i */
+    char *allowed = (char *)calloc((size_t)N, 1);
+    for (int j = i; j >= 0; j = par[j]) allowed[j] = 1;
+    int64_t n_keys = L + N;
+    double *s = (double *)malloc(sizeof(double) * (size_t)n_keys);
+    const uint16_t *qrow = q + (((int64_t)b * N + i) * Hq + h) * D;
+    double m = -INFINITY;
+    for (int64_t t = 0; t < n_keys; ++t) {
+      const uint16_t *krow;
+      if (t < L) {
+        krow = c.k + cache_row_offset(&c, b, t, g);
+      } else {
+        int j = (int)(t - L);
+        if (!allowed[j]) { s[t] = -INFINITY; continue; }
+        krow = k_tree + (((int64_t)b * N + j) * Hkv + g) * D;
+      }
+      double acc = 0.0;
+      for (int d = 0; d < D; ++d) acc += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
+      s[t] = scale * acc;
+      if (s[t] > m) m = s[t];
+    }
+    double denom = 0.0;
+    for (int64_t t = 0; t < n_keys; ++t) {
+      if (s[t] == -INFINITY) continue;
+      double w = exp(s[t] - m);
+      denom += w;
+      const uint16_t *vrow = (t < L) ? c.v + cache_row_offset(&c, b, t, g)
+                                     : v_tree + (((int64_t)b * N + (t - L)) * Hkv + g) * D;
+      for (int d = 0; d < D; ++d) o[d] += w * bf16_to_f64(vrow[d]);
+    }
+    for (int d = 0; d < D; ++d) o[d] /= denom;
+    if (out_bf16) for (int d = 0; d < D; ++d) out_bf16[r * D + d] = f64_to_bf16(o[d]);
+    if (lse) lse[r] = m + log(denom);
+    free(s);
+    free(allowed);
+  }
+  return 0;
+}
+
+/* ids[r] = index of the first strict maximum of row r (rows of `vocab` bf16 values, stride ld). */
+int orc_argmax(int64_t n_rows, int vocab, int64_t ld, const uint16_t *logits, int32_t *ids) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < n_rows; ++r) {
+    const uint16_t *row = logits + r * ld;
+    double best = bf16_to_f64(row[0]);
+    int32_t arg = 0;
+    for (int v = 1; v < vocab; ++v) {
+      double x = bf16_to_f64(row[v]);
+      if (x > best) { best = x; arg = v; }
+    }
+    ids[r] = arg;
+  }
+  return 0;
+}
+
+/*
+ * Greedy acceptance walk.  Node 0 is the root (the token the target emitted last; always
+ * accepted).  From the current node, the target's choice is ids[cur]; the drafted child carrying
+ * exactly that token (lowest index if the precondition of distinct siblings is broken) is
+ * accepted and becomes current; otherwise the walk ends.  next_token = ids[last accepted].
+ * Malformed parent[] (node 0 not the only root, parent[i] >= i or < -1) or a path longer than
+ * path_cap: status = ORC_ERR_TREE, accept_len = 0, next_token = -1, accept_idx all -1.
+ */
+int orc_accept_walk(int B, int N, int path_cap, const int32_t *parent, const int32_t *tokens,
+                    const int32_t *ids, int32_t *accept_len, int32_t *accept_idx,
+                    int32_t *next_token, int32_t *status) {
+  for (int b = 0; b < B; ++b) {
+    const int32_t *par = parent + (int64_t)b * N, *tok = tokens + (int64_t)b * N;
+    const int32_t *id = ids + (int64_t)b * N;
+    int32_t *path = accept_idx + (int64_t)b * path_cap;
+    for (int j = 0; j < path_cap; ++j) path[j] = -1;
+    status[b] = ORC_OK;
+    int ok = tree_ok(par, N, 0) && path_cap >= 1;
+    int len = 0, cur = 0;
+    if (ok) {
+      path[len++] = 0;
+      for (;;) {
+        int t = id[cur], found = -1;
+        for (int cnode = cur + 1; cnode < N; ++cnode)
+          if (par[cnode] == cur && tok[cnode] == t) { found = cnode; break; }
+        if (found < 0) break;
+        if (len == path_cap) { ok = 0; break; }
+        path[len++] = found;
+        cur = found;
+      }
+    }
+    if (!ok) {
+      for (int j = 0; j < path_cap; ++j) path[j] = -1;
+      status[b] = ORC_ERR_TREE;
+      accept_len[b] = 0;
+      next_token[b] = -1;
+    } else {
+      accept_len[b] = len;
+      next_token[b] = id[cur];
+    }
+  }
+  return 0;
+}
+
+/*
+ * Commit: cache rows ctx_len[b] + j  <-  tree rows accept_idx[b][j], j < accept_len[b], K and V,
+ * every kv head.  ctx_len_out[b] = ctx_len[b] + accept_len[b].  The cache buffers are modified in
+ * place (the caller passes copies).  A sequence whose accepted rows would not fit its capacity
+ * (contiguous: cap_tokens; paged: its block-table entries must exist and be valid), or whose
+ * accept_len / accept_idx are out of range, is left untouched: status = ORC_ERR_TREE and
+ * ctx_len_out[b] = ctx_len[b].
+ */
+int orc_kv_commit(int B, int N, int Hkv, int D, int path_cap, uint16_t *kc, uint16_t *vc, int paged,
+                  int cap_tokens, int page_size, int n_pages, int max_pages,
+                  const int32_t *block_table, const uint16_t *k_tree, const uint16_t *v_tree,
+                  const int32_t *accept_idx, const int32_t *accept_len, const int32_t *ctx_len,
+                  int32_t *ctx_len_out, int32_t *status) {
+  orc_cache c = {kc, vc, paged, cap_tokens, page_size, max_pages, Hkv, D, block_table};
+  for (int b = 0; b < B; ++b) {
+    int64_t L = ctx_len[b];
+    int len = accept_len[b];
+    int ok = (L >= 0) && (len >= 0) && (len <= path_cap);
+    for (int j = 0; ok && j < len; ++j) {
+      int a = accept_idx[(int64_t)b * path_cap + j];
+      if (a < 0 || a >= N) ok = 0;
+      int64_t t = L + j;
+      if (paged) {
+        if (t / page_size >= max_pages) ok = 0;
+        else {
+          int pg = block_table[(int64_t)b * max_pages + t / page_size];
+          if (pg < 0 || pg >= n_pages) ok = 0;
+        }
+      } else if (t >= cap_tokens) ok = 0;
+    }
+    if (!ok) { status[b] = ORC_ERR_TREE; ctx_len_out[b] = (int32_t)L; continue; }
+    status[b] = ORC_OK;
+    for (int j = 0; j < len; ++j) {
+      int a = accept_idx[(int64_t)b * path_cap + j];
+      for (int g = 0; g < Hkv; ++g) {
+        int64_t dst = cache_row_offset(&c, b, L + j, g);
+        int64_t src = (((int64_t)b * N + a) * Hkv + g) * D;
+        memcpy(kc + dst, k_tree + src, sizeof(uint16_t) * (size_t)D);
+        memcpy(vc + dst, v_tree + src, sizeof(uint16_t) * (size_t)D);
+      }
+    }
+    ctx_len_out[b] = (int32_t)(L + len);
+  }
+  return 0;
+}
+
+/* Exposed so a test can pin the rounding helper against an independent bf16 conversion. */
+uint16_t orc_f64_to_bf16(double d) { return f64_to_bf16(d); }
