@@ -1,0 +1,209 @@
+/*
+ * clv - tree verification for Clover-2-style speculative decoding on one B200 (sm_100a).
+ *
+ * The library implements the target model's verification step that the paper describes in
+ * Sec. 2.1 ("Speculative Decoding and Tree Attention"): the target ingests all N tokens of a draft
+ * token tree at once, attention uses the tree's topology matrix as its causal mask, wrong drafts
+ * are filtered out, and the result equals plain decoding.  Four stream-ordered calls cover it:
+ *
+ *   clv_tree_attn      tree-masked attention of the N tree tokens against the committed KV cache
+ *                      and against their own ancestors            (Sec. 2.1, Fig. 2 caption;
+ *                      the mask is derived from parent[] on chip, cf. App. A.1 "compressed tree
+ *                      mask": the N x N matrix never exists in memory)
+ *   clv_accept_argmax  the target's greedy choice per tree node   (Sec. 4.2: temperature 0 is
+ *                      greedy decoding of the target)
+ *   clv_accept_walk    longest root-to-node path the target agrees with (Sec. 2.1 verification
+ *                      phase; greedy rule of the tree-sampling algorithm adopted in Sec. 4.1)
+ *   clv_kv_commit      append the accepted nodes' K/V rows to the cache (implied by the
+ *                      equivalence requirement of Sec. 2.1: afterwards the cache holds what plain
+ *                      decoding of the accepted tokens would hold)
+ *
+ * Conventions
+ *   - Plain C ABI.  Every pointer is a DEVICE pointer unless the comment says "host".
+ *     The two descriptor structs live in host memory and are read during the call only.
+ *   - The caller owns every buffer, including the workspace.  The library allocates no device
+ *     memory, never synchronises, and only enqueues work on the given stream (a cudaStream_t
+ *     passed as void*; NULL = the legacy default stream).
+ *   - Inputs are const.  Only the documented outputs are written; clv_kv_commit writes cache
+ *     rows [ctx_len[b], ctx_len[b] + accept_len[b]) of each sequence and nothing else.
+ *   - bf16 tensors are dense, innermost dimension contiguous, base 16-byte aligned.
+ *   - Host-detectable mistakes return an error code and enqueue nothing.  Mistakes only the
+ *     device can see (a malformed parent[], a context that does not fit its capacity, an invalid
+ *     block-table entry) never trap: the sequence is skipped and CLV_ERR_TREE is written to its
+ *     slot of the caller's int32 status[batch] array (0 = fine).
+ *   - Notation: B sequences, N tree nodes per sequence (node 0 = root = the last token the target
+ *     emitted; parent[b][0] = -1, parent[b][i] in [0, i)), Hq query heads, Hkv KV heads,
+ *     G = Hq / Hkv, D = 128, L_b = ctx_len[b] committed tokens.
+ */
+#ifndef CLV_H_
+#define CLV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t clv_status;
+enum {
+  CLV_OK = 0,
+  CLV_ERR_NULL = 1,        /* a required pointer is NULL                                        */
+  CLV_ERR_SHAPE = 2,       /* non-positive size, Hq not a multiple of Hkv, ld < vocab, ...      */
+  CLV_ERR_UNSUPPORTED = 3, /* head_dim != 128, n_nodes > 128, page_size != 64, forbidden alias  */
+  CLV_ERR_ALIGN = 4,       /* a tensor base (or logits row stride) is not 16-byte aligned       */
+  CLV_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than clv_workspace_bytes()              */
+  CLV_ERR_CUDA = 6,        /* a CUDA runtime call failed; see clv_last_cuda_error()             */
+  CLV_ERR_TREE = 7,        /* device status[] only: malformed tree or capacity exceeded         */
+  CLV_ERR_TIMEOUT = 8      /* device status[] only: a bounded on-chip wait gave up              */
+};
+
+#define CLV_MAX_NODES 128
+#define CLV_HEAD_DIM 128
+#define CLV_PAGE_SIZE 64
+
+/* Shape of one verify step (host memory). */
+typedef struct {
+  int32_t batch;      /* B >= 1                                                    */
+  int32_t n_nodes;    /* N in [1, 128]                                             */
+  int32_t n_q_heads;  /* Hq, a multiple of n_kv_heads                              */
+  int32_t n_kv_heads; /* Hkv                                                       */
+  int32_t head_dim;   /* must be 128                                               */
+  int32_t vocab;      /* V, used by clv_accept_argmax only                         */
+  int32_t path_cap;   /* columns of accept_idx; >= (maximum tree depth + 1)        */
+} clv_shape;
+
+/* KV cache descriptor (host memory; k, v and block_table are device pointers). */
+typedef struct {
+  void* k;            /* contiguous: [B, cap_tokens, Hkv, 128] bf16                          */
+  void* v;            /* paged:      [n_pages, 64, Hkv, 128] bf16                            */
+  int32_t paged;      /* 0 contiguous, 1 paged                                               */
+  int32_t cap_tokens; /* contiguous: rows per sequence                                       */
+  int32_t page_size;  /* paged: must be 64                                                   */
+  int32_t n_pages;    /* paged: pages in the pool                                            */
+  int32_t max_pages_per_seq;  /* paged: columns of block_table                               */
+  const int32_t* block_table; /* paged: [B, max_pages_per_seq], logical page -> pool page    */
+} clv_kv_cache;
+
+/*
+ * Workspace.  clv_tree_attn and clv_accept_argmax split their work over more thread blocks than
+ * there are independent outputs and combine the pieces through the workspace.
+ * clv_workspace_bytes: bytes needed for this shape with contexts up to max_ctx_len (host call).
+ * clv_workspace_init : must be enqueued ONCE on a fresh workspace before its first use (it clears
+ *                      the arrival counters; every call leaves them cleared again).  One workspace
+ *                      serves both calls and any shape it is large enough for, but calls that
+ *                      share a workspace must not overlap on the device.
+ */
+size_t clv_workspace_bytes(const clv_shape* shape, const clv_kv_cache* cache, int32_t max_ctx_len);
+clv_status clv_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Tree attention (Sec. 2.1; Fig. 2 caption).  For every sequence b, node i and query head h:
+ *   keys   = cache rows 0 .. L_b-1 of kv head h / G, then the tree rows j that are i itself or an
+ *            ancestor of i (row i of the tree's topology matrix),
+ *   out    = softmax(softmax_scale * q . k) . v   over those keys, fp32 accumulation, rounded to
+ *            bf16 (nearest even);   lse = natural-log sum-exp of the scaled scores (optional).
+ * q/k are taken as given (rotary positions L_b + depth(i) are the caller's business).
+ * Several roots (extra -1 parents) are accepted here.  L_b = 0 is allowed.
+ * status[b] = CLV_ERR_TREE if parent[b] is malformed, L_b < 0, L_b exceeds the cache capacity or
+ * a needed block-table entry is outside [0, n_pages); that sequence's outputs are unspecified.
+ * max_ctx_len (host): an upper bound of ctx_len[], used only to choose the split count; the
+ * result does not depend on it.
+ */
+clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache,
+                         const void* q,        /* bf16 [B, N, Hq, 128]            */
+                         const void* k_tree,   /* bf16 [B, N, Hkv, 128]           */
+                         const void* v_tree,   /* bf16 [B, N, Hkv, 128]           */
+                         const int32_t* parent,  /* [B, N]                        */
+                         const int32_t* ctx_len, /* [B]                           */
+                         int32_t max_ctx_len, float softmax_scale,
+                         void* out,            /* bf16 [B, N, Hq, 128]            */
+                         float* lse,           /* fp32 [B, N, Hq] or NULL         */
+                         int32_t* status,      /* [B]                             */
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Greedy target choice (Sec. 4.2, temperature 0): argmax_ids[b][i] = the lowest v that maximises
+ * logits[b][i][v], v < vocab.  +0 and -0 compare equal; NaN entries are ignored (treated as
+ * -infinity); a row of only -infinity/NaN gives 0.  ld = row stride in elements, a multiple of 8.
+ */
+clv_status clv_accept_argmax(const clv_shape* shape,
+                             const void* logits, /* bf16 [B*N, ld]               */
+                             int64_t ld,
+                             int32_t* argmax_ids, /* [B, N]                      */
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Greedy acceptance walk (Sec. 2.1 verification phase; Sec. 4.1).  Start at the root; at node cur
+ * the target wants argmax_ids[cur]; the child of cur whose drafted token equals it (the lowest
+ * index if siblings repeat a token) is accepted and becomes cur; otherwise stop.
+ *   accept_len[b]  nodes on the accepted path, root included (>= 1)
+ *   accept_idx[b]  their node indices in path order, padded with -1 to path_cap columns
+ *   next_token[b]  argmax_ids of the last accepted node (the token the target emits next)
+ * status[b] = CLV_ERR_TREE when parent[b] is malformed (node 0 must be the only root) or the path
+ * does not fit path_cap; then accept_len = 0, next_token = -1, accept_idx = -1.
+ */
+clv_status clv_accept_walk(const clv_shape* shape, const int32_t* parent /* [B,N] */,
+                           const int32_t* tokens /* [B,N] */, const int32_t* argmax_ids /* [B,N] */,
+                           int32_t* accept_len /* [B] */, int32_t* accept_idx /* [B,path_cap] */,
+                           int32_t* next_token /* [B] */, int32_t* status /* [B] */,
+                           void* cuda_stream);
+
+/*
+ * KV commit (from the equivalence requirement of Sec. 2.1).  For j < accept_len[b]:
+ *   cache row (L_b + j)  <-  tree row accept_idx[b][j], K and V, all Hkv heads;
+ *   ctx_len_out[b] = L_b + accept_len[b]   (ctx_len_out may be the same array as ctx_len).
+ * k_tree / v_tree must not overlap the cache buffers (CLV_ERR_UNSUPPORTED if they do).
+ * status[b] = CLV_ERR_TREE and the sequence is left untouched (ctx_len_out[b] = L_b) if the rows
+ * do not fit (contiguous: cap_tokens; paged: block-table entry missing or invalid) or accept_len /
+ * accept_idx are out of range.
+ */
+clv_status clv_kv_commit(const clv_shape* shape, const clv_kv_cache* cache,
+                         const void* k_tree, const void* v_tree, /* bf16 [B, N, Hkv, 128] */
+                         const int32_t* accept_idx /* [B,path_cap] */,
+                         const int32_t* accept_len /* [B] */, const int32_t* ctx_len /* [B] */,
+                         int32_t* ctx_len_out /* [B] */, int32_t* status /* [B] */,
+                         void* cuda_stream);
+
+/*
+ * One whole verify step from HOST buffers (Sec. 2.1: attention, greedy choice, walk, commit in
+ * that order).  The per-step inputs are copied from (preferably pinned) host memory to the
+ * caller's device staging buffer, the four calls above run, and the results are copied back; all
+ * on the given stream, without a synchronisation (results are valid once the stream has drained).
+ * The KV cache and ctx_len stay on the device; ctx_len is advanced in place.
+ */
+typedef struct {          /* host memory; every pointer is a HOST pointer */
+  const void* q;          /* bf16 [B, N, Hq, 128]   */
+  const void* k_tree;     /* bf16 [B, N, Hkv, 128]  */
+  const void* v_tree;     /* bf16 [B, N, Hkv, 128]  */
+  const int32_t* parent;  /* [B, N]                 */
+  const int32_t* tokens;  /* [B, N]                 */
+  const void* logits;     /* bf16 [B*N, ld]         */
+  int64_t ld;
+} clv_host_inputs;
+
+typedef struct {          /* host memory; every pointer is a HOST pointer, written asynchronously */
+  void* out;              /* bf16 [B, N, Hq, 128]   */
+  int32_t* argmax_ids;    /* [B, N]                 */
+  int32_t* accept_len;    /* [B]                    */
+  int32_t* accept_idx;    /* [B, path_cap]          */
+  int32_t* next_token;    /* [B]                    */
+  int32_t* status;        /* [3, B]: attention, walk, commit */
+} clv_host_outputs;
+
+size_t clv_staging_bytes(const clv_shape* shape, int64_t ld);
+clv_status clv_verify_step_host(const clv_shape* shape, const clv_kv_cache* cache,
+                                const clv_host_inputs* in, const clv_host_outputs* out,
+                                int32_t* ctx_len /* device [B], updated in place */,
+                                int32_t max_ctx_len, float softmax_scale,
+                                void* staging, size_t staging_bytes, /* device */
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+const char* clv_status_string(clv_status s);
+int clv_last_cuda_error(void); /* cudaError_t of the most recent CLV_ERR_CUDA on this thread */
+int clv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLV_H_ */

@@ -1,0 +1,171 @@
+// Per-node greedy choice: argmax over the vocabulary of each logits row (Sec. 4.2, T = 0).
+//
+// Pure HBM stream: every logit is read once with 16-byte loads that bypass L1.  A row is cut into
+// `chunks` pieces so that the grid covers the machine even for few rows; each block reduces its
+// piece to one (value, lowest index) pair, packs it into a 64-bit key whose unsigned order is
+// "higher value first, then lower index", and the last block to arrive for a row takes the
+// maximum key.  The result is independent of the chunking and of block scheduling.
+#include <limits.h>
+
+#include "clv_internal.cuh"
+
+namespace clv {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;  // 16-byte loads in flight per thread
+
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) {
+  return *reinterpret_cast<__nv_bfloat162*>(&u);
+}
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+// Running (best value, lowest index of it) of one thread; indices are visited in ascending order.
+struct Best {
+  float v;
+  int i;
+};
+
+__device__ __forceinline__ void take_vec(Best& b, const uint4& w, int idx0) {
+  // maximum of the 8 values (NaN operands are dropped by max.bf16x2)
+  __nv_bfloat162 m = __hmax2(__hmax2(as_bf162(w.x), as_bf162(w.y)),
+                             __hmax2(as_bf162(w.z), as_bf162(w.w)));
+  float vm = fmaxf(__low2float(m), __high2float(m));
+  if (vm > b.v) {  // rare after the first few vectors
+    b.v = vm;
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+    int at = 7;
+#pragma unroll
+    for (int e = 3; e >= 0; --e) {  // descending, so the lowest matching position survives
+      if (bf16hi(u[e]) == vm) at = 2 * e + 1;
+      if (bf16lo(u[e]) == vm) at = 2 * e;
+    }
+    b.i = idx0 + at;
+  }
+}
+
+__device__ __forceinline__ bool better(float v, int i, float bv, int bi) {
+  return (v > bv) || (v == bv && i < bi);
+}
+
+__device__ __forceinline__ unsigned long long pack_key(float v, int i) {
+  if (v == 0.0f) v = 0.0f;  // -0 and +0 are the same value: one bit pattern
+  uint32_t f = __float_as_uint(v);
+  uint32_t ord = (f & 0x80000000u) ? ~f : (f | 0x80000000u);
+  return ((unsigned long long)ord << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+}
+
+struct Params {
+  const uint16_t* logits;
+  int64_t ld;
+  int vocab;
+  int chunks;
+  int chunk_elems;
+  int32_t* ids;
+  unsigned* tickets;
+  unsigned long long* partial;
+};
+
+__global__ void __launch_bounds__(kThreads) argmax_kernel(Params p) {
+  const int row = blockIdx.x / p.chunks;
+  const int chunk = blockIdx.x - row * p.chunks;
+  const int begin = chunk * p.chunk_elems;
+  const int end = min(p.vocab, begin + p.chunk_elems);
+  const uint16_t* base = p.logits + (int64_t)row * p.ld;
+  const int nvec = (end - begin) >> 3;
+  const uint4* vp = reinterpret_cast<const uint4*>(base + begin);
+  const int tid = threadIdx.x;
+
+  Best best = {-INFINITY, INT_MAX};
+  int i = tid;
+  for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
+    uint4 w[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) w[u] = ld_stream16(vp + i + u * kThreads);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) take_vec(best, w[u], begin + 8 * (i + u * kThreads));
+  }
+  for (; i < nvec; i += kThreads) take_vec(best, ld_stream16(vp + i), begin + 8 * i);
+  // ragged end of the row (vocab not a multiple of 8): at most 7 scalars, after all vectors
+  {
+    const int t0 = begin + 8 * nvec + tid;
+    if (t0 < end) {
+      float x = __uint_as_float((uint32_t)base[t0] << 16);
+      if (x > best.v) { best.v = x; best.i = t0; }
+    }
+  }
+
+  // block reduction in the order (value descending, index ascending)
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xFFFFFFFFu, best.v, o);
+    int oi = __shfl_xor_sync(0xFFFFFFFFu, best.i, o);
+    if (better(ov, oi, best.v, best.i)) { best.v = ov; best.i = oi; }
+  }
+  __shared__ float sv[kThreads / 32];
+  __shared__ int si[kThreads / 32];
+  if ((tid & 31) == 0) { sv[tid >> 5] = best.v; si[tid >> 5] = best.i; }
+  __syncthreads();
+  if (tid != 0) return;
+  for (int w = 1; w < kThreads / 32; ++w)
+    if (better(sv[w], si[w], best.v, best.i)) { best.v = sv[w]; best.i = si[w]; }
+
+  unsigned long long key = pack_key(best.v, best.i);
+  if (p.chunks > 1) {
+    unsigned long long* mine = p.partial + (size_t)row * p.chunks;
+    __stcg(mine + chunk, key);
+    __threadfence();
+    const unsigned arrived = atomicInc(p.tickets + row, (unsigned)p.chunks - 1);  // wraps to 0
+    if (arrived != (unsigned)p.chunks - 1) return;
+    __threadfence();
+    for (int c = 0; c < p.chunks; ++c) {
+      unsigned long long k = __ldcg(mine + c);
+      key = k > key ? k : key;
+    }
+  }
+  int idx = (int)(0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull));
+  p.ids[row] = (idx == INT_MAX) ? 0 : idx;  // a row of only -inf / NaN: first index
+}
+
+}  // namespace
+
+ArgmaxPlan argmax_plan(int rows, int vocab) {
+  ArgmaxPlan pl;
+  pl.rows = rows;
+  // about 32 KB of logits per block, but enough blocks to cover the machine a few times
+  const int unit = kThreads * 8;  // elements one pass of the block covers
+  int chunk_elems = 8 * unit;     // 16384 elements = 32 KB
+  const int want_blocks = 4 * sm_count();
+  while (chunk_elems > unit && (int64_t)rows * ((vocab + chunk_elems - 1) / chunk_elems) < want_blocks)
+    chunk_elems >>= 1;
+  pl.chunk_elems = chunk_elems;
+  pl.chunks = (vocab + chunk_elems - 1) / chunk_elems;
+  pl.scratch_bytes = pl.chunks > 1 ? sizeof(unsigned long long) * (size_t)rows * pl.chunks : 0;
+  return pl;
+}
+
+cudaError_t launch_argmax(const ArgmaxPlan& plan, const void* logits, int64_t ld, int vocab,
+                          int32_t* ids, unsigned* tickets, void* scratch, cudaStream_t stream) {
+  Params p;
+  p.logits = static_cast<const uint16_t*>(logits);
+  p.ld = ld;
+  p.vocab = vocab;
+  p.chunks = plan.chunks;
+  p.chunk_elems = plan.chunk_elems;
+  p.ids = ids;
+  p.tickets = tickets;
+  p.partial = static_cast<unsigned long long*>(scratch);
+  argmax_kernel<<<(unsigned)((int64_t)plan.rows * plan.chunks), kThreads, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace clv

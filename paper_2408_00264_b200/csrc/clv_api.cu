@@ -1,0 +1,280 @@
+// C ABI of libclv: argument checks and dispatch.  No device memory is allocated here, nothing
+// synchronises, every launch goes to the caller's stream.
+#include <stdint.h>
+#include <string.h>
+
+#include "clv_internal.cuh"
+
+namespace clv {
+
+static thread_local int g_last_cuda_error = 0;
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      n = 148;  // B200; used for sizing only when no device can be queried
+    (void)cudaGetLastError();
+  }
+  return n;
+}
+
+static clv_status cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return CLV_ERR_CUDA;
+}
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static clv_status check_shape(const clv_shape* s) {
+  if (!s) return CLV_ERR_NULL;
+  if (s->batch < 1 || s->n_nodes < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1) return CLV_ERR_SHAPE;
+  if (s->n_q_heads % s->n_kv_heads) return CLV_ERR_SHAPE;
+  if (s->head_dim != CLV_HEAD_DIM || s->n_nodes > CLV_MAX_NODES) return CLV_ERR_UNSUPPORTED;
+  return CLV_OK;
+}
+
+static clv_status check_cache(const clv_kv_cache* c) {
+  if (!c || !c->k || !c->v) return CLV_ERR_NULL;
+  if (!aligned16(c->k) || !aligned16(c->v)) return CLV_ERR_ALIGN;
+  if (c->paged) {
+    if (!c->block_table) return CLV_ERR_NULL;
+    if (c->page_size != CLV_PAGE_SIZE) return CLV_ERR_UNSUPPORTED;
+    if (c->n_pages < 1 || c->max_pages_per_seq < 1) return CLV_ERR_SHAPE;
+  } else if (c->cap_tokens < 1) {
+    return CLV_ERR_SHAPE;
+  }
+  return CLV_OK;
+}
+
+static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace clv
+
+using namespace clv;
+
+extern "C" {
+
+size_t clv_workspace_bytes(const clv_shape* shape, const clv_kv_cache* cache, int32_t max_ctx_len) {
+  (void)cache;
+  if (check_shape(shape) != CLV_OK) return 0;
+  if (max_ctx_len < 0) max_ctx_len = 0;
+  const AttnPlan ap = attn_plan(*shape, max_ctx_len);
+  size_t scratch = ap.scratch_bytes;
+  if (shape->vocab > 0) {
+    const ArgmaxPlan gp = argmax_plan(shape->batch * shape->n_nodes, shape->vocab);
+    if (gp.scratch_bytes > scratch) scratch = gp.scratch_bytes;
+  }
+  return kWsFixedBytes + round_up(scratch, 256);
+}
+
+clv_status clv_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!workspace) return CLV_ERR_NULL;
+  if (workspace_bytes < kWsFixedBytes) return CLV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  cudaError_t e = cudaMemsetAsync(workspace, 0, kWsFixedBytes, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, const void* q,
+                         const void* k_tree, const void* v_tree, const int32_t* parent,
+                         const int32_t* ctx_len, int32_t max_ctx_len, float softmax_scale,
+                         void* out, float* lse, int32_t* status, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  st = check_cache(cache);
+  if (st != CLV_OK) return st;
+  if (!q || !k_tree || !v_tree || !parent || !ctx_len || !out || !status) return CLV_ERR_NULL;
+  if (!aligned16(q) || !aligned16(k_tree) || !aligned16(v_tree) || !aligned16(out)) return CLV_ERR_ALIGN;
+  if (max_ctx_len < 0) return CLV_ERR_SHAPE;
+  const AttnPlan plan = attn_plan(*shape, max_ctx_len);
+  if (plan.splits > 1) {
+    if (!workspace || workspace_bytes < kWsFixedBytes + plan.scratch_bytes) return CLV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  }
+  cudaError_t e = launch_tree_attn(plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len,
+                                   softmax_scale, out, lse, status,
+                                   workspace ? ws_tickets(workspace) : nullptr,
+                                   workspace ? ws_scratch(workspace) : nullptr,
+                                   static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+clv_status clv_accept_argmax(const clv_shape* shape, const void* logits, int64_t ld,
+                             int32_t* argmax_ids, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  if (!logits || !argmax_ids) return CLV_ERR_NULL;
+  if (shape->vocab < 1 || ld < shape->vocab) return CLV_ERR_SHAPE;
+  if (!aligned16(logits) || (ld % 8) != 0) return CLV_ERR_ALIGN;
+  const int64_t rows = (int64_t)shape->batch * shape->n_nodes;
+  if (rows > kTickets) return CLV_ERR_UNSUPPORTED;
+  const ArgmaxPlan plan = argmax_plan((int)rows, shape->vocab);
+  if (plan.chunks > 1) {
+    if (!workspace || workspace_bytes < kWsFixedBytes + plan.scratch_bytes) return CLV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  }
+  cudaError_t e = launch_argmax(plan, logits, ld, shape->vocab, argmax_ids,
+                                workspace ? ws_tickets(workspace) : nullptr,
+                                workspace ? ws_scratch(workspace) : nullptr,
+                                static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+clv_status clv_accept_walk(const clv_shape* shape, const int32_t* parent, const int32_t* tokens,
+                           const int32_t* argmax_ids, int32_t* accept_len, int32_t* accept_idx,
+                           int32_t* next_token, int32_t* status, void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  if (!parent || !tokens || !argmax_ids || !accept_len || !accept_idx || !next_token || !status)
+    return CLV_ERR_NULL;
+  if (shape->path_cap < 1) return CLV_ERR_SHAPE;
+  cudaError_t e = launch_walk(*shape, parent, tokens, argmax_ids, accept_len, accept_idx, next_token,
+                              status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + nb && y < x + na;
+}
+
+clv_status clv_kv_commit(const clv_shape* shape, const clv_kv_cache* cache, const void* k_tree,
+                         const void* v_tree, const int32_t* accept_idx, const int32_t* accept_len,
+                         const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
+                         void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  st = check_cache(cache);
+  if (st != CLV_OK) return st;
+  if (!k_tree || !v_tree || !accept_idx || !accept_len || !ctx_len || !ctx_len_out || !status)
+    return CLV_ERR_NULL;
+  if (!aligned16(k_tree) || !aligned16(v_tree)) return CLV_ERR_ALIGN;
+  if (shape->path_cap < 1) return CLV_ERR_SHAPE;
+  const size_t row = (size_t)shape->n_kv_heads * CLV_HEAD_DIM * 2;
+  const size_t tree_bytes = (size_t)shape->batch * shape->n_nodes * row;
+  const size_t cache_bytes = cache->paged ? (size_t)cache->n_pages * CLV_PAGE_SIZE * row
+                                          : (size_t)shape->batch * cache->cap_tokens * row;
+  if (overlaps(k_tree, tree_bytes, cache->k, cache_bytes) ||
+      overlaps(k_tree, tree_bytes, cache->v, cache_bytes) ||
+      overlaps(v_tree, tree_bytes, cache->k, cache_bytes) ||
+      overlaps(v_tree, tree_bytes, cache->v, cache_bytes))
+    return CLV_ERR_UNSUPPORTED;  // a destination row could be another thread's source row
+  cudaError_t e = launch_commit(*shape, *cache, k_tree, v_tree, accept_idx, accept_len, ctx_len,
+                                ctx_len_out, status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+// ---- whole step from host buffers ---------------------------------------------------------------
+namespace {
+struct Staging {
+  size_t q, k_tree, v_tree, parent, tokens, logits, out, ids, alen, aidx, next, status, total;
+};
+Staging staging_layout(const clv_shape& s, int64_t ld) {
+  Staging L;
+  const size_t B = s.batch, N = s.n_nodes;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o += round_up(bytes, 256); return at; };
+  L.q = take(B * N * s.n_q_heads * CLV_HEAD_DIM * 2);
+  L.k_tree = take(B * N * s.n_kv_heads * CLV_HEAD_DIM * 2);
+  L.v_tree = take(B * N * s.n_kv_heads * CLV_HEAD_DIM * 2);
+  L.parent = take(B * N * 4);
+  L.tokens = take(B * N * 4);
+  L.logits = take(B * N * (size_t)ld * 2);
+  L.out = take(B * N * s.n_q_heads * CLV_HEAD_DIM * 2);
+  L.ids = take(B * N * 4);
+  L.alen = take(B * 4);
+  L.aidx = take(B * (size_t)s.path_cap * 4);
+  L.next = take(B * 4);
+  L.status = take(3 * B * 4);
+  L.total = o;
+  return L;
+}
+}  // namespace
+
+size_t clv_staging_bytes(const clv_shape* shape, int64_t ld) {
+  if (check_shape(shape) != CLV_OK || ld < 1 || shape->path_cap < 1) return 0;
+  return staging_layout(*shape, ld).total;
+}
+
+clv_status clv_verify_step_host(const clv_shape* shape, const clv_kv_cache* cache,
+                                const clv_host_inputs* in, const clv_host_outputs* out,
+                                int32_t* ctx_len, int32_t max_ctx_len, float softmax_scale,
+                                void* staging, size_t staging_bytes, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  if (!in || !out || !ctx_len || !staging) return CLV_ERR_NULL;
+  if (!in->q || !in->k_tree || !in->v_tree || !in->parent || !in->tokens || !in->logits ||
+      !out->out || !out->argmax_ids || !out->accept_len || !out->accept_idx || !out->next_token ||
+      !out->status)
+    return CLV_ERR_NULL;
+  if (shape->path_cap < 1 || in->ld < shape->vocab || shape->vocab < 1) return CLV_ERR_SHAPE;
+  if (!aligned16(staging)) return CLV_ERR_ALIGN;
+  const Staging L = staging_layout(*shape, in->ld);
+  if (staging_bytes < L.total) return CLV_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* d = static_cast<char*>(staging);
+  const size_t B = shape->batch, N = shape->n_nodes;
+  const size_t qb = B * N * shape->n_q_heads * CLV_HEAD_DIM * 2;
+  const size_t tb = B * N * shape->n_kv_heads * CLV_HEAD_DIM * 2;
+  cudaError_t e;
+#define CLV_COPY(dst, src, n, kind) \
+  if ((e = cudaMemcpyAsync(dst, src, n, kind, s)) != cudaSuccess) return cuda_fail(e)
+  CLV_COPY(d + L.q, in->q, qb, cudaMemcpyHostToDevice);
+  CLV_COPY(d + L.k_tree, in->k_tree, tb, cudaMemcpyHostToDevice);
+  CLV_COPY(d + L.v_tree, in->v_tree, tb, cudaMemcpyHostToDevice);
+  CLV_COPY(d + L.parent, in->parent, B * N * 4, cudaMemcpyHostToDevice);
+  CLV_COPY(d + L.tokens, in->tokens, B * N * 4, cudaMemcpyHostToDevice);
+  CLV_COPY(d + L.logits, in->logits, B * N * (size_t)in->ld * 2, cudaMemcpyHostToDevice);
+  int32_t* dstat = reinterpret_cast<int32_t*>(d + L.status);
+  st = clv_tree_attn(shape, cache, d + L.q, d + L.k_tree, d + L.v_tree,
+                     reinterpret_cast<int32_t*>(d + L.parent), ctx_len, max_ctx_len, softmax_scale,
+                     d + L.out, nullptr, dstat, workspace, workspace_bytes, cuda_stream);
+  if (st != CLV_OK) return st;
+  st = clv_accept_argmax(shape, d + L.logits, in->ld, reinterpret_cast<int32_t*>(d + L.ids),
+                         workspace, workspace_bytes, cuda_stream);
+  if (st != CLV_OK) return st;
+  st = clv_accept_walk(shape, reinterpret_cast<int32_t*>(d + L.parent),
+                       reinterpret_cast<int32_t*>(d + L.tokens), reinterpret_cast<int32_t*>(d + L.ids),
+                       reinterpret_cast<int32_t*>(d + L.alen), reinterpret_cast<int32_t*>(d + L.aidx),
+                       reinterpret_cast<int32_t*>(d + L.next), dstat + B, cuda_stream);
+  if (st != CLV_OK) return st;
+  st = clv_kv_commit(shape, cache, d + L.k_tree, d + L.v_tree, reinterpret_cast<int32_t*>(d + L.aidx),
+                     reinterpret_cast<int32_t*>(d + L.alen), ctx_len, ctx_len, dstat + 2 * B,
+                     cuda_stream);
+  if (st != CLV_OK) return st;
+  CLV_COPY(out->out, d + L.out, qb, cudaMemcpyDeviceToHost);
+  CLV_COPY(out->argmax_ids, d + L.ids, B * N * 4, cudaMemcpyDeviceToHost);
+  CLV_COPY(out->accept_len, d + L.alen, B * 4, cudaMemcpyDeviceToHost);
+  CLV_COPY(out->accept_idx, d + L.aidx, B * (size_t)shape->path_cap * 4, cudaMemcpyDeviceToHost);
+  CLV_COPY(out->next_token, d + L.next, B * 4, cudaMemcpyDeviceToHost);
+  CLV_COPY(out->status, d + L.status, 3 * B * 4, cudaMemcpyDeviceToHost);
+#undef CLV_COPY
+  return CLV_OK;
+}
+
+const char* clv_status_string(clv_status s) {
+  switch (s) {
+    case CLV_OK: return "ok";
+    case CLV_ERR_NULL: return "a required pointer is NULL";
+    case CLV_ERR_SHAPE: return "invalid shape";
+    case CLV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case CLV_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case CLV_ERR_WORKSPACE: return "workspace missing or too small";
+    case CLV_ERR_CUDA: return "CUDA runtime error";
+    case CLV_ERR_TREE: return "malformed tree or capacity exceeded";
+    case CLV_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    default: return "unknown status";
+  }
+}
+
+int clv_last_cuda_error(void) { return g_last_cuda_error; }
+int clv_version(void) { return 100; }
+
+}  // extern "C"

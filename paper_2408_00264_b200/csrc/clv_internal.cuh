@@ -1,0 +1,61 @@
+// Internal declarations shared by the translation units of libclv (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "clv.h"
+
+namespace clv {
+
+// ---- workspace layout -------------------------------------------------------------------------
+// [0, 256)                     header (reserved)
+// [256, 256 + 4*kTickets)      arrival counters, zero between calls (self-resetting atomicInc)
+// [kWsFixedBytes, ...)         scratch for partial results (contents are garbage between calls)
+constexpr size_t kWsHeaderBytes = 256;
+constexpr int kTickets = 65536;
+constexpr size_t kWsFixedBytes = kWsHeaderBytes + sizeof(unsigned) * (size_t)kTickets;
+
+inline unsigned* ws_tickets(void* ws) {
+  return reinterpret_cast<unsigned*>(static_cast<char*>(ws) + kWsHeaderBytes);
+}
+inline void* ws_scratch(void* ws) { return static_cast<char*>(ws) + kWsFixedBytes; }
+
+// ---- argmax -----------------------------------------------------------------------------------
+struct ArgmaxPlan {
+  int rows;         // B * N
+  int chunks;       // thread blocks per row
+  int chunk_elems;  // multiple of 8
+  size_t scratch_bytes;
+};
+ArgmaxPlan argmax_plan(int rows, int vocab);
+cudaError_t launch_argmax(const ArgmaxPlan& plan, const void* logits, int64_t ld, int vocab,
+                          int32_t* ids, unsigned* tickets, void* scratch, cudaStream_t stream);
+
+// ---- walk / commit ----------------------------------------------------------------------------
+cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
+                        const int32_t* ids, int32_t* accept_len, int32_t* accept_idx,
+                        int32_t* next_token, int32_t* status, cudaStream_t stream);
+cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void* k_tree,
+                          const void* v_tree, const int32_t* accept_idx, const int32_t* accept_len,
+                          const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
+                          cudaStream_t stream);
+
+// ---- tree attention ---------------------------------------------------------------------------
+struct AttnPlan {
+  int m_tiles;   // row tiles per (sequence, kv head): ceil(G*N / rows per tile)
+  int splits;    // thread blocks along the key axis per row tile
+  size_t scratch_bytes;
+  int tickets;   // counters used
+};
+AttnPlan attn_plan(const clv_shape& s, int max_ctx_len);
+cudaError_t launch_tree_attn(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,
+                             const void* q, const void* k_tree, const void* v_tree,
+                             const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
+                             float* lse, int32_t* status, unsigned* tickets, void* scratch,
+                             cudaStream_t stream);
+
+int sm_count();
+
+}  // namespace clv

@@ -1,0 +1,155 @@
+// Greedy acceptance walk (Sec. 2.1 verification phase) and KV commit (equivalence requirement of
+// Sec. 2.1).  Both are latency-bound: one warp per sequence for the walk, one thread block per
+// sequence for the row copies.
+#include <limits.h>
+
+#include "clv_internal.cuh"
+
+namespace clv {
+namespace {
+
+// ------------------------------------------------------------------------------------ walk
+__global__ void __launch_bounds__(32) walk_kernel(int N, int path_cap, const int32_t* parent,
+                                                  const int32_t* tokens, const int32_t* ids,
+                                                  int32_t* accept_len, int32_t* accept_idx,
+                                                  int32_t* next_token, int32_t* status) {
+  __shared__ int sp[CLV_MAX_NODES], st[CLV_MAX_NODES], si[CLV_MAX_NODES], path[CLV_MAX_NODES];
+  const int b = blockIdx.x, lane = threadIdx.x;
+  const int64_t o = (int64_t)b * N;
+  bool bad = false;
+  for (int i = lane; i < N; i += 32) {
+    const int p = parent[o + i];
+    sp[i] = p;
+    st[i] = tokens[o + i];
+    si[i] = ids[o + i];
+    bad |= (i == 0) ? (p != -1) : (p < 0 || p >= i);  // node 0 is the only root
+  }
+  bad = __any_sync(0xFFFFFFFFu, bad) || path_cap < 1;
+  __syncwarp();
+  int len = 0, cur = 0;
+  if (!bad) {
+    if (lane == 0) path[0] = 0;
+    len = 1;
+    for (int step = 1; step < N; ++step) {  // a path has at most N nodes
+      const int want = si[cur];
+      int found = INT_MAX;
+      for (int c = cur + 1 + lane; c < N; c += 32)
+        if (sp[c] == cur && st[c] == want) { found = c; break; }
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) found = min(found, __shfl_xor_sync(0xFFFFFFFFu, found, s));
+      if (found == INT_MAX) break;
+      if (len == path_cap || len == CLV_MAX_NODES) { bad = true; break; }
+      if (lane == 0) path[len] = found;
+      ++len;
+      cur = found;
+    }
+  }
+  __syncwarp();
+  if (bad) len = 0;
+  for (int j = lane; j < path_cap; j += 32)
+    accept_idx[(int64_t)b * path_cap + j] = (j < len) ? path[j] : -1;
+  if (lane == 0) {
+    accept_len[b] = len;
+    next_token[b] = bad ? -1 : si[cur];
+    status[b] = bad ? CLV_ERR_TREE : CLV_OK;
+  }
+}
+
+// ------------------------------------------------------------------------------------ commit
+struct CommitParams {
+  uint4* kc;
+  uint4* vc;
+  const uint4* k_tree;
+  const uint4* v_tree;
+  const int32_t* block_table;
+  const int32_t* accept_idx;
+  const int32_t* accept_len;
+  const int32_t* ctx_len;
+  int32_t* ctx_len_out;
+  int32_t* status;
+  int N, path_cap, paged, cap_tokens, n_pages, max_pages;
+  int row_vec;  // 16-byte vectors per token row: Hkv * 128 * 2 / 16
+};
+
+__global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
+  __shared__ int s_src[CLV_MAX_NODES];
+  __shared__ long long s_dst[CLV_MAX_NODES];  // destination token row (global row index)
+  __shared__ int s_ok;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int L = p.ctx_len[b];
+  const int len = p.accept_len[b];
+  if (tid == 0) s_ok = (L >= 0 && len >= 0 && len <= p.path_cap && len <= CLV_MAX_NODES) ? 1 : 0;
+  __syncthreads();
+  if (s_ok) {
+    for (int j = tid; j < len; j += blockDim.x) {
+      const int a = p.accept_idx[(int64_t)b * p.path_cap + j];
+      const long long t = (long long)L + j;
+      long long row = -1;
+      if (p.paged) {
+        const long long lp = t / CLV_PAGE_SIZE;
+        if (lp < p.max_pages) {
+          const int pg = p.block_table[(int64_t)b * p.max_pages + lp];
+          if (pg >= 0 && pg < p.n_pages) row = (long long)pg * CLV_PAGE_SIZE + t % CLV_PAGE_SIZE;
+        }
+      } else if (t < p.cap_tokens) {
+        row = (long long)b * p.cap_tokens + t;
+      }
+      if (a < 0 || a >= p.N || row < 0) s_ok = 0;  // benign race: every writer stores 0
+      s_src[j] = a;
+      s_dst[j] = row;
+    }
+  }
+  __syncthreads();
+  if (!s_ok) {
+    if (tid == 0) { p.ctx_len_out[b] = L; p.status[b] = CLV_ERR_TREE; }
+    return;
+  }
+  const int per_row = 2 * p.row_vec;  // K then V
+  for (int w = tid; w < len * per_row; w += blockDim.x) {
+    const int j = w / per_row, r = w - j * per_row;
+    const int c = (r < p.row_vec) ? r : r - p.row_vec;
+    const int64_t src = ((int64_t)b * p.N + s_src[j]) * p.row_vec + c;
+    const int64_t dst = s_dst[j] * p.row_vec + c;
+    if (r < p.row_vec) p.kc[dst] = p.k_tree[src];
+    else p.vc[dst] = p.v_tree[src];
+  }
+  if (tid == 0) { p.ctx_len_out[b] = L + len; p.status[b] = CLV_OK; }
+}
+
+}  // namespace
+
+cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
+                        const int32_t* ids, int32_t* accept_len, int32_t* accept_idx,
+                        int32_t* next_token, int32_t* status, cudaStream_t stream) {
+  walk_kernel<<<s.batch, 32, 0, stream>>>(s.n_nodes, s.path_cap, parent, tokens, ids, accept_len,
+                                          accept_idx, next_token, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void* k_tree,
+                          const void* v_tree, const int32_t* accept_idx, const int32_t* accept_len,
+                          const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
+                          cudaStream_t stream) {
+  CommitParams p;
+  p.kc = static_cast<uint4*>(c.k);
+  p.vc = static_cast<uint4*>(c.v);
+  p.k_tree = static_cast<const uint4*>(k_tree);
+  p.v_tree = static_cast<const uint4*>(v_tree);
+  p.block_table = c.block_table;
+  p.accept_idx = accept_idx;
+  p.accept_len = accept_len;
+  p.ctx_len = ctx_len;
+  p.ctx_len_out = ctx_len_out;
+  p.status = status;
+  p.N = s.n_nodes;
+  p.path_cap = s.path_cap;
+  p.paged = c.paged;
+  p.cap_tokens = c.cap_tokens;
+  p.n_pages = c.n_pages;
+  p.max_pages = c.max_pages_per_seq;
+  p.row_vec = s.n_kv_heads * CLV_HEAD_DIM * 2 / 16;
+  commit_kernel<<<s.batch, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace clv
