@@ -1,0 +1,218 @@
+"""ctypes binding of libclv.so: argument marshalling only.
+
+Every function has the name of the C entry point it forwards to (see ``include/clv.h``) and takes
+torch CUDA tensors; all arithmetic of the verify step runs in the library's kernels.  There is no
+CPU fallback: if the shared library has not been built, :func:`lib` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libclv.so")
+
+CLV_OK = 0
+CLV_ERR_NULL, CLV_ERR_SHAPE, CLV_ERR_UNSUPPORTED, CLV_ERR_ALIGN = 1, 2, 3, 4
+CLV_ERR_WORKSPACE, CLV_ERR_CUDA, CLV_ERR_TREE, CLV_ERR_TIMEOUT = 5, 6, 7, 8
+
+EXPORTS = (
+    "clv_workspace_bytes", "clv_workspace_init", "clv_tree_attn", "clv_accept_argmax",
+    "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
+    "clv_status_string", "clv_last_cuda_error", "clv_version",
+)
+
+
+class ClvShape(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_nodes", ctypes.c_int32),
+                ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("vocab", ctypes.c_int32),
+                ("path_cap", ctypes.c_int32)]
+
+
+class ClvKvCache(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("paged", ctypes.c_int32),
+                ("cap_tokens", ctypes.c_int32), ("page_size", ctypes.c_int32),
+                ("n_pages", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
+                ("block_table", ctypes.c_void_p)]
+
+
+class ClvHostInputs(ctypes.Structure):
+    _fields_ = [("q", ctypes.c_void_p), ("k_tree", ctypes.c_void_p), ("v_tree", ctypes.c_void_p),
+                ("parent", ctypes.c_void_p), ("tokens", ctypes.c_void_p),
+                ("logits", ctypes.c_void_p), ("ld", ctypes.c_int64)]
+
+
+class ClvHostOutputs(ctypes.Structure):
+    _fields_ = [("out", ctypes.c_void_p), ("argmax_ids", ctypes.c_void_p),
+                ("accept_len", ctypes.c_void_p), ("accept_idx", ctypes.c_void_p),
+                ("next_token", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+class ClvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().clv_status_string(code).decode()
+        if code == CLV_ERR_CUDA:
+            msg += " (cudaError %d)" % lib().clv_last_cuda_error()
+        super().__init__("%s: %s" % (where, msg))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libclv.so is missing at %s: build it with `python -m paper_2408_00264_b200.build`"
+                % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz, f32 = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t,
+                                 ctypes.c_float)
+        L.clv_workspace_bytes.restype = sz
+        L.clv_workspace_bytes.argtypes = [vp, vp, i32]
+        L.clv_workspace_init.restype = i32
+        L.clv_workspace_init.argtypes = [vp, sz, vp]
+        L.clv_tree_attn.restype = i32
+        L.clv_tree_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, sz, vp]
+        L.clv_accept_argmax.restype = i32
+        L.clv_accept_argmax.argtypes = [vp, vp, i64, vp, vp, sz, vp]
+        L.clv_accept_walk.restype = i32
+        L.clv_accept_walk.argtypes = [vp] * 9
+        L.clv_kv_commit.restype = i32
+        L.clv_kv_commit.argtypes = [vp] * 10
+        L.clv_staging_bytes.restype = sz
+        L.clv_staging_bytes.argtypes = [vp, i64]
+        L.clv_verify_step_host.restype = i32
+        L.clv_verify_step_host.argtypes = [vp, vp, vp, vp, vp, i32, f32, vp, sz, vp, sz, vp]
+        L.clv_status_string.restype = ctypes.c_char_p
+        L.clv_status_string.argtypes = [i32]
+        L.clv_last_cuda_error.restype = ctypes.c_int
+        L.clv_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ref(s):
+    return ctypes.cast(ctypes.byref(s), ctypes.c_void_p)
+
+
+def make_shape(batch, n_nodes, n_q_heads, n_kv_heads, vocab=0, path_cap=1, head_dim=128) -> ClvShape:
+    return ClvShape(batch, n_nodes, n_q_heads, n_kv_heads, head_dim, vocab, path_cap)
+
+
+def make_cache(k: torch.Tensor, v: torch.Tensor, block_table: Optional[torch.Tensor] = None
+               ) -> ClvKvCache:
+    """Contiguous cache [B, cap, Hkv, 128] or, with a block table, a paged pool [P, 64, Hkv, 128]."""
+    if block_table is None:
+        return ClvKvCache(k.data_ptr(), v.data_ptr(), 0, k.shape[1], 64, 0, 0, None)
+    return ClvKvCache(k.data_ptr(), v.data_ptr(), 1, 0, k.shape[1], k.shape[0],
+                      block_table.shape[1], block_table.data_ptr())
+
+
+def _check(code: int, where: str) -> None:
+    if code != CLV_OK:
+        raise ClvError(code, where)
+
+
+def clv_workspace_bytes(shape: ClvShape, cache: Optional[ClvKvCache], max_ctx_len: int) -> int:
+    return int(lib().clv_workspace_bytes(_ref(shape), None if cache is None else _ref(cache),
+                                         int(max_ctx_len)))
+
+
+def clv_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check(lib().clv_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                    _stream(stream)), "clv_workspace_init")
+
+
+def new_workspace(shape: ClvShape, cache: Optional[ClvKvCache], max_ctx_len: int,
+                  device="cuda") -> torch.Tensor:
+    """Allocate (through torch) and initialise a workspace of the required size."""
+    n = clv_workspace_bytes(shape, cache, max_ctx_len)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    clv_workspace_init(ws)
+    return ws
+
+
+def clv_tree_attn(shape, cache, q, k_tree, v_tree, parent, ctx_len, max_ctx_len, softmax_scale,
+                  out, lse, status, workspace, stream=None, check=True) -> int:
+    code = lib().clv_tree_attn(_ref(shape), _ref(cache), _ptr(q), _ptr(k_tree), _ptr(v_tree),
+                               _ptr(parent), _ptr(ctx_len), int(max_ctx_len), float(softmax_scale),
+                               _ptr(out), _ptr(lse), _ptr(status), _ptr(workspace),
+                               0 if workspace is None else workspace.numel() * workspace.element_size(),
+                               _stream(stream))
+    if check:
+        _check(code, "clv_tree_attn")
+    return code
+
+
+def clv_accept_argmax(shape, logits, ld, argmax_ids, workspace, stream=None, check=True) -> int:
+    code = lib().clv_accept_argmax(_ref(shape), _ptr(logits), int(ld), _ptr(argmax_ids),
+                                   _ptr(workspace),
+                                   0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                   _stream(stream))
+    if check:
+        _check(code, "clv_accept_argmax")
+    return code
+
+
+def clv_accept_walk(shape, parent, tokens, argmax_ids, accept_len, accept_idx, next_token, status,
+                    stream=None, check=True) -> int:
+    code = lib().clv_accept_walk(_ref(shape), _ptr(parent), _ptr(tokens), _ptr(argmax_ids),
+                                 _ptr(accept_len), _ptr(accept_idx), _ptr(next_token), _ptr(status),
+                                 _stream(stream))
+    if check:
+        _check(code, "clv_accept_walk")
+    return code
+
+
+def clv_kv_commit(shape, cache, k_tree, v_tree, accept_idx, accept_len, ctx_len, ctx_len_out, status,
+                  stream=None, check=True) -> int:
+    code = lib().clv_kv_commit(_ref(shape), _ref(cache), _ptr(k_tree), _ptr(v_tree),
+                               _ptr(accept_idx), _ptr(accept_len), _ptr(ctx_len), _ptr(ctx_len_out),
+                               _ptr(status), _stream(stream))
+    if check:
+        _check(code, "clv_kv_commit")
+    return code
+
+
+def clv_staging_bytes(shape: ClvShape, ld: int) -> int:
+    return int(lib().clv_staging_bytes(_ref(shape), int(ld)))
+
+
+def clv_verify_step_host(shape, cache, host_in: ClvHostInputs, host_out: ClvHostOutputs, ctx_len,
+                         max_ctx_len, softmax_scale, staging, workspace, stream=None,
+                         check=True) -> int:
+    code = lib().clv_verify_step_host(_ref(shape), _ref(cache), _ref(host_in), _ref(host_out),
+                                      _ptr(ctx_len), int(max_ctx_len), float(softmax_scale),
+                                      _ptr(staging), staging.numel() * staging.element_size(),
+                                      _ptr(workspace),
+                                      0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                      _stream(stream))
+    if check:
+        _check(code, "clv_verify_step_host")
+    return code
+
+
+def clv_version() -> int:
+    return int(lib().clv_version())
+
+
+def clv_status_string(code: int) -> str:
+    return lib().clv_status_string(int(code)).decode()

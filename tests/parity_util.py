@@ -1,0 +1,36 @@
+"""Comparison helpers shared by the GPU parity tests."""
+import numpy as np
+
+from paper_2408_00264_b200 import workloads as W
+
+ATTN_MAX_ABS = 2e-2      # stated tolerance of the verify step: bf16 output, fp32 accumulation
+ATTN_MAX_REL = 1e-2
+
+
+def attn_errors(got_bits: np.ndarray, ref: np.ndarray):
+    """got_bits [..., D] bf16 bits, ref [..., D] float64.  Returns (max abs error, max relative
+    error), the relative error taken against max(|ref|, row max-abs / 64) so that entries that
+    happen to be near zero do not dominate."""
+    got = W.bf16_bits_to_f64(got_bits)
+    err = np.abs(got - ref)
+    floor = np.abs(ref).max(axis=-1, keepdims=True) / 64.0
+    rel = err / np.maximum(np.abs(ref), np.maximum(floor, 1e-30))
+    return float(err.max()), float(rel.max())
+
+
+def assert_attn_close(got_bits, ref, what=""):
+    assert np.isfinite(W.bf16_bits_to_f64(got_bits)).all(), what
+    a, r = attn_errors(got_bits, ref)
+    assert a <= ATTN_MAX_ABS and r <= ATTN_MAX_REL, "%s max-abs %.3e max-rel %.3e" % (what, a, r)
+
+
+def sample_rows(w, n, seed=0):
+    """n random (b, i, h) triples, always including first/last node and head of each sequence."""
+    c = w.cfg
+    rng = np.random.default_rng(seed)
+    rows = [(b, i, h) for b in (0, c.batch - 1) for i in (0, c.n_nodes - 1)
+            for h in (0, c.n_q_heads - 1)]
+    while len(rows) < n:
+        rows.append((int(rng.integers(c.batch)), int(rng.integers(c.n_nodes)),
+                     int(rng.integers(c.n_q_heads))))
+    return np.array(sorted(set(rows)), dtype=np.int32)
