@@ -229,6 +229,8 @@ def _draw_tokens(parent: np.ndarray, vocab: int, rng: np.random.Generator) -> np
     tok = rng.integers(0, vocab, size=n, dtype=np.int64)
     for p in range(-1, n):
         kids = np.flatnonzero(parent == p)
+        if len(kids) > vocab:
+            raise ValueError("a node has more children than there are distinct tokens")
         seen = set()
         for c in kids:
             while int(tok[c]) in seen:
@@ -247,6 +249,8 @@ def _plant_winners(parent: np.ndarray, tokens: np.ndarray, vocab: int, p: float,
             win[i] = tokens[kids[rng.integers(0, len(kids))]]
         else:
             kid_tok = set(int(t) for t in tokens[kids])
+            if len(kid_tok) >= vocab:
+                raise ValueError("no token left that is not a child's token")
             w = int(rng.integers(0, vocab))
             while w in kid_tok:
                 w = int(rng.integers(0, vocab))

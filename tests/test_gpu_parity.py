@@ -238,8 +238,8 @@ def test_walk_random_trees_and_errors(clv, oracle):
     B, N = 64, 48
     cfg = W.small_config(batch=B, n_nodes=N, vocab=16, n_q_heads=1, n_kv_heads=1, ctx=1)
     w = W.generate(cfg)
-    ids = rng.integers(0, 6, size=(B, N)).astype(np.int32)
-    tokens = np.stack([W._draw_tokens(w.parent[b], 6, rng) for b in range(B)])
+    tokens = np.stack([W._draw_tokens(w.parent[b], 64, rng) for b in range(B)])
+    ids = np.stack([W._plant_winners(w.parent[b], tokens[b], 64, 0.7, rng) for b in range(B)])
     w.parent[3, 0] = 0                        # root is not a root
     w.parent[4, 9] = -1                       # second root
     w.parent[5, 7] = 7                        # self parent

@@ -68,7 +68,7 @@ def test_walk_equals_brute_force_on_tiny_trees(oracle):
     for trial in range(300):
         n = int(rng.integers(1, 13))
         parent = W.tree_random(n, 5, rng)
-        vocab = 6                                   # small vocabulary: many chance agreements
+        vocab = 12                                  # small vocabulary: many chance agreements
         tokens = W._draw_tokens(parent, vocab, rng)
         ids = rng.integers(0, vocab, size=n).astype(np.int32)
         alen, aidx, nxt, st = oracle.accept_walk(parent[None], tokens[None], ids[None], 13)
