@@ -264,21 +264,23 @@ def run_clv(args):
     ctx0 = s0.ctx_len.clone()
     h2d = sum(t.numel() * t.element_size() for t in host)
     d2h = sum(t.numel() * t.element_size() for t in (o_out, o_ids, o_len, o_idx, o_nxt, o_st))
-    n_e2e = max(3, min(args.steps, 50))
+    n_e2e = 0 if args.no_e2e else max(3, min(args.steps, 50))
 
     def host_step():
         s0.ctx_len.copy_(ctx0, non_blocking=True)   # keep the context length fixed across steps
         clv.clv_verify_step_host(s0.shape, s0.cache, hin, hout, s0.ctx_len, s0.max_ctx_len, s0.scale,
                                  staging, s0.workspace)
-    for _ in range(3):
-        host_step()
-    barrier()
-    e0.record(stream)
-    for _ in range(n_e2e):
-        host_step()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / n_e2e
+    e2e_ms = float("nan")
+    if n_e2e:
+        for _ in range(3):
+            host_step()
+        barrier()
+        e0.record(stream)
+        for _ in range(n_e2e):
+            host_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
 
     # ---- max over ranks ------------------------------------------------------------------------
     if dist is not None:
@@ -340,6 +342,7 @@ def main():
     ap.add_argument("--impl", default="clv", choices=["clv", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch the four calls per step directly")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
