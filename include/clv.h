@@ -55,7 +55,8 @@ enum {
   CLV_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than clv_workspace_bytes()              */
   CLV_ERR_CUDA = 6,        /* a CUDA runtime call failed; see clv_last_cuda_error()             */
   CLV_ERR_TREE = 7,        /* device status[] only: malformed tree or capacity exceeded         */
-  CLV_ERR_TIMEOUT = 8      /* device status[] only: a bounded on-chip wait gave up              */
+  CLV_ERR_TIMEOUT = 8,     /* device status[] only: a bounded on-chip wait gave up              */
+  CLV_ERR_TOO_LARGE = 9    /* clv_accept_argmax_noalloc: the problem exceeds its built-in scratch */
 };
 
 #define CLV_MAX_NODES 128
@@ -132,6 +133,31 @@ clv_status clv_accept_argmax(const clv_shape* shape,
                              int64_t ld,
                              int32_t* argmax_ids, /* [B, N]                      */
                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * clv_accept_argmax without any caller-provided scratch.  The paper has no counterpart to this
+ * entry point; it exists for integration reasons only.  Some hosts of this library may not
+ * allocate device memory when they call it: code running inside a serving engine that handed all
+ * of the GPU's memory to its own pool at start-up, a plug-in that is only ever given input and
+ * output tensors, or a caller on a latency path where cudaMalloc's implicit synchronisation is
+ * not acceptable.  For them the arrival counters and per-chunk partial results live in a fixed
+ * array inside the library's device image instead of a workspace.
+ *   - Same inputs, outputs and result as clv_accept_argmax (bit-identical ids).
+ *   - Limit: B * N <= 4096 rows and rows * (thread blocks per row) <= 131072; anything larger is
+ *     refused with CLV_ERR_TOO_LARGE and nothing is enqueued.  The array is about 1.04 MB and
+ *     stays resident on every GPU that loads the library until the process exits.
+ *   - The call allocates and frees nothing (no cudaMalloc / cudaFree, no allocating library
+ *     routine).  The first call on a device looks up the array's device address (with that device
+ *     current) and remembers it; make that first call outside of any stream capture.
+ *   - All calls on one GPU share the array, and it keeps the previous call's contents; each call
+ *     clears the counters it needs on the given stream first.  Two calls that overlap on the GPU
+ *     (different streams, or different host threads without ordering) race on it: serialise them.
+ */
+clv_status clv_accept_argmax_noalloc(const clv_shape* shape,
+                                     const void* logits, /* bf16 [B*N, ld]       */
+                                     int64_t ld,
+                                     int32_t* argmax_ids, /* [B, N]              */
+                                     void* cuda_stream);
 
 /*
  * Greedy acceptance walk (Sec. 2.1 verification phase; Sec. 4.1).  Start at the root; at node cur

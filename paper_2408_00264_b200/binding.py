@@ -18,11 +18,12 @@ LIB_PATH = os.path.join(_PKG, "libclv.so")
 CLV_OK = 0
 CLV_ERR_NULL, CLV_ERR_SHAPE, CLV_ERR_UNSUPPORTED, CLV_ERR_ALIGN = 1, 2, 3, 4
 CLV_ERR_WORKSPACE, CLV_ERR_CUDA, CLV_ERR_TREE, CLV_ERR_TIMEOUT = 5, 6, 7, 8
+CLV_ERR_TOO_LARGE = 9
 
 EXPORTS = (
     "clv_workspace_bytes", "clv_workspace_init", "clv_tree_attn", "clv_accept_argmax",
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
-    "clv_status_string", "clv_last_cuda_error", "clv_version",
+    "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
 )
 
 
@@ -83,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.clv_tree_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, sz, vp]
         L.clv_accept_argmax.restype = i32
         L.clv_accept_argmax.argtypes = [vp, vp, i64, vp, vp, sz, vp]
+        L.clv_accept_argmax_noalloc.restype = i32
+        L.clv_accept_argmax_noalloc.argtypes = [vp, vp, i64, vp, vp]
         L.clv_accept_walk.restype = i32
         L.clv_accept_walk.argtypes = [vp] * 9
         L.clv_kv_commit.restype = i32
@@ -169,6 +172,16 @@ def clv_accept_argmax(shape, logits, ld, argmax_ids, workspace, stream=None, che
                                    _stream(stream))
     if check:
         _check(code, "clv_accept_argmax")
+    return code
+
+
+def clv_accept_argmax_noalloc(shape, logits, ld, argmax_ids, stream=None, check=True) -> int:
+    """clv_accept_argmax for callers that may not allocate device memory: no workspace argument,
+    the scratch is a fixed array inside the library (limits and sharing rules in clv.h)."""
+    code = lib().clv_accept_argmax_noalloc(_ref(shape), _ptr(logits), int(ld), _ptr(argmax_ids),
+                                           _stream(stream))
+    if check:
+        _check(code, "clv_accept_argmax_noalloc")
     return code
 
 

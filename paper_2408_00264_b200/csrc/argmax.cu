@@ -168,4 +168,50 @@ cudaError_t launch_argmax(const ArgmaxPlan& plan, const void* logits, int64_t ld
   return cudaGetLastError();
 }
 
+// ---- variant whose scratch lives in the library image ------------------------------------------
+// For callers that cannot allocate device memory at all.  The scratch (arrival counters followed
+// by the per-chunk keys) is a fixed array in this module's device image: every GPU that loads the
+// library holds it until the process exits, and every call on that GPU shares it.
+namespace {
+constexpr int kStaticMaxRows = 4096;         // B * N
+constexpr int kStaticMaxKeys = 131072;       // rows * chunks
+constexpr size_t kStaticTicketBytes = sizeof(unsigned) * (size_t)kStaticMaxRows;
+constexpr size_t kStaticBytes = kStaticTicketBytes + sizeof(unsigned long long) * (size_t)kStaticMaxKeys;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+}  // namespace
+
+bool argmax_static_fits(int rows, int vocab) {
+  if (rows > kStaticMaxRows) return false;
+  const ArgmaxPlan plan = argmax_plan(rows, vocab);
+  return (int64_t)rows * plan.chunks <= kStaticMaxKeys;
+}
+
+cudaError_t launch_argmax_static(const void* logits, int64_t ld, int rows, int vocab, int32_t* ids,
+                                 cudaStream_t stream) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (g_static_ptr[dev] == nullptr) {
+    // In host code the array's name is only a handle; the address the kernel can use has to be
+    // asked for, with the device that will run the kernel current.
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  unsigned char* base = g_static_ptr[dev];
+  const ArgmaxPlan plan = argmax_plan(rows, vocab);
+  if (plan.chunks > 1) {
+    // the counters must start at zero whatever an earlier (possibly aborted) call left behind
+    e = cudaMemsetAsync(base, 0, sizeof(unsigned) * (size_t)rows, stream);
+    if (e != cudaSuccess) return e;
+  }
+  return launch_argmax(plan, logits, ld, vocab, ids, reinterpret_cast<unsigned*>(base),
+                       base + kStaticTicketBytes, stream);
+}
+
 }  // namespace clv

@@ -126,6 +126,20 @@ clv_status clv_accept_argmax(const clv_shape* shape, const void* logits, int64_t
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
+clv_status clv_accept_argmax_noalloc(const clv_shape* shape, const void* logits, int64_t ld,
+                                     int32_t* argmax_ids, void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  if (!logits || !argmax_ids) return CLV_ERR_NULL;
+  if (shape->vocab < 1 || ld < shape->vocab) return CLV_ERR_SHAPE;
+  if (!aligned16(logits) || (ld % 8) != 0) return CLV_ERR_ALIGN;
+  const int64_t rows = (int64_t)shape->batch * shape->n_nodes;
+  if (rows > INT32_MAX || !argmax_static_fits((int)rows, shape->vocab)) return CLV_ERR_TOO_LARGE;
+  cudaError_t e = launch_argmax_static(logits, ld, (int)rows, shape->vocab, argmax_ids,
+                                       static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
 clv_status clv_accept_walk(const clv_shape* shape, const int32_t* parent, const int32_t* tokens,
                            const int32_t* argmax_ids, int32_t* accept_len, int32_t* accept_idx,
                            int32_t* next_token, int32_t* status, void* cuda_stream) {
@@ -270,6 +284,7 @@ const char* clv_status_string(clv_status s) {
     case CLV_ERR_CUDA: return "CUDA runtime error";
     case CLV_ERR_TREE: return "malformed tree or capacity exceeded";
     case CLV_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    case CLV_ERR_TOO_LARGE: return "problem exceeds the fixed built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }

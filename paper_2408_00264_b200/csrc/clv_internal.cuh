@@ -33,6 +33,11 @@ ArgmaxPlan argmax_plan(int rows, int vocab);
 cudaError_t launch_argmax(const ArgmaxPlan& plan, const void* logits, int64_t ld, int vocab,
                           int32_t* ids, unsigned* tickets, void* scratch, cudaStream_t stream);
 
+// variant with its scratch in a fixed device array of the library (no caller workspace)
+bool argmax_static_fits(int rows, int vocab);
+cudaError_t launch_argmax_static(const void* logits, int64_t ld, int rows, int vocab, int32_t* ids,
+                                 cudaStream_t stream);
+
 // ---- walk / commit ----------------------------------------------------------------------------
 cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
                         const int32_t* ids, int32_t* accept_len, int32_t* accept_idx,

@@ -1,0 +1,66 @@
+"""The argmax entry point for callers that cannot allocate device memory.
+
+Some users of the library run where device allocation is off the table at call time: inside an
+engine that gave the whole GPU to its own memory pool at start-up, as a plug-in that only ever
+receives input and output tensors, or on a latency path that must not hit cudaMalloc's implicit
+synchronisation.  `clv_accept_argmax_noalloc` keeps its counters and partial results in a fixed
+array inside the library instead of a workspace.  This file checks, through the C ABI, that it
+returns exactly what `clv_accept_argmax` returns, twice in a row (the array keeps the previous
+call's contents), and that it refuses problems beyond its fixed capacity.
+
+The file name sorts last on purpose, so a run that stops at the first failure has already
+executed every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2408_00264_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def clv():
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    from paper_2408_00264_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _logits(rows, vocab, seed):
+    rng = np.random.default_rng(seed)
+    winner = rng.integers(0, vocab, size=rows)
+    ld = (vocab + 7) // 8 * 8
+    return W.make_logits(rows, vocab, ld, winner, 0.5, seed=seed + 1), ld
+
+
+@pytest.mark.parametrize("batch,nodes,vocab", [(2, 5, 2049), (4, 64, 128256), (1, 16, 32000)])
+def test_noalloc_matches_workspace_entry_point_twice(clv, batch, nodes, vocab):
+    shape = clv.make_shape(batch, nodes, 1, 1, vocab, 1)
+    ws = clv.new_workspace(shape, None, 0)
+    ids_ref = torch.empty(batch, nodes, dtype=torch.int32, device="cuda")
+    ids_new = torch.full((batch, nodes), -7, dtype=torch.int32, device="cuda")
+    for call in range(2):                       # second call: different data, same built-in array
+        lg, ld = _logits(batch * nodes, vocab, seed=100 * call + vocab)
+        if call == 1:
+            lg[0, :] = 0x3F80                   # a row of equal values: the lowest index must win
+        d = torch.from_numpy(lg.view(np.int16)).cuda()
+        clv.clv_accept_argmax(shape, d, ld, ids_ref, ws)
+        ids_new.fill_(-7)
+        clv.clv_accept_argmax_noalloc(shape, d, ld, ids_new)
+        torch.cuda.synchronize()
+        assert torch.equal(ids_new, ids_ref)    # integer output: exact
+        assert int(ids_new.min()) >= 0 and int(ids_new.max()) < vocab
+
+
+def test_noalloc_rejects_sizes_beyond_its_fixed_scratch(clv):
+    d = torch.zeros(16, dtype=torch.int16, device="cuda")
+    ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    too_many_rows = clv.make_shape(64, 128, 1, 1, 32000, 1)          # 8192 rows > 4096
+    code = clv.clv_accept_argmax_noalloc(too_many_rows, d, 32000, ids, check=False)
+    assert code == clv.CLV_ERR_TOO_LARGE
+    assert "scratch" in clv.clv_status_string(code)
+    with pytest.raises(clv.ClvError):
+        clv.clv_accept_argmax_noalloc(too_many_rows, d, 32000, ids)
