@@ -1,6 +1,7 @@
 // C ABI of libclv: argument checks and dispatch.  No device memory is allocated here, nothing
 // synchronises, every launch goes to the caller's stream.
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "clv_internal.cuh"
@@ -52,6 +53,14 @@ static clv_status check_cache(const clv_kv_cache* c) {
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Which attention kernel serves a call: the tcgen05 kernel whenever the shape allows it.
+// CLV_ATTN_PATH=mma (environment, read at each call) forces the warp-level path, for comparisons.
+static bool use_tc_path(const clv_shape& s, const clv_kv_cache& c) {
+  const char* e = getenv("CLV_ATTN_PATH");
+  if (e && strcmp(e, "mma") == 0) return false;
+  return tc_attn_supported(s, c);
+}
+
 }  // namespace clv
 
 using namespace clv;
@@ -63,7 +72,8 @@ size_t clv_workspace_bytes(const clv_shape* shape, const clv_kv_cache* cache, in
   if (check_shape(shape) != CLV_OK) return 0;
   if (max_ctx_len < 0) max_ctx_len = 0;
   const AttnPlan ap = attn_plan(*shape, max_ctx_len);
-  size_t scratch = ap.scratch_bytes;
+  const AttnPlan tp = tc_attn_plan(*shape, max_ctx_len);   // either kernel may serve the call
+  size_t scratch = ap.scratch_bytes > tp.scratch_bytes ? ap.scratch_bytes : tp.scratch_bytes;
   if (shape->vocab > 0) {
     const ArgmaxPlan gp = argmax_plan(shape->batch * shape->n_nodes, shape->vocab);
     if (gp.scratch_bytes > scratch) scratch = gp.scratch_bytes;
@@ -91,16 +101,16 @@ clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, cons
   if (!q || !k_tree || !v_tree || !parent || !ctx_len || !out || !status) return CLV_ERR_NULL;
   if (!aligned16(q) || !aligned16(k_tree) || !aligned16(v_tree) || !aligned16(out)) return CLV_ERR_ALIGN;
   if (max_ctx_len < 0) return CLV_ERR_SHAPE;
-  const AttnPlan plan = attn_plan(*shape, max_ctx_len);
-  if (plan.splits > 1) {
+  const bool tc = use_tc_path(*shape, *cache);
+  const AttnPlan plan = tc ? tc_attn_plan(*shape, max_ctx_len) : attn_plan(*shape, max_ctx_len);
+  if (plan.scratch_bytes > 0) {
     if (!workspace || workspace_bytes < kWsFixedBytes + plan.scratch_bytes) return CLV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return CLV_ERR_ALIGN;
   }
-  cudaError_t e = launch_tree_attn(plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len,
-                                   softmax_scale, out, lse, status,
-                                   workspace ? ws_tickets(workspace) : nullptr,
-                                   workspace ? ws_scratch(workspace) : nullptr,
-                                   static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = (tc ? launch_tree_attn_tc : launch_tree_attn)(
+      plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len, softmax_scale, out, lse, status,
+      workspace ? ws_tickets(workspace) : nullptr, workspace ? ws_scratch(workspace) : nullptr,
+      static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 

@@ -61,6 +61,15 @@ cudaError_t launch_tree_attn(const AttnPlan& plan, const clv_shape& s, const clv
                              float* lse, int32_t* status, unsigned* tickets, void* scratch,
                              cudaStream_t stream);
 
+// tcgen05 / TMA path (row tiles must hold whole nodes: G divides 128)
+bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c);
+AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len);
+cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,
+                                const void* q, const void* k_tree, const void* v_tree,
+                                const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
+                                float* lse, int32_t* status, unsigned* tickets, void* scratch,
+                                cudaStream_t stream);
+
 int sm_count();
 
 }  // namespace clv

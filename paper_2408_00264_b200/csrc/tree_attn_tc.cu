@@ -1,0 +1,772 @@
+// Tree attention (Sec. 2.1) on the 5th-generation tensor cores: tcgen05.mma with accumulators in
+// tensor memory, K/V/Q tiles staged by TMA into 128-byte-swizzled shared memory.
+//
+// One thread block owns up to 256 query rows of one (sequence, kv head) - a row is a
+// (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes reuse every
+// K/V byte - and a contiguous range of 64-key tiles (cache tiles first, then the tree's own keys).
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation), warps 2-5 and
+// 6-9 = two softmax groups of 128 threads, one thread per query row ("slot" 0 and 1).
+//   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
+//   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
+//           accumulators are merged like split-KV partials.
+// Per slot and key tile:  S = Q K^T (tcgen05.mma -> TMEM)  ->  softmax thread reads its row of S,
+// masks, exponentiates against a lazily updated reference maximum, writes P (bf16) to shared
+// memory  ->  O += P V (tcgen05.mma, accumulator stays in TMEM).  While one slot is in its softmax
+// the tensor core works for the other.  The tree columns are masked with per-node ancestor
+// bitsets derived from parent[] on chip; masked scores are replaced, not added to, so they
+// contribute exactly zero.  Every mbarrier wait is bounded: on expiry the block raises a flag,
+// all roles leave their loops, in-flight copies and MMAs are drained, TMEM is released and
+// CLV_ERR_TIMEOUT is reported for the sequence.
+#include <cuda.h>
+#include <math.h>
+
+#include "clv_internal.cuh"
+#include "tmem_access.cuh"
+
+namespace clv {
+namespace {
+
+constexpr int BN = 64;                 // keys per tile (= page size)
+constexpr int HD = CLV_HEAD_DIM;       // 128
+constexpr int BM = 128;                // rows per MMA / per slot
+constexpr int kThreads = 320;
+constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
+constexpr uint32_t kKVTile = BN * HD * 2;     // 16 KB: two [64 keys][64 d] swizzled halves
+constexpr uint32_t kPTile = BM * BN * 2;      // 16 KB: [128 rows][64 keys] swizzled
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleGap = 8.0f;           // log2 units: P stays below 2^8
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;  // 1 s per wait
+
+template <int MT>
+struct Cfg {
+  static constexpr int kStages = (MT == 2) ? 3 : 4;
+  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kKVTile + 2 * kPTile + 1024;
+};
+
+struct Params {
+  const int32_t* block_table;
+  const int32_t* parent;
+  const int32_t* ctx_len;
+  uint16_t* out;
+  float* lse;
+  int32_t* status;
+  unsigned* tickets;
+  float* part_o;   // [row tile][partial][128][128]
+  float* part_ml;  // [row tile][partial][128][2]
+  int B, N, Hq, Hkv, G;
+  int paged, cap_tokens, n_pages, max_pages;
+  int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
+  int splits;      // thread blocks along the key axis
+  float scale_log2;
+};
+
+// ------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major operands: rows are 128 bytes apart,
+// sbo = distance between 8-row groups (1024).  MN-major operands: lbo = distance between
+// 64-element column blocks, sbo = distance between 8-row (K) groups.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version of this architecture
+  d |= 2ull << 61;  // swizzle mode: 128 bytes
+  return d;
+}
+// Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, A K-major.
+constexpr uint32_t make_idesc(int m, int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x 64]  = Q[128 x 16k] K[64 x 16k]^T
+constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------------------------ kernel
+template <int MT>
+__global__ void __launch_bounds__(kThreads, 1)
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
+                    const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
+                    const __grid_constant__ CUtensorMap tm_vt, const Params p) {
+  constexpr int NST = Cfg<MT>::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
+  __shared__ int s_parent[CLV_MAX_NODES];
+  __shared__ __align__(8) unsigned long long s_bar[2 * NST + 1 + 6 + 1];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ int s_last;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int unit = blockIdx.x / p.row_ctas, row_cta = blockIdx.x - unit * p.row_ctas;
+  const int split = blockIdx.y;
+  const int b = unit / p.Hkv, kvh = unit - b * p.Hkv;
+  const int N = p.N, G = p.G, rows_total = G * N;
+
+  // ---- per-sequence checks (same verdict in every block of the sequence) ------------------
+  const int L = p.ctx_len[b];
+  bool bad = false;
+  for (int i = tid; i < N; i += kThreads) {
+    const int par = p.parent[(int64_t)b * N + i];
+    s_parent[i] = par;
+    bad |= (par < -1 || par >= i);
+  }
+  bad |= (L < 0);
+  const int t_cache = L > 0 ? (L + BN - 1) / BN : 0;
+  if (p.paged) bad |= (t_cache > p.max_pages);
+  else bad |= (L > p.cap_tokens);
+  const int seq_bad = __syncthreads_or(bad ? 1 : 0);
+  const bool reporter = (row_cta == 0 && split == 0 && kvh == 0);
+  if (reporter) {
+    bool pbad = false;
+    if (p.paged && !seq_bad) {
+      for (int pg = tid; pg < t_cache; pg += kThreads) {
+        const int e = p.block_table[(int64_t)b * p.max_pages + pg];
+        pbad |= (e < 0 || e >= p.n_pages);
+      }
+    }
+    const int page_bad = __syncthreads_or(pbad ? 1 : 0);
+    if (tid == 0) p.status[b] = (seq_bad || page_bad) ? CLV_ERR_TREE : CLV_OK;
+  }
+  if (seq_bad) return;  // before any barrier or TMEM exists
+
+  // ancestor bitsets: row i of the tree's topology matrix
+  for (int i = tid; i < N; i += kThreads) {
+    uint32_t w[4] = {0, 0, 0, 0};
+    int j = i;
+    for (int hop = 0; hop < N && j >= 0; ++hop) {
+      w[j >> 5] |= 1u << (j & 31);
+      j = s_parent[j];
+    }
+    s_anc[i][0] = w[0]; s_anc[i][1] = w[1]; s_anc[i][2] = w[2]; s_anc[i][3] = w[3];
+  }
+
+  // ---- tile range and per-slot rounds -------------------------------------------------------
+  const int t_tree = (N + BN - 1) / BN;
+  const int t_total = t_cache + t_tree;
+  const int t_begin = (int)((int64_t)split * t_total / p.splits);
+  const int t_end = (int)((int64_t)(split + 1) * t_total / p.splits);
+  const int n_tiles = t_end - t_begin;
+  // local tile index of round r of slot s: MT == 2: r;  MT == 1: 2 r + s
+  const int rounds0 = (MT == 2) ? n_tiles : (n_tiles + 1) / 2;
+  const int rounds1 = (MT == 2) ? n_tiles : n_tiles / 2;
+
+  // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = smem_base;
+  const uint32_t sKV = sQ + MT * kQTile;             // stage i: K at +i*32K, V at +i*32K + 16K
+  const uint32_t sP = sKV + NST * 2 * kKVTile;        // slot s at + s*16K
+  uint8_t* const sP_gen = smem_raw + (sP - smem_u32(smem_raw));
+  uint8_t* const sKV_gen = smem_raw + (sKV - smem_u32(smem_raw));
+
+  const uint32_t bar0 = smem_u32(&s_bar[0]);
+  auto bar_kv_full = [&](int st) { return bar0 + 8u * st; };
+  auto bar_kv_empty = [&](int st) { return bar0 + 8u * (NST + st); };
+  const uint32_t bar_q = bar0 + 8u * (2 * NST);
+  auto bar_s_full = [&](int s) { return bar0 + 8u * (2 * NST + 1 + s); };
+  auto bar_p_full = [&](int s) { return bar0 + 8u * (2 * NST + 3 + s); };
+  auto bar_pv_done = [&](int s) { return bar0 + 8u * (2 * NST + 5 + s); };
+  const uint32_t bar_drain = bar0 + 8u * (2 * NST + 7);
+
+  if (tid == 0) {
+    for (int i = 0; i < NST; ++i) { mbar_init(bar_kv_full(i), 1); mbar_init(bar_kv_empty(i), 1); }
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_s_full(s), 1);
+      mbar_init(bar_p_full(s), BM);
+      mbar_init(bar_pv_done(s), 1);
+    }
+    mbar_init(bar_drain, 1);
+    s_abort = 0;
+    fence_barrier_init();
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abort_flag = &s_abort;
+  auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
+  auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + s * HD); };
+
+  int issued_tiles = 0;  // producer bookkeeping for the drain
+
+  if (warp == 0) {
+    // =========================== TMA producer ===============================================
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
+      tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
+    }
+    if (n_tiles > 0) {
+      if (lane == 0) {
+        mbar_expect_tx(bar_q, MT * kQTile);
+        const int nodes_per_tile = BM / G;
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          const int node0 = b * N + (row_cta * MT + m) * nodes_per_tile;
+          tma_load_3d(sQ + m * kQTile, &tm_q, 0, kvh * G, node0, bar_q);
+          tma_load_3d(sQ + m * kQTile + kQTile / 2, &tm_q, 64, kvh * G, node0, bar_q);
+        }
+      }
+      int page_cache = 0;  // lane j holds the pool page of cache tile (batch base + j)
+      bool ok = true;
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const int t = t_begin + i;
+        const int st = i % NST;
+        if (p.paged && (i % 32) == 0) {
+          const int tt = t + lane;
+          page_cache = (tt < t_cache) ? p.block_table[(int64_t)b * p.max_pages + tt] : 0;
+        }
+        int pg = __shfl_sync(0xFFFFFFFFu, page_cache, i % 32);
+        if (lane == 0) {
+          if (i >= NST) ok = mbar_wait(bar_kv_empty(st), ((i / NST) - 1) & 1, abort_flag);
+          if (ok) {
+            const uint32_t dK = sKV + st * 2 * kKVTile, dV = dK + kKVTile;
+            mbar_expect_tx(bar_kv_full(st), 2 * kKVTile);
+            if (t < t_cache) {
+              int row0;
+              if (p.paged) {
+                if (pg < 0 || pg >= p.n_pages) pg = 0;  // flagged by the reporter; rows get masked
+                row0 = pg * BN;
+              } else {
+                row0 = b * p.cap_tokens + t * BN;
+              }
+              tma_load_3d(dK, &tm_kc, 0, kvh, row0, bar_kv_full(st));
+              tma_load_3d(dK + kKVTile / 2, &tm_kc, 64, kvh, row0, bar_kv_full(st));
+              tma_load_3d(dV, &tm_vc, 0, kvh, row0, bar_kv_full(st));
+              tma_load_3d(dV + kKVTile / 2, &tm_vc, 64, kvh, row0, bar_kv_full(st));
+            } else {
+              const int row0 = b * N + (t - t_cache) * BN;
+              tma_load_3d(dK, &tm_kt, 0, kvh, row0, bar_kv_full(st));
+              tma_load_3d(dK + kKVTile / 2, &tm_kt, 64, kvh, row0, bar_kv_full(st));
+              tma_load_3d(dV, &tm_vt, 0, kvh, row0, bar_kv_full(st));
+              tma_load_3d(dV + kKVTile / 2, &tm_vt, 64, kvh, row0, bar_kv_full(st));
+            }
+            issued_tiles = i + 1;
+          }
+        }
+        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+      }
+    }
+  } else if (warp == 1) {
+    // =========================== MMA issuer ===================================================
+    if (lane == 0 && n_tiles > 0) {
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      tc_fence_after();
+      auto local_tile = [&](int s, int r) { return (MT == 2) ? r : 2 * r + s; };
+      auto issue_qk = [&](int s, int r) -> bool {
+        const int i = local_tile(s, r), st = i % NST;
+        if (!mbar_wait(bar_kv_full(st), (i / NST) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t qb = sQ + ((MT == 2) ? s : 0) * kQTile;
+        const uint32_t kb = sKV + st * 2 * kKVTile;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
+          const uint32_t ko = (ks >> 2) * (kKVTile / 2) + (ks & 3) * 32;
+          umma_bf16(tmem_S(s), smem_desc(qb + qo, 16, 1024), smem_desc(kb + ko, 16, 1024), kIdescQK,
+                    ks > 0 ? 1u : 0u);
+        }
+        umma_commit(bar_s_full(s));
+        return true;
+      };
+      const int rounds[2] = {rounds0, rounds1};
+      for (int s = 0; s < 2 && ok; ++s)
+        if (rounds[s] > 0) ok = issue_qk(s, 0);
+      for (int r = 0; r < rounds0 && ok; ++r) {
+        for (int s = 0; s < 2 && ok; ++s) {
+          if (r >= rounds[s]) continue;
+          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int i = local_tile(s, r), st = i % NST;
+          const uint32_t pb = sP + s * kPTile;
+          const uint32_t vb = sKV + st * 2 * kKVTile + kKVTile;
+#pragma unroll
+          for (int kk = 0; kk < BN / 16; ++kk) {
+            umma_bf16(tmem_O(s), smem_desc(pb + kk * 32, 16, 1024),
+                      smem_desc(vb + kk * 2048, kKVTile / 2, 1024), kIdescPV, (r > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(bar_pv_done(s));
+          if (MT == 1 || s == 1) umma_commit(bar_kv_empty(st));  // last reader of this stage
+          if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
+        }
+      }
+    }
+  } else {
+    // =========================== softmax groups ===============================================
+    const int slot = (warp - 2) >> 2;
+    const int quarter = warp & 3;                  // TMEM lanes this warp may touch
+    const int row = quarter * 32 + lane;           // row inside the 128-row tile
+    const int rounds = slot == 0 ? rounds0 : rounds1;
+    const int mtile = row_cta * MT + ((MT == 2) ? slot : 0);
+    const int r_glob = mtile * BM + row;
+    const bool row_valid = r_glob < rows_total;
+    const int node = row_valid ? r_glob / G : 0;
+    const int gq = row_valid ? r_glob - node * G : 0;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    float m_ref = -INFINITY, l_run = 0.f;
+    bool ok = true;
+
+    for (int r = 0; r < rounds && ok; ++r) {
+      const int i = (MT == 2) ? r : 2 * r + slot;
+      const int t = t_begin + i;
+      const int st = i % NST;
+      // allowed columns of this row in this tile, and how many V rows of the tile are real
+      uint32_t a_lo, a_hi;
+      int v_rows;
+      if (t < t_cache) {
+        v_rows = min(BN, L - t * BN);
+        if (p.paged) {
+          const int pg = p.block_table[(int64_t)b * p.max_pages + t];
+          if (pg < 0 || pg >= p.n_pages) v_rows = 0;
+        }
+        const uint64_t bits = v_rows >= 64 ? ~0ull : ((1ull << v_rows) - 1ull);
+        a_lo = (uint32_t)bits; a_hi = (uint32_t)(bits >> 32);
+      } else {
+        const int tt = t - t_cache;
+        v_rows = min(BN, N - tt * BN);
+        a_lo = s_anc[node][2 * tt]; a_hi = s_anc[node][2 * tt + 1];
+      }
+      if (!row_valid) a_lo = a_hi = 0;
+      const bool full = (a_lo & a_hi) == 0xFFFFFFFFu;
+
+      ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t sv[BN];
+      tmem_ld_x64(tmem_S(slot) + lane_addr, sv);
+      tmem_wait_ld();
+
+      float mx = -INFINITY;
+      if (__all_sync(0xFFFFFFFFu, full)) {
+#pragma unroll
+        for (int j = 0; j < BN; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < BN; ++j) {
+          const uint32_t wbits = j < 32 ? a_lo : a_hi;
+          const float x = ((wbits >> (j & 31)) & 1u) ? __uint_as_float(sv[j]) : -INFINITY;
+          sv[j] = __float_as_uint(x);
+          mx = fmaxf(mx, x);
+        }
+      }
+      mx *= p.scale_log2;  // scale > 0; -inf stays -inf
+      const bool need = mx > m_ref + kRescaleGap;  // also true for the first finite maximum
+      const bool any_need = __any_sync(0xFFFFFFFFu, need);
+
+      if (r > 0) {  // P buffer free again and O no longer being written
+        ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      if (any_need) {
+        const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
+        if (need) { m_ref = mx; l_run *= alpha; }
+        if (r > 0) {
+#pragma unroll 1
+          for (int c = 0; c < HD; c += 32) {
+            uint32_t ov[32];
+            tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+            tmem_st_x32(tmem_O(slot) + lane_addr + c, ov);
+          }
+          tmem_wait_st();
+        }
+      }
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      float sum = 0.f;
+      uint8_t* prow = sP_gen + slot * kPTile + row * 128;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = ex2(fmaf(__uint_as_float(sv[c * 8 + 2 * e]), p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[c * 8 + 2 * e + 1]), p.scale_log2, neg_m));
+          sum += p0 + p1;
+          pk[e] = pack_bf16(p0, p1);
+        }
+        *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+      l_run += sum;
+
+      if (v_rows < BN) {
+        // Rows of the V tile beyond the real keys hold whatever lies behind them in memory; their
+        // probabilities are exactly 0, but 0 * NaN would poison O, so clear them.
+        ok = mbar_wait(bar_kv_full(st), (i / NST) & 1, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        uint8_t* vt = sKV_gen + st * 2 * kKVTile + kKVTile;
+        const int n_chunks = (BN - v_rows) * 8 * 2;  // 16-byte chunks: rows x 8 x two halves
+        for (int c = (warp - 2 - slot * 4) * 32 + lane; c < n_chunks; c += BM) {
+          const int half = c / ((BN - v_rows) * 8), rem = c - half * (BN - v_rows) * 8;
+          const int vr = v_rows + (rem >> 3), ch = rem & 7;
+          *reinterpret_cast<uint4*>(vt + half * (kKVTile / 2) + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_async_smem();   // P (and cleared V rows) visible to the tensor core's reads
+      tc_fence_before();
+      mbar_arrive(bar_p_full(slot));
+    }
+
+    // ---- epilogue of this slot: final O out of TMEM ------------------------------------------
+    if (ok && rounds > 0) {
+      ok = mbar_wait(bar_pv_done(slot), (rounds - 1) & 1, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (ok) tc_fence_after();
+    }
+    const int partials = p.splits * (MT == 1 ? 2 : 1);
+    if (ok) {
+      const float kLn2 = 0.6931471805599453f;
+      if (partials == 1) {
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD;
+#pragma unroll 1
+        for (int c = 0; c < HD; c += 32) {
+          uint32_t ov[32];
+          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+          tmem_wait_ld();
+          if (row_valid) {
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              uint4 v;
+              v.x = pack_bf16(__uint_as_float(ov[q4 * 8 + 0]) * inv, __uint_as_float(ov[q4 * 8 + 1]) * inv);
+              v.y = pack_bf16(__uint_as_float(ov[q4 * 8 + 2]) * inv, __uint_as_float(ov[q4 * 8 + 3]) * inv);
+              v.z = pack_bf16(__uint_as_float(ov[q4 * 8 + 4]) * inv, __uint_as_float(ov[q4 * 8 + 5]) * inv);
+              v.w = pack_bf16(__uint_as_float(ov[q4 * 8 + 6]) * inv, __uint_as_float(ov[q4 * 8 + 7]) * inv);
+              *reinterpret_cast<uint4*>(dst + c + q4 * 8) = v;
+            }
+          }
+        }
+        if (p.lse != nullptr && row_valid)
+          p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
+      } else {
+        const int64_t rt = (int64_t)blockIdx.x * MT + ((MT == 2) ? slot : 0);
+        const int pi = (MT == 2) ? split : split * 2 + slot;
+        float* po = p.part_o + ((rt * partials + pi) * BM + row) * (int64_t)HD;
+        float* pml = p.part_ml + ((rt * partials + pi) * BM + row) * 2;
+        if (rounds > 0) {
+#pragma unroll 1
+          for (int c = 0; c < HD; c += 32) {
+            uint32_t ov[32];
+            tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4)
+              __stcg(reinterpret_cast<uint4*>(po + c + q4 * 4),
+                     make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]));
+          }
+        }
+        __stcg(reinterpret_cast<float2*>(pml), make_float2(rounds > 0 ? m_ref : -INFINITY, rounds > 0 ? l_run : 0.f));
+      }
+    }
+  }
+
+  // ---- teardown: drain what is still in flight, release TMEM --------------------------------
+  __syncwarp();
+  if (*abort_flag) {
+    if (warp == 0 && lane == 0) {
+      // TMA copies that were issued land on their own; wait for the newest phase of each stage
+      for (int i = max(0, issued_tiles - NST); i < issued_tiles; ++i) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try(bar_kv_full(i % NST), (i / NST) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      }
+      if (n_tiles > 0) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try(bar_q, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    if (warp == 1 && lane == 0) {
+      umma_commit(bar_drain);  // completes when every MMA issued so far has finished
+      const unsigned long long t0 = globaltimer_ns();
+      while (!mbar_try(bar_drain, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+    }
+  }
+  tc_fence_before();
+  __threadfence();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+  if (*abort_flag) {
+    if (tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
+    return;
+  }
+
+  // ---- merge of the partial results ------------------------------------------------------------
+  const int partials = p.splits * (MT == 1 ? 2 : 1);
+  if (partials == 1) return;
+  if (p.splits > 1) {
+    if (tid == 0) {
+      const unsigned arrived = atomicInc(p.tickets + blockIdx.x, (unsigned)p.splits - 1);  // wraps to 0
+      s_last = (arrived == (unsigned)p.splits - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+  }
+  // Phase 1: one thread per output row turns the (m, l) pairs into normalised weights, kept in the
+  // (now idle) tile memory.  Phase 2: every thread combines 4-column pieces, 32 consecutive
+  // threads covering one 512-byte row of each partial, all loads independent of each other.
+  const float kLn2 = 0.6931471805599453f;
+  float* s_w = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));  // [partial][MT*128]
+  const int n_rows = MT * BM;
+  for (int rr = tid; rr < n_rows; rr += kThreads) {
+    const int row = rr % BM;
+    const int64_t rt = (int64_t)blockIdx.x * MT + rr / BM;
+    const float* ml = p.part_ml + (rt * partials * BM + row) * 2;
+    float mmax = -INFINITY;
+    for (int q = 0; q < partials; ++q) mmax = fmaxf(mmax, __ldcg(ml + (int64_t)q * BM * 2));
+    const float mu = (mmax == -INFINITY) ? 0.f : mmax;
+    float lsum = 0.f;
+    for (int q = 0; q < partials; ++q) {
+      const float2 v = __ldcg(reinterpret_cast<const float2*>(ml + (int64_t)q * BM * 2));
+      const float w = (v.y > 0.f) ? ex2(v.x - mu) : 0.f;  // an empty partial gets weight 0
+      s_w[q * n_rows + rr] = w;
+      lsum += w * v.y;
+    }
+    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+    for (int q = 0; q < partials; ++q) s_w[q * n_rows + rr] *= inv;
+    const int r_glob = (row_cta * MT + rr / BM) * BM + row;
+    if (p.lse != nullptr && r_glob < rows_total) {
+      const int node = r_glob / G, gq = r_glob - node * G;
+      p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (mmax + log2f(lsum)) * kLn2;
+    }
+  }
+  __syncthreads();
+  for (int item = tid; item < n_rows * 32; item += kThreads) {
+    const int rr = item >> 5, piece = item & 31;
+    const int row = rr % BM;
+    const int r_glob = (row_cta * MT + rr / BM) * BM + row;
+    if (r_glob >= rows_total) continue;
+    const int node = r_glob / G, gq = r_glob - node * G;
+    const int64_t rt = (int64_t)blockIdx.x * MT + rr / BM;
+    const float* po = p.part_o + (rt * partials * BM + row) * (int64_t)HD + piece * 4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int q = 0; q < partials; ++q) {
+      const float w = s_w[q * n_rows + rr];
+      if (w != 0.f) {  // a skipped partial may hold anything, even NaN
+        const float4 x = __ldcg(reinterpret_cast<const float4*>(po + (int64_t)q * BM * HD));
+        acc.x += w * x.x; acc.y += w * x.y; acc.z += w * x.z; acc.w += w * x.w;
+      }
+    }
+    uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD + piece * 4;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+  }
+}
+
+// ------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    (void)cudaGetLastError();
+  }
+  return fn;
+}
+
+// bf16 tensor [rows][heads][128]; box = 64 elements x box_heads x box_rows, 128-byte swizzle
+bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t heads, uint32_t box_heads,
+              uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)HD, heads, rows};
+  const cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)HD * 2 * heads};
+  const cuuint32_t box[3] = {64, box_heads, box_rows};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
+  const int G = s.n_q_heads / s.n_kv_heads;
+  if (G > BM || (BM % G) != 0) return false;           // a row tile must hold whole nodes
+  const int64_t cache_rows = c.paged ? (int64_t)c.n_pages * CLV_PAGE_SIZE : (int64_t)s.batch * c.cap_tokens;
+  if (cache_rows >= (1ll << 31) || (int64_t)s.batch * s.n_nodes >= (1ll << 31)) return false;
+  return encode_fn() != nullptr;
+}
+
+AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
+  AttnPlan pl;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  const int rows = G * s.n_nodes;
+  const int mt = rows > BM ? 2 : 1;
+  const int row_ctas = (rows + mt * BM - 1) / (mt * BM);
+  pl.m_tiles = row_ctas;
+  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * row_ctas;
+  const int key_tiles = (max_ctx_len > 0 ? (max_ctx_len + BN - 1) / BN : 0) + (s.n_nodes + BN - 1) / BN;
+  int64_t want = sm_count() / (ctas > 0 ? ctas : 1);   // one resident block per SM
+  const int per_cta_min = mt == 1 ? 2 : 1;             // MT == 1 blocks eat two tiles per round
+  if (want > key_tiles / per_cta_min) want = key_tiles / per_cta_min;
+  if (want > 32) want = 32;                            // weights of all partials fit the tile memory
+  if (want < 1 || ctas > kTickets) want = 1;
+  pl.splits = (int)want;
+  pl.tickets = pl.splits > 1 ? (int)ctas : 0;
+  const int partials = pl.splits * (mt == 1 ? 2 : 1);
+  pl.scratch_bytes = partials > 1
+      ? (size_t)ctas * mt * partials * (BM * HD + BM * 2) * sizeof(float) : 0;
+  return pl;
+}
+
+cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,
+                                const void* q, const void* k_tree, const void* v_tree,
+                                const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
+                                float* lse, int32_t* status, unsigned* tickets, void* scratch,
+                                cudaStream_t stream) {
+  const int G = s.n_q_heads / s.n_kv_heads;
+  const int rows = G * s.n_nodes;
+  const int mt = rows > BM ? 2 : 1;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)Cfg<1>::kSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(tree_attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Cfg<2>::kSmem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt;
+  const uint64_t cache_rows = c.paged ? (uint64_t)c.n_pages * CLV_PAGE_SIZE : (uint64_t)s.batch * c.cap_tokens;
+  const uint64_t tree_rows = (uint64_t)s.batch * s.n_nodes;
+  if (!make_map(&tm_q, q, tree_rows, s.n_q_heads, G, BM / G) ||
+      !make_map(&tm_kc, c.k, cache_rows, s.n_kv_heads, 1, BN) ||
+      !make_map(&tm_vc, c.v, cache_rows, s.n_kv_heads, 1, BN) ||
+      !make_map(&tm_kt, k_tree, tree_rows, s.n_kv_heads, 1, BN) ||
+      !make_map(&tm_vt, v_tree, tree_rows, s.n_kv_heads, 1, BN))
+    return cudaErrorInvalidValue;
+
+  Params p;
+  p.block_table = c.block_table;
+  p.parent = parent;
+  p.ctx_len = ctx_len;
+  p.out = static_cast<uint16_t*>(out);
+  p.lse = lse;
+  p.status = status;
+  p.tickets = tickets;
+  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
+  const int partials = plan.splits * (mt == 1 ? 2 : 1);
+  p.part_o = static_cast<float*>(scratch);
+  p.part_ml = p.part_o + ctas * mt * partials * (int64_t)(BM * HD);
+  p.B = s.batch; p.N = s.n_nodes; p.Hq = s.n_q_heads; p.Hkv = s.n_kv_heads; p.G = G;
+  p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
+  p.row_ctas = plan.m_tiles;
+  p.splits = plan.splits;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  dim3 grid((unsigned)ctas, (unsigned)plan.splits, 1);
+  if (mt == 1)
+    tree_attn_tc_kernel<1><<<grid, kThreads, Cfg<1>::kSmem, stream>>>(tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  else
+    tree_attn_tc_kernel<2><<<grid, kThreads, Cfg<2>::kSmem, stream>>>(tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  return cudaGetLastError();
+}
+
+}  // namespace clv

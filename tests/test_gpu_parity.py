@@ -139,6 +139,7 @@ def test_attention_many_splits_and_ragged(clv, oracle):
     w.ctx_len[0] = 40
     st = make_step(w)
     st.max_ctx_len = 2500
+    st.workspace = clv.new_workspace(st.shape, st.cache, 2500)
     st.tree_attn()
     torch.cuda.synchronize()
     check_attention(oracle, w, st)
