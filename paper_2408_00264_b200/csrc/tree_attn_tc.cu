@@ -32,15 +32,14 @@ constexpr int BM = 128;                // rows per MMA / per slot
 constexpr int kThreads = 320;
 constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kKVTile = BN * HD * 2;     // 16 KB: two [64 keys][64 d] swizzled halves
-constexpr uint32_t kPTile = BM * BN * 2;      // 16 KB: [128 rows][64 keys] swizzled
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleGap = 8.0f;           // log2 units: P stays below 2^8
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;  // 1 s per wait
+constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: about a second
 
 template <int MT>
 struct Cfg {
-  static constexpr int kStages = (MT == 2) ? 3 : 4;
-  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kKVTile + 2 * kPTile + 1024;
+  static constexpr int kStages = (MT == 2) ? 4 : 5;
+  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kKVTile + 1024;
 };
 
 struct Params {
@@ -64,11 +63,6 @@ struct Params {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -90,17 +84,25 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
+// try_wait itself suspends the thread for a hardware-bounded time, so the first polls need no
+// clock; after that the SM clock (cheap to read, unlike the global timer) bounds the wait.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
+#pragma unroll 1
+  for (int spin = 0; spin < 32; ++spin)
+    if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
   for (;;) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+    if (clock64() - t0 > kWaitLimitCycles) {
       *abort_flag = 1;
       return false;
     }
   }
+}
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {  // teardown only
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity) && clock64() - t0 < kWaitLimitCycles) {}
 }
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -138,6 +140,16 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Same with the A operand read from tensor memory (lane = row, two bf16 per 32-bit column).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // Shared-memory matrix descriptor, 128-byte swizzle.  K-major operands: rows are 128 bytes apart,
@@ -243,8 +255,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem_base;
   const uint32_t sKV = sQ + MT * kQTile;             // stage i: K at +i*32K, V at +i*32K + 16K
-  const uint32_t sP = sKV + NST * 2 * kKVTile;        // slot s at + s*16K
-  uint8_t* const sP_gen = smem_raw + (sP - smem_u32(smem_raw));
   uint8_t* const sKV_gen = smem_raw + (sKV - smem_u32(smem_raw));
 
   const uint32_t bar0 = smem_u32(&s_bar[0]);
@@ -275,8 +285,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abort_flag = &s_abort;
+  // columns: S of slot s at 64 s; P (bf16 pairs) at 128 + 32 s; O at 192 + 128 s
   auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + s * HD); };
+  auto tmem_P = [&](int s) { return tmem + (uint32_t)(2 * BN + s * (BN / 2)); };
+  auto tmem_O = [&](int s) { return tmem + (uint32_t)(3 * BN + s * HD); };
 
   int issued_tiles = 0;  // producer bookkeeping for the drain
 
@@ -369,12 +381,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (!ok) break;
           tc_fence_after();
           const int i = local_tile(s, r), st = i % NST;
-          const uint32_t pb = sP + s * kPTile;
           const uint32_t vb = sKV + st * 2 * kKVTile + kKVTile;
 #pragma unroll
           for (int kk = 0; kk < BN / 16; ++kk) {
-            umma_bf16(tmem_O(s), smem_desc(pb + kk * 32, 16, 1024),
-                      smem_desc(vb + kk * 2048, kKVTile / 2, 1024), kIdescPV, (r > 0 || kk > 0) ? 1u : 0u);
+            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, smem_desc(vb + kk * 2048, kKVTile / 2, 1024),
+                         kIdescPV, (r > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(bar_pv_done(s));
           if (MT == 1 || s == 1) umma_commit(bar_kv_empty(st));  // last reader of this stage
@@ -469,19 +480,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float sum = 0.f;
-      uint8_t* prow = sP_gen + slot * kPTile + row * 128;
+      uint32_t pk[BN / 2];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        uint32_t pk[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float p0 = ex2(fmaf(__uint_as_float(sv[c * 8 + 2 * e]), p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[c * 8 + 2 * e + 1]), p.scale_log2, neg_m));
-          sum += p0 + p1;
-          pk[e] = pack_bf16(p0, p1);
-        }
-        *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      for (int j = 0; j < BN / 2; ++j) {
+        const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+        sum += p0 + p1;
+        pk[j] = pack_bf16(p0, p1);
       }
+      tmem_st_x32(tmem_P(slot) + lane_addr, pk);   // P stays in tensor memory as the A operand
+      tmem_wait_st();
       l_run += sum;
 
       if (v_rows < BN) {
@@ -497,8 +505,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int vr = v_rows + (rem >> 3), ch = rem & 7;
           *reinterpret_cast<uint4*>(vt + half * (kKVTile / 2) + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
         }
+        fence_async_smem();   // cleared V rows visible to the tensor core's reads
       }
-      fence_async_smem();   // P (and cleared V rows) visible to the tensor core's reads
       tc_fence_before();
       mbar_arrive(bar_p_full(slot));
     }
@@ -539,17 +547,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int pi = (MT == 2) ? split : split * 2 + slot;
         float* po = p.part_o + ((rt * partials + pi) * BM + row) * (int64_t)HD;
         float* pml = p.part_ml + ((rt * partials + pi) * BM + row) * 2;
-        if (rounds > 0) {
 #pragma unroll 1
-          for (int c = 0; c < HD; c += 32) {
-            uint32_t ov[32];
+        for (int c = 0; c < HD; c += 32) {
+          uint32_t ov[32];
+          if (rounds > 0) {
             tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
             tmem_wait_ld();
+          } else {  // a slot without tiles publishes zeros so the merge can read unconditionally
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4)
-              __stcg(reinterpret_cast<uint4*>(po + c + q4 * 4),
-                     make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]));
+            for (int j = 0; j < 32; ++j) ov[j] = 0u;
           }
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            __stcg(reinterpret_cast<uint4*>(po + c + q4 * 4),
+                   make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]));
         }
         __stcg(reinterpret_cast<float2*>(pml), make_float2(rounds > 0 ? m_ref : -INFINITY, rounds > 0 ? l_run : 0.f));
       }
@@ -561,19 +572,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (*abort_flag) {
     if (warp == 0 && lane == 0) {
       // TMA copies that were issued land on their own; wait for the newest phase of each stage
-      for (int i = max(0, issued_tiles - NST); i < issued_tiles; ++i) {
-        const unsigned long long t0 = globaltimer_ns();
-        while (!mbar_try(bar_kv_full(i % NST), (i / NST) & 1) && globaltimer_ns() - t0 < kWaitLimitNs) {}
-      }
-      if (n_tiles > 0) {
-        const unsigned long long t0 = globaltimer_ns();
-        while (!mbar_try(bar_q, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
-      }
+      for (int i = max(0, issued_tiles - NST); i < issued_tiles; ++i)
+        mbar_drain(bar_kv_full(i % NST), (i / NST) & 1);
+      if (n_tiles > 0) mbar_drain(bar_q, 0);
     }
     if (warp == 1 && lane == 0) {
       umma_commit(bar_drain);  // completes when every MMA issued so far has finished
-      const unsigned long long t0 = globaltimer_ns();
-      while (!mbar_try(bar_drain, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      mbar_drain(bar_drain, 0);
     }
   }
   tc_fence_before();
@@ -638,11 +643,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
     for (int q = 0; q < partials; ++q) {
-      const float w = s_w[q * n_rows + rr];
-      if (w != 0.f) {  // a skipped partial may hold anything, even NaN
-        const float4 x = __ldcg(reinterpret_cast<const float4*>(po + (int64_t)q * BM * HD));
-        acc.x += w * x.x; acc.y += w * x.y; acc.z += w * x.z; acc.w += w * x.w;
-      }
+      const float w = s_w[q * n_rows + rr];   // every partial holds finite numbers
+      const float4 x = __ldcg(reinterpret_cast<const float4*>(po + (int64_t)q * BM * HD));
+      acc.x += w * x.x; acc.y += w * x.y; acc.z += w * x.z; acc.w += w * x.w;
     }
     uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD + piece * 4;
     *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
