@@ -9,19 +9,25 @@
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
 //   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
 //           accumulators are merged like split-KV partials.
+// Split-KV: the blocks that share a row tile form a thread-block cluster; each stages its
+// accumulators in its own shared memory and every block finalises a share of the rows by reading
+// its peers' staging areas (distributed shared memory), so no partial result touches global memory.
 // Per slot and key tile:  S = Q K^T (tcgen05.mma -> TMEM)  ->  softmax thread reads its row of S,
-// masks, exponentiates against a lazily updated reference maximum, writes P (bf16) to shared
-// memory  ->  O += P V (tcgen05.mma, accumulator stays in TMEM).  While one slot is in its softmax
+// masks, exponentiates against a lazily updated reference maximum, writes P (bf16) back to tensor
+// memory  ->  O += P V (tcgen05.mma with A from TMEM, accumulator stays in TMEM).  While one slot is in its softmax
 // the tensor core works for the other.  The tree columns are masked with per-node ancestor
 // bitsets derived from parent[] on chip; masked scores are replaced, not added to, so they
 // contribute exactly zero.  Every mbarrier wait is bounded: on expiry the block raises a flag,
 // all roles leave their loops, in-flight copies and MMAs are drained, TMEM is released and
 // CLV_ERR_TIMEOUT is reported for the sequence.
+#include <cooperative_groups.h>
 #include <cuda.h>
 #include <math.h>
 
 #include "clv_internal.cuh"
 #include "tmem_access.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace clv {
 namespace {
@@ -49,13 +55,10 @@ struct Params {
   uint16_t* out;
   float* lse;
   int32_t* status;
-  unsigned* tickets;
-  float* part_o;   // [row tile][partial][128][128]
-  float* part_ml;  // [row tile][partial][128][2]
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
   int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
-  int splits;      // thread blocks along the key axis
+  int splits;      // thread blocks along the key axis = cluster size (1, 2, 4 or 8)
   float scale_log2;
 };
 
@@ -195,7 +198,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ __align__(8) unsigned long long s_bar[2 * NST + 1 + 6 + 1];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ int s_last;
+  __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.x / p.row_ctas, row_cta = blockIdx.x - unit * p.row_ctas;
@@ -291,6 +294,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto tmem_O = [&](int s) { return tmem + (uint32_t)(3 * BN + s * HD); };
 
   int issued_tiles = 0;  // producer bookkeeping for the drain
+
+  // per-thread state of the softmax groups (warps 2..9); declared here because the epilogue runs
+  // after block-wide synchronisation points that all roles must reach together
+  const int slot = warp >= 2 ? (warp - 2) >> 2 : 0;
+  const int quarter = warp & 3;                  // TMEM lanes this warp may touch
+  const int row = quarter * 32 + lane;           // row inside the 128-row tile
+  const int my_rounds = slot == 0 ? rounds0 : rounds1;
+  const int r_glob = (row_cta * MT + ((MT == 2) ? slot : 0)) * BM + row;
+  const bool row_valid = r_glob < rows_total;
+  const int node = row_valid ? r_glob / G : 0;
+  const int gq = row_valid ? r_glob - node * G : 0;
+  const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+  float m_ref = -INFINITY, l_run = 0.f;
 
   if (warp == 0) {
     // =========================== TMA producer ===============================================
@@ -395,17 +411,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   } else {
     // =========================== softmax groups ===============================================
-    const int slot = (warp - 2) >> 2;
-    const int quarter = warp & 3;                  // TMEM lanes this warp may touch
-    const int row = quarter * 32 + lane;           // row inside the 128-row tile
-    const int rounds = slot == 0 ? rounds0 : rounds1;
-    const int mtile = row_cta * MT + ((MT == 2) ? slot : 0);
-    const int r_glob = mtile * BM + row;
-    const bool row_valid = r_glob < rows_total;
-    const int node = row_valid ? r_glob / G : 0;
-    const int gq = row_valid ? r_glob - node * G : 0;
-    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-    float m_ref = -INFINITY, l_run = 0.f;
+    const int rounds = my_rounds;
     bool ok = true;
 
     for (int r = 0; r < rounds && ok; ++r) {
@@ -511,63 +517,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_arrive(bar_p_full(slot));
     }
 
-    // ---- epilogue of this slot: final O out of TMEM ------------------------------------------
-    if (ok && rounds > 0) {
+    if (ok && rounds > 0) {  // the last P V of this slot has landed in O
       ok = mbar_wait(bar_pv_done(slot), (rounds - 1) & 1, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
-      if (ok) tc_fence_after();
-    }
-    const int partials = p.splits * (MT == 1 ? 2 : 1);
-    if (ok) {
-      const float kLn2 = 0.6931471805599453f;
-      if (partials == 1) {
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-        uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD;
-#pragma unroll 1
-        for (int c = 0; c < HD; c += 32) {
-          uint32_t ov[32];
-          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
-          tmem_wait_ld();
-          if (row_valid) {
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              uint4 v;
-              v.x = pack_bf16(__uint_as_float(ov[q4 * 8 + 0]) * inv, __uint_as_float(ov[q4 * 8 + 1]) * inv);
-              v.y = pack_bf16(__uint_as_float(ov[q4 * 8 + 2]) * inv, __uint_as_float(ov[q4 * 8 + 3]) * inv);
-              v.z = pack_bf16(__uint_as_float(ov[q4 * 8 + 4]) * inv, __uint_as_float(ov[q4 * 8 + 5]) * inv);
-              v.w = pack_bf16(__uint_as_float(ov[q4 * 8 + 6]) * inv, __uint_as_float(ov[q4 * 8 + 7]) * inv);
-              *reinterpret_cast<uint4*>(dst + c + q4 * 8) = v;
-            }
-          }
-        }
-        if (p.lse != nullptr && row_valid)
-          p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
-      } else {
-        const int64_t rt = (int64_t)blockIdx.x * MT + ((MT == 2) ? slot : 0);
-        const int pi = (MT == 2) ? split : split * 2 + slot;
-        float* po = p.part_o + ((rt * partials + pi) * BM + row) * (int64_t)HD;
-        float* pml = p.part_ml + ((rt * partials + pi) * BM + row) * 2;
-#pragma unroll 1
-        for (int c = 0; c < HD; c += 32) {
-          uint32_t ov[32];
-          if (rounds > 0) {
-            tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
-            tmem_wait_ld();
-          } else {  // a slot without tiles publishes zeros so the merge can read unconditionally
-#pragma unroll
-            for (int j = 0; j < 32; ++j) ov[j] = 0u;
-          }
-#pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4)
-            __stcg(reinterpret_cast<uint4*>(po + c + q4 * 4),
-                   make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]));
-        }
-        __stcg(reinterpret_cast<float2*>(pml), make_float2(rounds > 0 ? m_ref : -INFINITY, rounds > 0 ? l_run : 0.f));
-      }
     }
   }
 
-  // ---- teardown: drain what is still in flight, release TMEM --------------------------------
+  // ---- every role meets here: all MMAs and copies of this block are complete -----------------
   __syncwarp();
   if (*abort_flag) {
     if (warp == 0 && lane == 0) {
@@ -582,74 +538,110 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   }
   tc_fence_before();
-  __threadfence();
   __syncthreads();
   tc_fence_after();
-  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-  if (*abort_flag) {
-    if (tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
-    return;
-  }
-
-  // ---- merge of the partial results ------------------------------------------------------------
-  const int partials = p.splits * (MT == 1 ? 2 : 1);
-  if (partials == 1) return;
-  if (p.splits > 1) {
-    if (tid == 0) {
-      const unsigned arrived = atomicInc(p.tickets + blockIdx.x, (unsigned)p.splits - 1);  // wraps to 0
-      s_last = (arrived == (unsigned)p.splits - 1);
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-  }
-  // Phase 1: one thread per output row turns the (m, l) pairs into normalised weights, kept in the
-  // (now idle) tile memory.  Phase 2: every thread combines 4-column pieces, 32 consecutive
-  // threads covering one 512-byte row of each partial, all loads independent of each other.
+  const bool aborted = *abort_flag != 0;
+  const int n_src = p.splits * (MT == 1 ? 2 : 1);  // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
-  float* s_w = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));  // [partial][MT*128]
-  const int n_rows = MT * BM;
-  for (int rr = tid; rr < n_rows; rr += kThreads) {
-    const int row = rr % BM;
-    const int64_t rt = (int64_t)blockIdx.x * MT + rr / BM;
-    const float* ml = p.part_ml + (rt * partials * BM + row) * 2;
-    float mmax = -INFINITY;
-    for (int q = 0; q < partials; ++q) mmax = fmaxf(mmax, __ldcg(ml + (int64_t)q * BM * 2));
-    const float mu = (mmax == -INFINITY) ? 0.f : mmax;
-    float lsum = 0.f;
-    for (int q = 0; q < partials; ++q) {
-      const float2 v = __ldcg(reinterpret_cast<const float2*>(ml + (int64_t)q * BM * 2));
-      const float w = (v.y > 0.f) ? ex2(v.x - mu) : 0.f;  // an empty partial gets weight 0
-      s_w[q * n_rows + rr] = w;
-      lsum += w * v.y;
-    }
-    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-    for (int q = 0; q < partials; ++q) s_w[q * n_rows + rr] *= inv;
-    const int r_glob = (row_cta * MT + rr / BM) * BM + row;
-    if (p.lse != nullptr && r_glob < rows_total) {
-      const int node = r_glob / G, gq = r_glob - node * G;
-      p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (mmax + log2f(lsum)) * kLn2;
+  // staging area for the merge: O of both slots as fp32 [slot][128 rows][128], 16-byte chunk c of
+  // row r stored at chunk (c ^ (r & 31)) so that row-per-thread writes and row-per-warp reads are
+  // both conflict free.  It reuses the tile memory, which nothing reads any more.
+  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));
+
+  if (!aborted && warp >= 2) {
+    if (n_src == 1) {
+      // only accumulator of these rows: normalise and store
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD; c += 32) {
+        uint32_t ov[32];
+        tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+        tmem_wait_ld();
+        if (row_valid) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(ov[q4 * 8 + 0]) * inv, __uint_as_float(ov[q4 * 8 + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(ov[q4 * 8 + 2]) * inv, __uint_as_float(ov[q4 * 8 + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(ov[q4 * 8 + 4]) * inv, __uint_as_float(ov[q4 * 8 + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(ov[q4 * 8 + 6]) * inv, __uint_as_float(ov[q4 * 8 + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + c + q4 * 8) = v;
+          }
+        }
+      }
+      if (p.lse != nullptr && row_valid)
+        p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
+    } else {
+      float* orow = sO + ((size_t)slot * BM + row) * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD; c += 32) {
+        uint32_t ov[32];
+        if (my_rounds > 0) {
+          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+          tmem_wait_ld();
+        } else {  // a slot without tiles contributes zeros with weight zero
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ov[j] = 0u;
+        }
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) {
+          const int chunk = (c >> 2) + q4;
+          *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 31)) << 2)) =
+              make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]);
+        }
+      }
+      s_ml[slot][row] = make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f);
     }
   }
+  tc_fence_before();
   __syncthreads();
-  for (int item = tid; item < n_rows * 32; item += kThreads) {
-    const int rr = item >> 5, piece = item & 31;
-    const int row = rr % BM;
-    const int r_glob = (row_cta * MT + rr / BM) * BM + row;
-    if (r_glob >= rows_total) continue;
-    const int node = r_glob / G, gq = r_glob - node * G;
-    const int64_t rt = (int64_t)blockIdx.x * MT + rr / BM;
-    const float* po = p.part_o + (rt * partials * BM + row) * (int64_t)HD + piece * 4;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+  if (aborted && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
+  if (n_src == 1) return;  // such a block is its own cluster
+
+  // ---- merge across the cluster (the split-KV blocks of one row tile) through distributed
+  //      shared memory: rank j finalises rows [j, j+1) * rows/splits of the tile(s) ------------
+  cg::cluster_group cluster = cg::this_cluster();
+  cluster.sync();  // every block's staging area is complete (also reached by an aborted block)
+  if (!aborted) {
+    const int n_rows = MT * BM, per_rank = n_rows / p.splits;
+    for (int rr = split * per_rank + warp; rr < (split + 1) * per_rank; rr += kThreads / 32) {
+      const int tile = rr / BM, trow = rr % BM;
+      const int rg = (row_cta * MT + tile) * BM + trow;
+      if (rg >= rows_total) continue;
+      const int onode = rg / G, ogq = rg - onode * G;
+      // source q: (block q, slot `tile`) when MT == 2, (block q / 2, slot q % 2) when MT == 1
+      const int src_cta = (MT == 2) ? lane : lane >> 1;
+      const int src_slot = (MT == 2) ? tile : lane & 1;
+      float2 ml = make_float2(-INFINITY, 0.f);
+      if (lane < n_src) ml = cluster.map_shared_rank(&s_ml[0][0], src_cta)[src_slot * BM + trow];
+      float mmax = ml.x;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
+      const float mu = (mmax == -INFINITY) ? 0.f : mmax;
+      float w = (ml.y > 0.f) ? ex2(ml.x - mu) : 0.f;
+      float lsum = w * ml.y;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+      w *= (lsum > 0.f ? 1.f / lsum : 0.f);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int chunk_off = (lane ^ (trow & 31)) << 2;
 #pragma unroll 4
-    for (int q = 0; q < partials; ++q) {
-      const float w = s_w[q * n_rows + rr];   // every partial holds finite numbers
-      const float4 x = __ldcg(reinterpret_cast<const float4*>(po + (int64_t)q * BM * HD));
-      acc.x += w * x.x; acc.y += w * x.y; acc.z += w * x.z; acc.w += w * x.w;
+      for (int q = 0; q < n_src; ++q) {
+        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+        const float wq = __shfl_sync(0xFFFFFFFFu, w, q);
+        const float* src = cluster.map_shared_rank(sO, qc) + ((size_t)qs * BM + trow) * HD + chunk_off;
+        const float4 x = *reinterpret_cast<const float4*>(src);
+        acc.x += wq * x.x; acc.y += wq * x.y; acc.z += wq * x.z; acc.w += wq * x.w;
+      }
+      uint16_t* dst = p.out + (((int64_t)b * N + onode) * p.Hq + kvh * G + ogq) * HD + lane * 4;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+      if (p.lse != nullptr && lane == 0)
+        p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
     }
-    uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD + piece * 4;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
   }
+  cluster.sync();  // no block may leave while a peer still reads its shared memory
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -706,16 +698,15 @@ AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
   pl.m_tiles = row_ctas;
   const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * row_ctas;
   const int key_tiles = (max_ctx_len > 0 ? (max_ctx_len + BN - 1) / BN : 0) + (s.n_nodes + BN - 1) / BN;
-  int64_t want = sm_count() / (ctas > 0 ? ctas : 1);   // one resident block per SM
-  const int per_cta_min = mt == 1 ? 2 : 1;             // MT == 1 blocks eat two tiles per round
-  if (want > key_tiles / per_cta_min) want = key_tiles / per_cta_min;
-  if (want > 32) want = 32;                            // weights of all partials fit the tile memory
-  if (want < 1 || ctas > kTickets) want = 1;
-  pl.splits = (int)want;
-  pl.tickets = pl.splits > 1 ? (int)ctas : 0;
-  const int partials = pl.splits * (mt == 1 ? 2 : 1);
-  pl.scratch_bytes = partials > 1
-      ? (size_t)ctas * mt * partials * (BM * HD + BM * 2) * sizeof(float) : 0;
+  // The key axis is split over a thread-block cluster (merged through distributed shared memory),
+  // so the split count is a power of two up to the portable cluster size; one block per SM.
+  const int per_cta_min = mt == 1 ? 2 : 1;  // MT == 1 blocks eat two tiles per round
+  int splits = 1;
+  while (splits < 8 && ctas * (splits * 2) <= sm_count() && key_tiles / (splits * 2) >= per_cta_min)
+    splits *= 2;
+  pl.splits = splits;
+  pl.tickets = 0;
+  pl.scratch_bytes = 0;  // nothing goes through global memory
   return pl;
 }
 
@@ -724,6 +715,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
                                 cudaStream_t stream) {
+  (void)tickets; (void)scratch;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = G * s.n_nodes;
   const int mt = rows > BM ? 2 : 1;
@@ -754,22 +746,27 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.status = status;
-  p.tickets = tickets;
   const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
-  const int partials = plan.splits * (mt == 1 ? 2 : 1);
-  p.part_o = static_cast<float*>(scratch);
-  p.part_ml = p.part_o + ctas * mt * partials * (int64_t)(BM * HD);
   p.B = s.batch; p.N = s.n_nodes; p.Hq = s.n_q_heads; p.Hkv = s.n_kv_heads; p.G = G;
   p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
   p.row_ctas = plan.m_tiles;
   p.splits = plan.splits;
   p.scale_log2 = scale * 1.4426950408889634f;
-  dim3 grid((unsigned)ctas, (unsigned)plan.splits, 1);
-  if (mt == 1)
-    tree_attn_tc_kernel<1><<<grid, kThreads, Cfg<1>::kSmem, stream>>>(tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
-  else
-    tree_attn_tc_kernel<2><<<grid, kThreads, Cfg<2>::kSmem, stream>>>(tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
-  return cudaGetLastError();
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)ctas, (unsigned)plan.splits, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = mt == 1 ? Cfg<1>::kSmem : Cfg<2>::kSmem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;  // the blocks that split one row tile's keys
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = (unsigned)plan.splits;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (mt == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<2>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
 }
 
 }  // namespace clv
