@@ -199,6 +199,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
+  __shared__ float2 s_src[2 * BM]; // merge: (weight, sum) of every (row of this rank, source)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.x / p.row_ctas, row_cta = blockIdx.x - unit * p.row_ctas;
@@ -371,18 +372,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       bool ok = mbar_wait(bar_q, 0, abort_flag);
       tc_fence_after();
       auto local_tile = [&](int s, int r) { return (MT == 2) ? r : 2 * r + s; };
+      // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
+      // constant (the address field counts 16-byte units and never carries out of its 14 bits).
+      const uint64_t q_desc = smem_desc(sQ, 16, 1024);
+      const uint64_t k_desc = smem_desc(sKV, 16, 1024);
+      const uint64_t v_desc = smem_desc(sKV + kKVTile, kKVTile / 2, 1024);
       auto issue_qk = [&](int s, int r) -> bool {
         const int i = local_tile(s, r), st = i % NST;
         if (!mbar_wait(bar_kv_full(st), (i / NST) & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t qb = sQ + ((MT == 2) ? s : 0) * kQTile;
-        const uint32_t kb = sKV + st * 2 * kKVTile;
+        const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
+        const uint64_t kd = k_desc + (uint64_t)((st * 2 * kKVTile) >> 4);
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
           const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
           const uint32_t ko = (ks >> 2) * (kKVTile / 2) + (ks & 3) * 32;
-          umma_bf16(tmem_S(s), smem_desc(qb + qo, 16, 1024), smem_desc(kb + ko, 16, 1024), kIdescQK,
-                    ks > 0 ? 1u : 0u);
+          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar_s_full(s));
         return true;
@@ -397,11 +402,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (!ok) break;
           tc_fence_after();
           const int i = local_tile(s, r), st = i % NST;
-          const uint32_t vb = sKV + st * 2 * kKVTile + kKVTile;
+          const uint64_t vd = v_desc + (uint64_t)((st * 2 * kKVTile) >> 4);
 #pragma unroll
           for (int kk = 0; kk < BN / 16; ++kk) {
-            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, smem_desc(vb + kk * 2048, kKVTile / 2, 1024),
-                         kIdescPV, (r > 0 || kk > 0) ? 1u : 0u);
+            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                         (r > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(bar_pv_done(s));
           if (MT == 1 || s == 1) umma_commit(bar_kv_empty(st));  // last reader of this stage
@@ -605,40 +610,75 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   cg::cluster_group cluster = cg::this_cluster();
   cluster.sync();  // every block's staging area is complete (also reached by an aborted block)
   if (!aborted) {
-    const int n_rows = MT * BM, per_rank = n_rows / p.splits;
-    for (int rr = split * per_rank + warp; rr < (split + 1) * per_rank; rr += kThreads / 32) {
-      const int tile = rr / BM, trow = rr % BM;
-      const int rg = (row_cta * MT + tile) * BM + trow;
-      if (rg >= rows_total) continue;
-      const int onode = rg / G, ogq = rg - onode * G;
-      // source q: (block q, slot `tile`) when MT == 2, (block q / 2, slot q % 2) when MT == 1
-      const int src_cta = (MT == 2) ? lane : lane >> 1;
-      const int src_slot = (MT == 2) ? tile : lane & 1;
-      float2 ml = make_float2(-INFINITY, 0.f);
-      if (lane < n_src) ml = cluster.map_shared_rank(&s_ml[0][0], src_cta)[src_slot * BM + trow];
-      float mmax = ml.x;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
+    // Every rank finalises per_rank rows; per_rank * n_src is 256 whatever the split count.
+    const int per_rank = MT * BM / p.splits;
+    // (a) fetch the (maximum, sum) pair of every (row, source); source q is (block q, slot `tile`)
+    //     when MT == 2 and (block q / 2, slot q % 2) when MT == 1
+    if (tid < per_rank * n_src) {
+      const int k = tid / n_src, q = tid - k * n_src;
+      const int rr = split * per_rank + k, tile = rr / BM, trow = rr % BM;
+      const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+      s_src[tid] = cluster.map_shared_rank(&s_ml[0][0], qc)[qs * BM + trow];
+    }
+    __syncthreads();
+    // (b) one thread per row: normalised weights, log-sum-exp
+    if (tid < per_rank) {
+      const int rr = split * per_rank + tid, tile = rr / BM, trow = rr % BM;
+      float mmax = -INFINITY;
+      for (int q = 0; q < n_src; ++q) mmax = fmaxf(mmax, s_src[tid * n_src + q].x);
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
-      float w = (ml.y > 0.f) ? ex2(ml.x - mu) : 0.f;
-      float lsum = w * ml.y;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
-      w *= (lsum > 0.f ? 1.f / lsum : 0.f);
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      const int chunk_off = (lane ^ (trow & 31)) << 2;
-#pragma unroll 4
+      float lsum = 0.f;
       for (int q = 0; q < n_src; ++q) {
-        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-        const float wq = __shfl_sync(0xFFFFFFFFu, w, q);
-        const float* src = cluster.map_shared_rank(sO, qc) + ((size_t)qs * BM + trow) * HD + chunk_off;
-        const float4 x = *reinterpret_cast<const float4*>(src);
-        acc.x += wq * x.x; acc.y += wq * x.y; acc.z += wq * x.z; acc.w += wq * x.w;
+        const float2 v = s_src[tid * n_src + q];
+        const float w = (v.y > 0.f) ? ex2(v.x - mu) : 0.f;
+        s_src[tid * n_src + q].x = w;
+        lsum += w * v.y;
       }
-      uint16_t* dst = p.out + (((int64_t)b * N + onode) * p.Hq + kvh * G + ogq) * HD + lane * 4;
-      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-      if (p.lse != nullptr && lane == 0)
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      for (int q = 0; q < n_src; ++q) s_src[tid * n_src + q].x *= inv;
+      const int rg = (row_cta * MT + tile) * BM + trow;
+      if (p.lse != nullptr && rg < rows_total) {
+        const int onode = rg / G, ogq = rg - onode * G;
         p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
+      }
+    }
+    __syncthreads();
+    // (c) one warp per pair of rows, lane j owns columns 4j..4j+3; all loads of a pair in flight
+    for (int k0 = warp * 2; k0 < per_rank; k0 += 2 * (kThreads / 32)) {
+      float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+      int rg[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int k = min(k0 + u, per_rank - 1);
+        const int rr = split * per_rank + k, tile = rr / BM, trow = rr % BM;
+        rg[u] = (k0 + u < per_rank) ? (row_cta * MT + tile) * BM + trow : rows_total;
+        const int chunk_off = (lane ^ (trow & 31)) << 2;
+        for (int q0 = 0; q0 < n_src; q0 += 4) {  // n_src is 2, 4, 8 or 16
+          float4 x[4];
+          float wq[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int q = min(q0 + j, n_src - 1);
+            const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+            x[j] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sO, qc) +
+                                                    ((size_t)qs * BM + trow) * HD + chunk_off);
+            wq[j] = (q0 + j < n_src) ? s_src[k * n_src + q].x : 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            acc[u].x += wq[j] * x[j].x; acc[u].y += wq[j] * x[j].y;
+            acc[u].z += wq[j] * x[j].z; acc[u].w += wq[j] * x[j].w;
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (rg[u] >= rows_total) continue;
+        const int onode = rg[u] / G, ogq = rg[u] - onode * G;
+        uint16_t* dst = p.out + (((int64_t)b * N + onode) * p.Hq + kvh * G + ogq) * HD + lane * 4;
+        *reinterpret_cast<uint2*>(dst) =
+            make_uint2(pack_bf16(acc[u].x, acc[u].y), pack_bf16(acc[u].z, acc[u].w));
+      }
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
