@@ -3,7 +3,11 @@
 //
 // One thread block owns up to 256 query rows of one (sequence, kv head) - a row is a
 // (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes reuse every
-// K/V byte - and a contiguous range of 64-key tiles (cache tiles first, then the tree's own keys).
+// K/V byte - and a contiguous range of key tiles (cache tiles first, then the tree's own keys).
+// A key tile is 128 keys when the block has two row tiles (an MMA costs about the same for 64 as
+// for 128 columns, so wide S tiles halve the tensor time) and 64 keys otherwise; tiles are loaded
+// as 64-key pieces, which is also the page size of a paged cache.  K and V travel through separate
+// rings so that a K buffer is refilled as soon as its Q K^T is done.
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation), warps 2-5 and
 // 6-9 = two softmax groups of 128 threads, one thread per query row ("slot" 0 and 1).
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
@@ -32,20 +36,22 @@ namespace cg = cooperative_groups;
 namespace clv {
 namespace {
 
-constexpr int BN = 64;                 // keys per tile (= page size)
+constexpr int PG = CLV_PAGE_SIZE;      // 64: keys per TMA piece (= page size)
 constexpr int HD = CLV_HEAD_DIM;       // 128
 constexpr int BM = 128;                // rows per MMA / per slot
 constexpr int kThreads = 320;
 constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
-constexpr uint32_t kKVTile = BN * HD * 2;     // 16 KB: two [64 keys][64 d] swizzled halves
+constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleGap = 8.0f;           // log2 units: P stays below 2^8
 constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: about a second
 
 template <int MT>
 struct Cfg {
-  static constexpr int kStages = (MT == 2) ? 4 : 5;
-  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kKVTile + 1024;
+  static constexpr int BN = (MT == 2) ? 128 : 64;        // keys per tile
+  static constexpr int kStages = (MT == 2) ? 2 : 5;      // ring depth, K and V each
+  static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
+  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kTile + 1024;
 };
 
 struct Params {
@@ -168,11 +174,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
   return d;
 }
 // Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, A K-major.
-constexpr uint32_t make_idesc(int m, int n, bool b_mn_major) {
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
-constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x 64]  = Q[128 x 16k] K[64 x 16k]^T
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
 
 __device__ __forceinline__ float ex2(float x) {
@@ -191,11 +196,16 @@ __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                     const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
                     const __grid_constant__ CUtensorMap tm_vt, const Params p) {
+  constexpr int BN = Cfg<MT>::BN;          // keys per tile
+  constexpr int PPT = BN / PG;             // 64-key pieces per tile
   constexpr int NST = Cfg<MT>::kStages;
+  constexpr uint32_t kTile = Cfg<MT>::kTile;
+  constexpr uint32_t kHalf = kTile / 2;    // one 64-wide half of the head dimension: [BN keys][64 d]
+  constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
-  __shared__ __align__(8) unsigned long long s_bar[2 * NST + 1 + 6 + 1];
+  __shared__ __align__(8) unsigned long long s_bar[4 * NST + 8];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
@@ -216,15 +226,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     bad |= (par < -1 || par >= i);
   }
   bad |= (L < 0);
-  const int t_cache = L > 0 ? (L + BN - 1) / BN : 0;
-  if (p.paged) bad |= (t_cache > p.max_pages);
+  const int p_cache = L > 0 ? (L + PG - 1) / PG : 0;  // 64-key pieces (pages) of the context
+  if (p.paged) bad |= (p_cache > p.max_pages);
   else bad |= (L > p.cap_tokens);
   const int seq_bad = __syncthreads_or(bad ? 1 : 0);
   const bool reporter = (row_cta == 0 && split == 0 && kvh == 0);
   if (reporter) {
     bool pbad = false;
     if (p.paged && !seq_bad) {
-      for (int pg = tid; pg < t_cache; pg += kThreads) {
+      for (int pg = tid; pg < p_cache; pg += kThreads) {
         const int e = p.block_table[(int64_t)b * p.max_pages + pg];
         pbad |= (e < 0 || e >= p.n_pages);
       }
@@ -232,7 +242,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int page_bad = __syncthreads_or(pbad ? 1 : 0);
     if (tid == 0) p.status[b] = (seq_bad || page_bad) ? CLV_ERR_TREE : CLV_OK;
   }
-  if (seq_bad) return;  // before any barrier or TMEM exists
+  if (seq_bad) return;  // before any barrier or TMEM exists; the whole cluster leaves together
 
   // ancestor bitsets: row i of the tree's topology matrix
   for (int i = tid; i < N; i += kThreads) {
@@ -246,6 +256,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
 
   // ---- tile range and per-slot rounds -------------------------------------------------------
+  const int t_cache = (p_cache + PPT - 1) / PPT;
   const int t_tree = (N + BN - 1) / BN;
   const int t_total = t_cache + t_tree;
   const int t_begin = (int)((int64_t)split * t_total / p.splits);
@@ -258,20 +269,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem_base;
-  const uint32_t sKV = sQ + MT * kQTile;             // stage i: K at +i*32K, V at +i*32K + 16K
-  uint8_t* const sKV_gen = smem_raw + (sKV - smem_u32(smem_raw));
+  const uint32_t sK = sQ + MT * kQTile;      // ring of NST K tiles
+  const uint32_t sV = sK + NST * kTile;      // ring of NST V tiles
+  uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
 
   const uint32_t bar0 = smem_u32(&s_bar[0]);
-  auto bar_kv_full = [&](int st) { return bar0 + 8u * st; };
-  auto bar_kv_empty = [&](int st) { return bar0 + 8u * (NST + st); };
-  const uint32_t bar_q = bar0 + 8u * (2 * NST);
-  auto bar_s_full = [&](int s) { return bar0 + 8u * (2 * NST + 1 + s); };
-  auto bar_p_full = [&](int s) { return bar0 + 8u * (2 * NST + 3 + s); };
-  auto bar_pv_done = [&](int s) { return bar0 + 8u * (2 * NST + 5 + s); };
-  const uint32_t bar_drain = bar0 + 8u * (2 * NST + 7);
+  auto bar_k_full = [&](int st) { return bar0 + 8u * st; };
+  auto bar_k_empty = [&](int st) { return bar0 + 8u * (NST + st); };
+  auto bar_v_full = [&](int st) { return bar0 + 8u * (2 * NST + st); };
+  auto bar_v_empty = [&](int st) { return bar0 + 8u * (3 * NST + st); };
+  const uint32_t bar_q = bar0 + 8u * (4 * NST);
+  auto bar_s_full = [&](int s) { return bar0 + 8u * (4 * NST + 1 + s); };
+  auto bar_p_full = [&](int s) { return bar0 + 8u * (4 * NST + 3 + s); };
+  auto bar_pv_done = [&](int s) { return bar0 + 8u * (4 * NST + 5 + s); };
+  const uint32_t bar_drain = bar0 + 8u * (4 * NST + 7);
 
   if (tid == 0) {
-    for (int i = 0; i < NST; ++i) { mbar_init(bar_kv_full(i), 1); mbar_init(bar_kv_empty(i), 1); }
+    for (int i = 0; i < 4 * NST; ++i) mbar_init(bar0 + 8u * i, 1);
     mbar_init(bar_q, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_s_full(s), 1);
@@ -289,10 +303,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abort_flag = &s_abort;
-  // columns: S of slot s at 64 s; P (bf16 pairs) at 128 + 32 s; O at 192 + 128 s
+  // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
+  // the scores have been read); O of slot s at 2 BN + 128 s
   auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_P = [&](int s) { return tmem + (uint32_t)(2 * BN + s * (BN / 2)); };
-  auto tmem_O = [&](int s) { return tmem + (uint32_t)(3 * BN + s * HD); };
+  auto tmem_P = [&](int s) { return tmem + (uint32_t)(s * BN); };
+  auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + s * HD); };
 
   int issued_tiles = 0;  // producer bookkeeping for the drain
 
@@ -326,39 +341,58 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tma_load_3d(sQ + m * kQTile + kQTile / 2, &tm_q, 64, kvh * G, node0, bar_q);
         }
       }
-      int page_cache = 0;  // lane j holds the pool page of cache tile (batch base + j)
+      constexpr int kBatch = 32 / PPT;  // tiles whose page numbers one warp-wide fetch covers
+      int page_cache = 0;               // lane j: pool page of piece (batch base * PPT + j)
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int t = t_begin + i;
         const int st = i % NST;
-        if (p.paged && (i % 32) == 0) {
-          const int tt = t + lane;
-          page_cache = (tt < t_cache) ? p.block_table[(int64_t)b * p.max_pages + tt] : 0;
+        if (p.paged && (i % kBatch) == 0) {
+          const int pc = t * PPT + lane;
+          page_cache = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
         }
-        int pg = __shfl_sync(0xFFFFFFFFu, page_cache, i % 32);
+        int row0[PPT];   // first source row of each piece, -1: piece not present
+        const CUtensorMap *mk, *mv;
+        if (t < t_cache) {
+          mk = &tm_kc; mv = &tm_vc;
+#pragma unroll
+          for (int j = 0; j < PPT; ++j) {
+            const int pc = t * PPT + j;
+            int pg = __shfl_sync(0xFFFFFFFFu, page_cache, (i % kBatch) * PPT + j);
+            if (pg < 0 || pg >= p.n_pages) pg = 0;  // flagged by the reporter; its keys get masked
+            row0[j] = (pc >= p_cache) ? -1 : (p.paged ? pg * PG : b * p.cap_tokens + pc * PG);
+          }
+        } else {
+          mk = &tm_kt; mv = &tm_vt;
+#pragma unroll
+          for (int j = 0; j < PPT; ++j) {
+            const int j0 = (t - t_cache) * BN + j * PG;
+            row0[j] = (j0 < N) ? b * N + j0 : -1;
+          }
+        }
         if (lane == 0) {
-          if (i >= NST) ok = mbar_wait(bar_kv_empty(st), ((i / NST) - 1) & 1, abort_flag);
+          int n_pieces = 0;
+#pragma unroll
+          for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
+          const uint32_t bytes = (uint32_t)n_pieces * 2u * kPiece;  // both halves of the head dim
+          if (i >= NST) ok = mbar_wait(bar_k_empty(st), ((i / NST) - 1) & 1, abort_flag);
           if (ok) {
-            const uint32_t dK = sKV + st * 2 * kKVTile, dV = dK + kKVTile;
-            mbar_expect_tx(bar_kv_full(st), 2 * kKVTile);
-            if (t < t_cache) {
-              int row0;
-              if (p.paged) {
-                if (pg < 0 || pg >= p.n_pages) pg = 0;  // flagged by the reporter; rows get masked
-                row0 = pg * BN;
-              } else {
-                row0 = b * p.cap_tokens + t * BN;
-              }
-              tma_load_3d(dK, &tm_kc, 0, kvh, row0, bar_kv_full(st));
-              tma_load_3d(dK + kKVTile / 2, &tm_kc, 64, kvh, row0, bar_kv_full(st));
-              tma_load_3d(dV, &tm_vc, 0, kvh, row0, bar_kv_full(st));
-              tma_load_3d(dV + kKVTile / 2, &tm_vc, 64, kvh, row0, bar_kv_full(st));
-            } else {
-              const int row0 = b * N + (t - t_cache) * BN;
-              tma_load_3d(dK, &tm_kt, 0, kvh, row0, bar_kv_full(st));
-              tma_load_3d(dK + kKVTile / 2, &tm_kt, 64, kvh, row0, bar_kv_full(st));
-              tma_load_3d(dV, &tm_vt, 0, kvh, row0, bar_kv_full(st));
-              tma_load_3d(dV + kKVTile / 2, &tm_vt, 64, kvh, row0, bar_kv_full(st));
+            mbar_expect_tx(bar_k_full(st), bytes);
+#pragma unroll
+            for (int j = 0; j < PPT; ++j) {
+              if (row0[j] < 0) continue;
+              tma_load_3d(sK + st * kTile + j * kPiece, mk, 0, kvh, row0[j], bar_k_full(st));
+              tma_load_3d(sK + st * kTile + kHalf + j * kPiece, mk, 64, kvh, row0[j], bar_k_full(st));
+            }
+            if (i >= NST) ok = mbar_wait(bar_v_empty(st), ((i / NST) - 1) & 1, abort_flag);
+          }
+          if (ok) {
+            mbar_expect_tx(bar_v_full(st), bytes);
+#pragma unroll
+            for (int j = 0; j < PPT; ++j) {
+              if (row0[j] < 0) continue;
+              tma_load_3d(sV + st * kTile + j * kPiece, mv, 0, kvh, row0[j], bar_v_full(st));
+              tma_load_3d(sV + st * kTile + kHalf + j * kPiece, mv, 64, kvh, row0[j], bar_v_full(st));
             }
             issued_tiles = i + 1;
           }
@@ -375,21 +409,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
       // constant (the address field counts 16-byte units and never carries out of its 14 bits).
       const uint64_t q_desc = smem_desc(sQ, 16, 1024);
-      const uint64_t k_desc = smem_desc(sKV, 16, 1024);
-      const uint64_t v_desc = smem_desc(sKV + kKVTile, kKVTile / 2, 1024);
+      const uint64_t k_desc = smem_desc(sK, 16, 1024);
+      const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
       auto issue_qk = [&](int s, int r) -> bool {
         const int i = local_tile(s, r), st = i % NST;
-        if (!mbar_wait(bar_kv_full(st), (i / NST) & 1, abort_flag)) return false;
+        if (!mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
-        const uint64_t kd = k_desc + (uint64_t)((st * 2 * kKVTile) >> 4);
+        const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
           const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
-          const uint32_t ko = (ks >> 2) * (kKVTile / 2) + (ks & 3) * 32;
+          const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
           umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar_s_full(s));
+        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
         return true;
       };
       const int rounds[2] = {rounds0, rounds1};
@@ -400,22 +435,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (r >= rounds[s]) continue;
           ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
           if (!ok) break;
-          tc_fence_after();
           const int i = local_tile(s, r), st = i % NST;
-          const uint64_t vd = v_desc + (uint64_t)((st * 2 * kKVTile) >> 4);
+          ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
           for (int kk = 0; kk < BN / 16; ++kk) {
             umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                          (r > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(bar_pv_done(s));
-          if (MT == 1 || s == 1) umma_commit(bar_kv_empty(st));  // last reader of this stage
+          if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
           if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
         }
       }
     }
   } else {
     // =========================== softmax groups ===============================================
+    constexpr int NH = BN / 64;   // the row of S is taken in 64-column halves (register budget)
     const int rounds = my_rounds;
     bool ok = true;
 
@@ -424,50 +462,69 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int t = t_begin + i;
       const int st = i % NST;
       // allowed columns of this row in this tile, and how many V rows of the tile are real
-      uint32_t a_lo, a_hi;
+      uint32_t allow[BN / 32];
       int v_rows;
       if (t < t_cache) {
         v_rows = min(BN, L - t * BN);
         if (p.paged) {
-          const int pg = p.block_table[(int64_t)b * p.max_pages + t];
-          if (pg < 0 || pg >= p.n_pages) v_rows = 0;
+#pragma unroll
+          for (int j = 0; j < PPT; ++j) {
+            const int pc = t * PPT + j;
+            if (pc < p_cache) {
+              const int pg = p.block_table[(int64_t)b * p.max_pages + pc];
+              if (pg < 0 || pg >= p.n_pages) v_rows = 0;  // sequence is flagged; hide the tile
+            }
+          }
         }
-        const uint64_t bits = v_rows >= 64 ? ~0ull : ((1ull << v_rows) - 1ull);
-        a_lo = (uint32_t)bits; a_hi = (uint32_t)(bits >> 32);
+#pragma unroll
+        for (int w = 0; w < BN / 32; ++w) {
+          const int left = v_rows - 32 * w;
+          allow[w] = left >= 32 ? 0xFFFFFFFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
+        }
       } else {
         const int tt = t - t_cache;
         v_rows = min(BN, N - tt * BN);
-        a_lo = s_anc[node][2 * tt]; a_hi = s_anc[node][2 * tt + 1];
+#pragma unroll
+        for (int w = 0; w < BN / 32; ++w) allow[w] = s_anc[node][tt * (BN / 32) + w];
       }
-      if (!row_valid) a_lo = a_hi = 0;
-      const bool full = (a_lo & a_hi) == 0xFFFFFFFFu;
+      bool full = row_valid;
+#pragma unroll
+      for (int w = 0; w < BN / 32; ++w) {
+        if (!row_valid) allow[w] = 0;
+        full = full && (allow[w] == 0xFFFFFFFFu);
+      }
+      const bool all_full = __all_sync(0xFFFFFFFFu, full);
 
       ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t sv[BN];
-      tmem_ld_x64(tmem_S(slot) + lane_addr, sv);
-      tmem_wait_ld();
 
-      float mx = -INFINITY;
-      if (__all_sync(0xFFFFFFFFu, full)) {
+      uint32_t sv[64];
+      // loads half h of the row and replaces the scores of columns that are not allowed by -inf
+      auto load_half = [&](int h) {
+        tmem_ld_x64(tmem_S(slot) + lane_addr + h * 64, sv);
+        tmem_wait_ld();
+        if (!all_full) {
 #pragma unroll
-        for (int j = 0; j < BN; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
-      } else {
-#pragma unroll
-        for (int j = 0; j < BN; ++j) {
-          const uint32_t wbits = j < 32 ? a_lo : a_hi;
-          const float x = ((wbits >> (j & 31)) & 1u) ? __uint_as_float(sv[j]) : -INFINITY;
-          sv[j] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
+          for (int j = 0; j < 64; ++j) {
+            const uint32_t wbits = allow[2 * h + (j >> 5)];
+            if (!((wbits >> (j & 31)) & 1u)) sv[j] = 0xFF800000u;  // -inf
+          }
         }
+      };
+      float mx = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        load_half(h);
+#pragma unroll
+        for (int j = 0; j < 64; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
       }
       mx *= p.scale_log2;  // scale > 0; -inf stays -inf
       const bool need = mx > m_ref + kRescaleGap;  // also true for the first finite maximum
       const bool any_need = __any_sync(0xFFFFFFFFu, need);
 
-      if (r > 0) {  // P buffer free again and O no longer being written
+      if (r > 0) {  // the previous P V has read P and is no longer writing O
         ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
@@ -491,30 +548,35 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float sum = 0.f;
-      uint32_t pk[BN / 2];
 #pragma unroll
-      for (int j = 0; j < BN / 2; ++j) {
-        const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-        sum += p0 + p1;
-        pk[j] = pack_bf16(p0, p1);
+      for (int h = 0; h < NH; ++h) {
+        if (NH > 1) load_half(h);  // with one half the scores are still in registers
+        uint32_t pk[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+          sum += p0 + p1;
+          pk[j] = pack_bf16(p0, p1);
+        }
+        // P (the A operand of P V) takes the place of score columns that have been consumed
+        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, pk);
       }
-      tmem_st_x32(tmem_P(slot) + lane_addr, pk);   // P stays in tensor memory as the A operand
       tmem_wait_st();
       l_run += sum;
 
       if (v_rows < BN) {
-        // Rows of the V tile beyond the real keys hold whatever lies behind them in memory; their
-        // probabilities are exactly 0, but 0 * NaN would poison O, so clear them.
-        ok = mbar_wait(bar_kv_full(st), (i / NST) & 1, abort_flag);
+        // Rows of the V tile beyond the real keys hold whatever lies behind them in memory (or were
+        // never loaded); their probabilities are exactly 0, but 0 * NaN would poison O: clear them.
+        ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        uint8_t* vt = sKV_gen + st * 2 * kKVTile + kKVTile;
-        const int n_chunks = (BN - v_rows) * 8 * 2;  // 16-byte chunks: rows x 8 x two halves
-        for (int c = (warp - 2 - slot * 4) * 32 + lane; c < n_chunks; c += BM) {
-          const int half = c / ((BN - v_rows) * 8), rem = c - half * (BN - v_rows) * 8;
+        uint8_t* vt = sV_gen + st * kTile;
+        const int per_half = (BN - v_rows) * 8;  // 16-byte chunks per half of the head dimension
+        for (int c = (warp - 2 - slot * 4) * 32 + lane; c < 2 * per_half; c += BM) {
+          const int half = c / per_half, rem = c - half * per_half;
           const int vr = v_rows + (rem >> 3), ch = rem & 7;
-          *reinterpret_cast<uint4*>(vt + half * (kKVTile / 2) + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(vt + half * kHalf + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();   // cleared V rows visible to the tensor core's reads
       }
@@ -533,8 +595,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (*abort_flag) {
     if (warp == 0 && lane == 0) {
       // TMA copies that were issued land on their own; wait for the newest phase of each stage
-      for (int i = max(0, issued_tiles - NST); i < issued_tiles; ++i)
-        mbar_drain(bar_kv_full(i % NST), (i / NST) & 1);
+      for (int i = max(0, issued_tiles - NST); i < issued_tiles; ++i) {
+        mbar_drain(bar_k_full(i % NST), (i / NST) & 1);
+        mbar_drain(bar_v_full(i % NST), (i / NST) & 1);
+      }
       if (n_tiles > 0) mbar_drain(bar_q, 0);
     }
     if (warp == 1 && lane == 0) {
@@ -737,6 +801,7 @@ AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
   const int row_ctas = (rows + mt * BM - 1) / (mt * BM);
   pl.m_tiles = row_ctas;
   const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * row_ctas;
+  const int BN = mt == 2 ? Cfg<2>::BN : Cfg<1>::BN;
   const int key_tiles = (max_ctx_len > 0 ? (max_ctx_len + BN - 1) / BN : 0) + (s.n_nodes + BN - 1) / BN;
   // The key axis is split over a thread-block cluster (merged through distributed shared memory),
   // so the split count is a power of two up to the portable cluster size; one block per SM.
@@ -773,10 +838,10 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   const uint64_t cache_rows = c.paged ? (uint64_t)c.n_pages * CLV_PAGE_SIZE : (uint64_t)s.batch * c.cap_tokens;
   const uint64_t tree_rows = (uint64_t)s.batch * s.n_nodes;
   if (!make_map(&tm_q, q, tree_rows, s.n_q_heads, G, BM / G) ||
-      !make_map(&tm_kc, c.k, cache_rows, s.n_kv_heads, 1, BN) ||
-      !make_map(&tm_vc, c.v, cache_rows, s.n_kv_heads, 1, BN) ||
-      !make_map(&tm_kt, k_tree, tree_rows, s.n_kv_heads, 1, BN) ||
-      !make_map(&tm_vt, v_tree, tree_rows, s.n_kv_heads, 1, BN))
+      !make_map(&tm_kc, c.k, cache_rows, s.n_kv_heads, 1, PG) ||
+      !make_map(&tm_vc, c.v, cache_rows, s.n_kv_heads, 1, PG) ||
+      !make_map(&tm_kt, k_tree, tree_rows, s.n_kv_heads, 1, PG) ||
+      !make_map(&tm_vt, v_tree, tree_rows, s.n_kv_heads, 1, PG))
     return cudaErrorInvalidValue;
 
   Params p;
