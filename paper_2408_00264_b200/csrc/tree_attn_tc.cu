@@ -4,13 +4,12 @@
 // One thread block owns up to 256 query rows of one (sequence, kv head) - a row is a
 // (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes reuse every
 // K/V byte - and a contiguous range of key tiles (cache tiles first, then the tree's own keys).
-// The tensor core fetches K-major shared-memory operands at about half the shared-memory rate
-// (measured: an MMA with both operands in shared memory costs (rows of A + rows of B) / 2 cycles
-// per 16-wide k-step), so the operands that are reused across all key tiles live in tensor memory:
-// each softmax thread copies its Q row (bf16 pairs) into TMEM once, and P is written there every
-// tile.  Q K^T then fetches only K (64 rows: 32 cycles = its math time) and P V only V.  Key tiles
-// are 64 keys (= the page size of a paged cache); K and V travel through separate rings so that a
-// K buffer is refilled as soon as its Q K^T is done.
+// Key tiles are 64 keys (= the page size of a paged cache); K and V travel through separate rings
+// so that a K buffer is refilled as soon as its Q K^T is done.
+// MMA issue order: consecutive tcgen05.mma instructions that accumulate into the same TMEM tile
+// are dependent and cost about 100 cycles each whatever their size (measured), far above the
+// 32-64 cycles of arithmetic of these small shapes.  The issuer therefore interleaves independent
+// accumulation chains: the P V of tile r (into O) with the Q K^T of tile r+1 (into S).
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation), warps 2-5 and
 // 6-9 = two softmax groups of 128 threads, one thread per query row ("slot" 0 and 1).
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
@@ -43,6 +42,7 @@ constexpr int PG = CLV_PAGE_SIZE;      // 64: keys per TMA piece (= page size)
 constexpr int HD = CLV_HEAD_DIM;       // 128
 constexpr int BM = 128;                // rows per MMA / per slot
 constexpr int kThreads = 320;
+constexpr uint32_t kQTile = BM * HD * 2;       // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleGap = 8.0f;           // log2 units: P stays below 2^8
@@ -51,13 +51,12 @@ constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: abo
 template <int MT>
 struct Cfg {
   static constexpr int BN = 64;                          // keys per tile
-  static constexpr int kStages = 6;                      // ring depth, K and V each
+  static constexpr int kStages = (MT == 2) ? 4 : 5;      // ring depth, K and V each
   static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
-  static constexpr uint32_t kSmem = kStages * 2 * kTile + 1024;
+  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kTile + 1024;
 };
 
 struct Params {
-  const uint16_t* q;
   const int32_t* block_table;
   const int32_t* parent;
   const int32_t* ctx_len;
@@ -144,8 +143,17 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem], bf16 inputs, fp32 accumulate; issued by one thread.  The A operand
-// is read from tensor memory (lane = row, two bf16 per 32-bit column).
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Same with the A operand read from tensor memory (lane = row, two bf16 per 32-bit column).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate) {
   asm volatile(
@@ -187,8 +195,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // ------------------------------------------------------------------------------------ kernel
 template <int MT>
 __global__ void __launch_bounds__(kThreads, 1)
-tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_constant__ CUtensorMap tm_vc,
-                    const __grid_constant__ CUtensorMap tm_kt,
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
+                    const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
                     const __grid_constant__ CUtensorMap tm_vt, const Params p) {
   constexpr int BN = Cfg<MT>::BN;          // keys per tile
   constexpr int PPT = BN / PG;             // 64-key pieces per tile
@@ -262,7 +270,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
 
   // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sK = smem_base;             // ring of NST K tiles
+  const uint32_t sQ = smem_base;
+  const uint32_t sK = sQ + MT * kQTile;      // ring of NST K tiles
   const uint32_t sV = sK + NST * kTile;      // ring of NST V tiles
   uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
 
@@ -279,7 +288,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
 
   if (tid == 0) {
     for (int i = 0; i < 4 * NST; ++i) mbar_init(bar0 + 8u * i, 1);
-    mbar_init(bar_q, 2 * BM);  // every softmax thread has put its Q row into tensor memory
+    mbar_init(bar_q, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_s_full(s), 1);
       mbar_init(bar_p_full(s), BM);
@@ -296,12 +305,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abort_flag = &s_abort;
-  // columns: S of slot s at 64 s (P, two bf16 per column, overwrites its first 32 columns once
-  // the scores have been read); Q of slot s (two bf16 per column) at 128 + 64 s; O at 256 + 128 s
+  // columns: S of slot s at 64 s; P (two bf16 per column) at 128 + 32 s; O at 192 + 128 s.
+  // P has columns of its own because Q K^T of the next tile runs interleaved with P V of this one.
   auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_P = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_Q = [&](int s) { return tmem + (uint32_t)(2 * BN + s * (HD / 2)); };
-  auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + HD + s * HD); };
+  auto tmem_P = [&](int s) { return tmem + (uint32_t)(2 * BN + s * (BN / 2)); };
+  auto tmem_O = [&](int s) { return tmem + (uint32_t)(3 * BN + s * HD); };
 
   int issued_tiles = 0;  // producer bookkeeping for the drain
 
@@ -321,10 +329,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
   if (warp == 0) {
     // =========================== TMA producer ===============================================
     if (lane == 0) {
-      tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
       tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
     }
     if (n_tiles > 0) {
+      if (lane == 0) {
+        mbar_expect_tx(bar_q, MT * kQTile);
+        const int nodes_per_tile = BM / G;
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          const int node0 = b * N + (row_cta * MT + m) * nodes_per_tile;
+          tma_load_3d(sQ + m * kQTile, &tm_q, 0, kvh * G, node0, bar_q);
+          tma_load_3d(sQ + m * kQTile + kQTile / 2, &tm_q, 64, kvh * G, node0, bar_q);
+        }
+      }
       constexpr int kBatch = 32 / PPT;  // tiles whose page numbers one warp-wide fetch covers
       int page_cache = 0;               // lane j: pool page of piece (batch base * PPT + j)
       bool ok = true;
@@ -392,43 +410,58 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
       auto local_tile = [&](int s, int r) { return (MT == 2) ? r : 2 * r + s; };
       // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
       // constant (the address field counts 16-byte units and never carries out of its 14 bits).
+      const uint64_t q_desc = smem_desc(sQ, 16, 1024);
       const uint64_t k_desc = smem_desc(sK, 16, 1024);
       const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
-      auto issue_qk = [&](int s, int r) -> bool {
-        const int i = local_tile(s, r), st = i % NST;
-        if (!mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag)) return false;
+      auto qk_step = [&](int s, uint64_t kd, int ks) {  // one 16-wide slice of the head dimension
+        const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
+        const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
+        const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
+        umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
+      };
+      const int rounds[2] = {rounds0, rounds1};
+      // first tile of each slot: nothing to interleave with yet
+      for (int s = 0; s < 2 && ok; ++s) {
+        if (rounds[s] == 0) continue;
+        const int i = local_tile(s, 0), st = i % NST;
+        ok = mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag);
+        if (!ok) break;
         tc_fence_after();
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ++ks) {
-          const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
-          umma_bf16_ts(tmem_S(s), tmem_Q(s) + ks * 8, kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
-        }
+        for (int ks = 0; ks < HD / 16; ++ks) qk_step(s, kd, ks);
         umma_commit(bar_s_full(s));
-        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
-        return true;
-      };
-      const int rounds[2] = {rounds0, rounds1};
-      for (int s = 0; s < 2 && ok; ++s)
-        if (rounds[s] > 0) ok = issue_qk(s, 0);
+        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));
+      }
       for (int r = 0; r < rounds0 && ok; ++r) {
         for (int s = 0; s < 2 && ok; ++s) {
           if (r >= rounds[s]) continue;
-          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
-          if (!ok) break;
+          const bool has_next = r + 1 < rounds[s];
           const int i = local_tile(s, r), st = i % NST;
-          ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+          const int i2 = local_tile(s, r + 1), st2 = i2 % NST;
+          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
+          if (ok) ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+          if (ok && has_next) ok = mbar_wait(bar_k_full(st2), (i2 / NST) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
+          const uint64_t kd = k_desc + (uint64_t)((st2 * kTile) >> 4);
+          // two independent accumulation chains, alternated: S(r+1) += Q K^T slices, O += P V slices
 #pragma unroll
-          for (int kk = 0; kk < BN / 16; ++kk) {
-            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
-                         (r > 0 || kk > 0) ? 1u : 0u);
+          for (int j = 0; j < HD / 16; ++j) {
+            if (has_next) qk_step(s, kd, j);
+            if (j < BN / 16)
+              umma_bf16_ts(tmem_O(s), tmem_P(s) + j * 8, vd + (uint64_t)((j * 2048) >> 4), kIdescPV,
+                           (r > 0 || j > 0) ? 1u : 0u);
+            if (j == BN / 16 - 1) {  // all of P V is queued: its completion frees P, V and O
+              umma_commit(bar_pv_done(s));
+              if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));
+            }
           }
-          umma_commit(bar_pv_done(s));
-          if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
-          if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
+          if (has_next) {
+            umma_commit(bar_s_full(s));
+            if (MT == 1 || s == 1) umma_commit(bar_k_empty(st2));
+          }
         }
       }
     }
@@ -437,24 +470,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
     constexpr int NH = BN / 64;   // the row of S is taken in 64-column halves (register budget)
     const int rounds = my_rounds;
     bool ok = true;
-    {
-      // this thread's query row, as stored (two bf16 per word), becomes the A operand of Q K^T
-      const uint4* qsrc = reinterpret_cast<const uint4*>(
-          p.q + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD);
-#pragma unroll
-      for (int c = 0; c < HD / 2; c += 32) {
-        uint32_t qv[32];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint4 v = row_valid ? __ldg(qsrc + (c >> 2) + j) : make_uint4(0, 0, 0, 0);
-          qv[4 * j] = v.x; qv[4 * j + 1] = v.y; qv[4 * j + 2] = v.z; qv[4 * j + 3] = v.w;
-        }
-        tmem_st_x32(tmem_Q(slot) + lane_addr + c, qv);
-      }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_q);
-    }
 
     for (int r = 0; r < rounds && ok; ++r) {
       const int i = (MT == 2) ? r : 2 * r + slot;
@@ -598,6 +613,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
         mbar_drain(bar_k_full(i % NST), (i / NST) & 1);
         mbar_drain(bar_v_full(i % NST), (i / NST) & 1);
       }
+      if (n_tiles > 0) mbar_drain(bar_q, 0);
     }
     if (warp == 1 && lane == 0) {
       umma_commit(bar_drain);  // completes when every MMA issued so far has finished
@@ -613,7 +629,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_kc, const __grid_cons
   // staging area for the merge: O of both slots as fp32 [slot][128 rows][128], 16-byte chunk c of
   // row r stored at chunk (c ^ (r & 31)) so that row-per-thread writes and row-per-warp reads are
   // both conflict free.  It reuses the tile memory, which nothing reads any more.
-  float* const sO = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
+  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));
 
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
@@ -784,6 +800,8 @@ bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t heads, 
 }  // namespace
 
 bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
+  const int G = s.n_q_heads / s.n_kv_heads;
+  if (G > BM || (BM % G) != 0) return false;           // a row tile must hold whole nodes
   const int64_t cache_rows = c.paged ? (int64_t)c.n_pages * CLV_PAGE_SIZE : (int64_t)s.batch * c.cap_tokens;
   if (cache_rows >= (1ll << 31) || (int64_t)s.batch * s.n_nodes >= (1ll << 31)) return false;
   return encode_fn() != nullptr;
@@ -830,17 +848,17 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  alignas(64) CUtensorMap tm_kc, tm_vc, tm_kt, tm_vt;
+  alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt;
   const uint64_t cache_rows = c.paged ? (uint64_t)c.n_pages * CLV_PAGE_SIZE : (uint64_t)s.batch * c.cap_tokens;
   const uint64_t tree_rows = (uint64_t)s.batch * s.n_nodes;
-  if (!make_map(&tm_kc, c.k, cache_rows, s.n_kv_heads, 1, PG) ||
+  if (!make_map(&tm_q, q, tree_rows, s.n_q_heads, G, BM / G) ||
+      !make_map(&tm_kc, c.k, cache_rows, s.n_kv_heads, 1, PG) ||
       !make_map(&tm_vc, c.v, cache_rows, s.n_kv_heads, 1, PG) ||
       !make_map(&tm_kt, k_tree, tree_rows, s.n_kv_heads, 1, PG) ||
       !make_map(&tm_vt, v_tree, tree_rows, s.n_kv_heads, 1, PG))
     return cudaErrorInvalidValue;
 
   Params p;
-  p.q = static_cast<const uint16_t*>(q);
   p.block_table = c.block_table;
   p.parent = parent;
   p.ctx_len = ctx_len;
@@ -866,8 +884,8 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (mt == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_kc, tm_vc, tm_kt, tm_vt, p);
-  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<2>, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  if (mt == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<2>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
 }
 
 }  // namespace clv
