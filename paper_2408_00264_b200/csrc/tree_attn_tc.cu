@@ -4,12 +4,10 @@
 // One thread block owns up to 256 query rows of one (sequence, kv head) - a row is a
 // (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes reuse every
 // K/V byte - and a contiguous range of key tiles (cache tiles first, then the tree's own keys).
-// Key tiles are 64 keys (= the page size of a paged cache); K and V travel through separate rings
-// so that a K buffer is refilled as soon as its Q K^T is done.
-// MMA issue order: consecutive tcgen05.mma instructions that accumulate into the same TMEM tile
-// are dependent and cost about 100 cycles each whatever their size (measured), far above the
-// 32-64 cycles of arithmetic of these small shapes.  The issuer therefore interleaves independent
-// accumulation chains: the P V of tile r (into O) with the Q K^T of tile r+1 (into S).
+// A key tile is 128 keys when the block has two row tiles (an MMA costs about the same for 64 as
+// for 128 columns, so wide S tiles halve the tensor time) and 64 keys otherwise; tiles are loaded
+// as 64-key pieces, which is also the page size of a paged cache.  K and V travel through separate
+// rings so that a K buffer is refilled as soon as its Q K^T is done.
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation), warps 2-5 and
 // 6-9 = two softmax groups of 128 threads, one thread per query row ("slot" 0 and 1).
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
@@ -42,7 +40,7 @@ constexpr int PG = CLV_PAGE_SIZE;      // 64: keys per TMA piece (= page size)
 constexpr int HD = CLV_HEAD_DIM;       // 128
 constexpr int BM = 128;                // rows per MMA / per slot
 constexpr int kThreads = 320;
-constexpr uint32_t kQTile = BM * HD * 2;       // 32 KB: two [128 rows][64 d] swizzled halves
+constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleGap = 8.0f;           // log2 units: P stays below 2^8
@@ -50,8 +48,8 @@ constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: abo
 
 template <int MT>
 struct Cfg {
-  static constexpr int BN = 64;                          // keys per tile
-  static constexpr int kStages = (MT == 2) ? 4 : 5;      // ring depth, K and V each
+  static constexpr int BN = (MT == 2) ? 128 : 64;        // keys per tile
+  static constexpr int kStages = (MT == 2) ? 2 : 5;      // ring depth, K and V each
   static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
   static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kTile + 1024;
 };
@@ -182,6 +180,27 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 }
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
 
+// Distributed shared memory: address of the same variable in block `rank` of the cluster, and a
+// 16-byte load from it.  The loads are volatile asm so that a batch of them is issued back to back
+// (all in flight together) before the first result is used.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 dsmem_ld8(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -190,6 +209,48 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Final combination of NSRC accumulators per output row, for the rows [k_begin, k_end) that this
+// block finalises.  One warp takes 16 / NSRC rows at a time (16 remote 16-byte loads in flight
+// per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the normalised weights.
+template <int NSRC, int MT>
+__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
+                                           int warp, int lane, int tile_base, int rows_total, int G,
+                                           int64_t seq_row0, int Hq, int head0, uint16_t* out) {
+  constexpr int RB = 16 / NSRC;
+  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
+    float4 x[RB * NSRC];
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      const int k = min(k0 + u, per_rank - 1);
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const uint32_t off = (uint32_t)(trow * HD + ((lane ^ (trow & 31)) << 2)) * 4u;
+#pragma unroll
+      for (int q = 0; q < NSRC; ++q) {
+        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+        x[u * NSRC + q] = dsmem_ld16(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 4) + off, qc));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      if (k0 + u >= per_rank) continue;
+      const int k = k0 + u;
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const int rg = (tile_base + tile) * BM + trow;
+      if (rg >= rows_total) continue;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int q = 0; q < NSRC; ++q) {
+        const float wq = w[k * NSRC + q];
+        const float4 v = x[u * NSRC + q];
+        acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
+      }
+      const int onode = rg / G, ogq = rg - onode * G;
+      uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------ kernel
@@ -211,7 +272,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
-  __shared__ float2 s_src[2 * BM]; // merge: (weight, sum) of every (row of this rank, source)
+  __shared__ float s_w[2 * BM];    // merge: normalised weight of every (row of this rank, source)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.x / p.row_ctas, row_cta = blockIdx.x - unit * p.row_ctas;
@@ -305,11 +366,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abort_flag = &s_abort;
-  // columns: S of slot s at 64 s; P (two bf16 per column) at 128 + 32 s; O at 192 + 128 s.
-  // P has columns of its own because Q K^T of the next tile runs interleaved with P V of this one.
+  // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
+  // the scores have been read); O of slot s at 2 BN + 128 s
   auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_P = [&](int s) { return tmem + (uint32_t)(2 * BN + s * (BN / 2)); };
-  auto tmem_O = [&](int s) { return tmem + (uint32_t)(3 * BN + s * HD); };
+  auto tmem_P = [&](int s) { return tmem + (uint32_t)(s * BN); };
+  auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + s * HD); };
 
   int issued_tiles = 0;  // producer bookkeeping for the drain
 
@@ -413,55 +474,43 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint64_t q_desc = smem_desc(sQ, 16, 1024);
       const uint64_t k_desc = smem_desc(sK, 16, 1024);
       const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
-      auto qk_step = [&](int s, uint64_t kd, int ks) {  // one 16-wide slice of the head dimension
-        const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
-        const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
-        const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
-        umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
-      };
-      const int rounds[2] = {rounds0, rounds1};
-      // first tile of each slot: nothing to interleave with yet
-      for (int s = 0; s < 2 && ok; ++s) {
-        if (rounds[s] == 0) continue;
-        const int i = local_tile(s, 0), st = i % NST;
-        ok = mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag);
-        if (!ok) break;
+      auto issue_qk = [&](int s, int r) -> bool {
+        const int i = local_tile(s, r), st = i % NST;
+        if (!mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag)) return false;
         tc_fence_after();
+        const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ++ks) qk_step(s, kd, ks);
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
+          const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
+          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
+        }
         umma_commit(bar_s_full(s));
-        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));
-      }
+        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
+        return true;
+      };
+      const int rounds[2] = {rounds0, rounds1};
+      for (int s = 0; s < 2 && ok; ++s)
+        if (rounds[s] > 0) ok = issue_qk(s, 0);
       for (int r = 0; r < rounds0 && ok; ++r) {
         for (int s = 0; s < 2 && ok; ++s) {
           if (r >= rounds[s]) continue;
-          const bool has_next = r + 1 < rounds[s];
-          const int i = local_tile(s, r), st = i % NST;
-          const int i2 = local_tile(s, r + 1), st2 = i2 % NST;
           ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
-          if (ok) ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
-          if (ok && has_next) ok = mbar_wait(bar_k_full(st2), (i2 / NST) & 1, abort_flag);
+          if (!ok) break;
+          const int i = local_tile(s, r), st = i % NST;
+          ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
-          const uint64_t kd = k_desc + (uint64_t)((st2 * kTile) >> 4);
-          // two independent accumulation chains, alternated: S(r+1) += Q K^T slices, O += P V slices
 #pragma unroll
-          for (int j = 0; j < HD / 16; ++j) {
-            if (has_next) qk_step(s, kd, j);
-            if (j < BN / 16)
-              umma_bf16_ts(tmem_O(s), tmem_P(s) + j * 8, vd + (uint64_t)((j * 2048) >> 4), kIdescPV,
-                           (r > 0 || j > 0) ? 1u : 0u);
-            if (j == BN / 16 - 1) {  // all of P V is queued: its completion frees P, V and O
-              umma_commit(bar_pv_done(s));
-              if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));
-            }
+          for (int kk = 0; kk < BN / 16; ++kk) {
+            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                         (r > 0 || kk > 0) ? 1u : 0u);
           }
-          if (has_next) {
-            umma_commit(bar_s_full(s));
-            if (MT == 1 || s == 1) umma_commit(bar_k_empty(st2));
-          }
+          umma_commit(bar_pv_done(s));
+          if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
+          if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
         }
       }
     }
@@ -690,73 +739,38 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (!aborted) {
     // Every rank finalises per_rank rows; per_rank * n_src is 256 whatever the split count.
     const int per_rank = MT * BM / p.splits;
-    // (a) fetch the (maximum, sum) pair of every (row, source); source q is (block q, slot `tile`)
-    //     when MT == 2 and (block q / 2, slot q % 2) when MT == 1
-    if (tid < per_rank * n_src) {
+    const int first_row = split * per_rank;
+    // (a) thread (k, q) fetches the (maximum, sum) pair of source q of row k; the n_src lanes of a
+    //     row sit side by side in one warp, so the normalised weights come from shuffles.
+    //     Source q is (block q, slot `tile`) when MT == 2 and (block q / 2, slot q % 2) when MT == 1.
+    if (tid < 2 * BM) {
       const int k = tid / n_src, q = tid - k * n_src;
-      const int rr = split * per_rank + k, tile = rr / BM, trow = rr % BM;
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
       const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-      s_src[tid] = cluster.map_shared_rank(&s_ml[0][0], qc)[qs * BM + trow];
-    }
-    __syncthreads();
-    // (b) one thread per row: normalised weights, log-sum-exp
-    if (tid < per_rank) {
-      const int rr = split * per_rank + tid, tile = rr / BM, trow = rr % BM;
-      float mmax = -INFINITY;
-      for (int q = 0; q < n_src; ++q) mmax = fmaxf(mmax, s_src[tid * n_src + q].x);
+      const float2 ml = dsmem_ld8(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
+      float mmax = ml.x;
+      for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
-      float lsum = 0.f;
-      for (int q = 0; q < n_src; ++q) {
-        const float2 v = s_src[tid * n_src + q];
-        const float w = (v.y > 0.f) ? ex2(v.x - mu) : 0.f;
-        s_src[tid * n_src + q].x = w;
-        lsum += w * v.y;
-      }
-      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-      for (int q = 0; q < n_src; ++q) s_src[tid * n_src + q].x *= inv;
+      const float wgt = (ml.y > 0.f) ? ex2(ml.x - mu) : 0.f;
+      float lsum = wgt * ml.y;
+      for (int o = 1; o < n_src; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+      s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f);
       const int rg = (row_cta * MT + tile) * BM + trow;
-      if (p.lse != nullptr && rg < rows_total) {
+      if (q == 0 && p.lse != nullptr && rg < rows_total) {
         const int onode = rg / G, ogq = rg - onode * G;
         p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
       }
     }
     __syncthreads();
-    // (c) one warp per pair of rows, lane j owns columns 4j..4j+3; all loads of a pair in flight
-    for (int k0 = warp * 2; k0 < per_rank; k0 += 2 * (kThreads / 32)) {
-      float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
-      int rg[2];
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int k = min(k0 + u, per_rank - 1);
-        const int rr = split * per_rank + k, tile = rr / BM, trow = rr % BM;
-        rg[u] = (k0 + u < per_rank) ? (row_cta * MT + tile) * BM + trow : rows_total;
-        const int chunk_off = (lane ^ (trow & 31)) << 2;
-        for (int q0 = 0; q0 < n_src; q0 += 4) {  // n_src is 2, 4, 8 or 16
-          float4 x[4];
-          float wq[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int q = min(q0 + j, n_src - 1);
-            const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-            x[j] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sO, qc) +
-                                                    ((size_t)qs * BM + trow) * HD + chunk_off);
-            wq[j] = (q0 + j < n_src) ? s_src[k * n_src + q].x : 0.f;
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            acc[u].x += wq[j] * x[j].x; acc[u].y += wq[j] * x[j].y;
-            acc[u].z += wq[j] * x[j].z; acc[u].w += wq[j] * x[j].w;
-          }
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        if (rg[u] >= rows_total) continue;
-        const int onode = rg[u] / G, ogq = rg[u] - onode * G;
-        uint16_t* dst = p.out + (((int64_t)b * N + onode) * p.Hq + kvh * G + ogq) * HD + lane * 4;
-        *reinterpret_cast<uint2*>(dst) =
-            make_uint2(pack_bf16(acc[u].x, acc[u].y), pack_bf16(acc[u].z, acc[u].w));
-      }
+    // (b) weighted sums, rows spread over the warps
+    const uint32_t sO_addr = smem_u32(sO);
+    uint16_t* outp = p.out;
+    const int64_t seq_row0 = (int64_t)b * N;
+    switch (n_src) {
+      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
