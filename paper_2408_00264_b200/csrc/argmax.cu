@@ -6,6 +6,7 @@
 // "higher value first, then lower index", and the last block to arrive for a row takes the
 // maximum key.  The result is independent of the chunking and of block scheduling.
 #include <limits.h>
+#include <stdlib.h>
 
 #include "clv_internal.cuh"
 
@@ -26,32 +27,33 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
 __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) {
   return *reinterpret_cast<__nv_bfloat162*>(&u);
 }
-__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
-__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
-// Running (best value, lowest index of it) of one thread; indices are visited in ascending order.
+// Per-thread state: for each of the 8 positions inside a 16-byte vector, the running maximum (bf16)
+// and the number of the visit at which it was first reached, both packed two per register.
+// Updating is branch free (compare mask, max, bit select): a data-dependent branch would be taken
+// by some lane of the warp at almost every step, because a thread only sees a few dozen vectors.
+struct Track {
+  __nv_bfloat162 m[4];
+  uint32_t at[4];  // two 16-bit visit numbers; 0xFFFF = nothing above -inf seen yet
+};
+__device__ __forceinline__ void track_init(Track& t) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { t.m[j] = as_bf162(0xFF80FF80u); t.at[j] = 0xFFFFFFFFu; }
+}
+__device__ __forceinline__ void take_vec(Track& t, const uint4& w, uint32_t visit2) {
+  const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const __nv_bfloat162 x = as_bf162(u[j]);
+    const uint32_t gt = __hgt2_mask(x, t.m[j]);  // strictly greater (false for NaN): first hit stays
+    t.m[j] = __hmax2(t.m[j], x);                 // NaN operands are dropped
+    t.at[j] = (t.at[j] & ~gt) | (visit2 & gt);
+  }
+}
 struct Best {
   float v;
   int i;
 };
-
-__device__ __forceinline__ void take_vec(Best& b, const uint4& w, int idx0) {
-  // maximum of the 8 values (NaN operands are dropped by max.bf16x2)
-  __nv_bfloat162 m = __hmax2(__hmax2(as_bf162(w.x), as_bf162(w.y)),
-                             __hmax2(as_bf162(w.z), as_bf162(w.w)));
-  float vm = fmaxf(__low2float(m), __high2float(m));
-  if (vm > b.v) {  // rare after the first few vectors
-    b.v = vm;
-    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
-    int at = 7;
-#pragma unroll
-    for (int e = 3; e >= 0; --e) {  // descending, so the lowest matching position survives
-      if (bf16hi(u[e]) == vm) at = 2 * e + 1;
-      if (bf16lo(u[e]) == vm) at = 2 * e;
-    }
-    b.i = idx0 + at;
-  }
-}
 
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) {
   return (v > bv) || (v == bv && i < bi);
@@ -85,16 +87,31 @@ __global__ void __launch_bounds__(kThreads) argmax_kernel(Params p) {
   const uint4* vp = reinterpret_cast<const uint4*>(base + begin);
   const int tid = threadIdx.x;
 
-  Best best = {-INFINITY, INT_MAX};
+  Track trk;
+  track_init(trk);
   int i = tid;
+  uint32_t visit2 = 0;  // visit number in both halves
   for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
     uint4 w[kUnroll];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) w[u] = ld_stream16(vp + i + u * kThreads);
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) take_vec(best, w[u], begin + 8 * (i + u * kThreads));
+    for (int u = 0; u < kUnroll; ++u) { take_vec(trk, w[u], visit2); visit2 += 0x00010001u; }
   }
-  for (; i < nvec; i += kThreads) take_vec(best, ld_stream16(vp + i), begin + 8 * i);
+  for (; i < nvec; i += kThreads) { take_vec(trk, ld_stream16(vp + i), visit2); visit2 += 0x00010001u; }
+  // the thread's best of its 8 positions: visit k of this thread is vector tid + k * kThreads
+  Best best = {-INFINITY, INT_MAX};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+#pragma unroll
+    for (int hlf = 0; hlf < 2; ++hlf) {
+      const uint32_t k = hlf ? (trk.at[j] >> 16) : (trk.at[j] & 0xFFFFu);
+      if (k == 0xFFFFu) continue;
+      const float v = hlf ? __high2float(trk.m[j]) : __low2float(trk.m[j]);
+      const int idx = begin + 8 * (tid + (int)k * kThreads) + 2 * j + hlf;
+      if ((v > best.v) || (v == best.v && idx < best.i)) { best.v = v; best.i = idx; }
+    }
+  }
   // ragged end of the row (vocab not a multiple of 8): at most 7 scalars, after all vectors
   {
     const int t0 = begin + 8 * nvec + tid;
@@ -141,17 +158,16 @@ __global__ void __launch_bounds__(kThreads) argmax_kernel(Params p) {
 ArgmaxPlan argmax_plan(int rows, int vocab) {
   ArgmaxPlan pl;
   pl.rows = rows;
-  // One wave of long-lived blocks: about four resident blocks per SM, each streaming a contiguous
-  // piece of one row (short blocks spend their time being launched and retired, and a grid of
-  // 1.7 waves leaves the machine half empty at the end).
+  // 16384 logits (32 KB) per block = one batch of kUnroll loads per thread, all in flight at
+  // once; fewer, smaller pieces only when there are too few rows to cover the machine.
   const int unit = kThreads * 8;  // elements one pass of the block covers
-  const int64_t want_blocks = 4LL * sm_count();
-  int64_t chunks = (want_blocks + rows - 1) / rows;
-  if (chunks < 1) chunks = 1;
-  int64_t chunk_elems = (vocab + chunks - 1) / chunks;
-  chunk_elems = (chunk_elems + unit - 1) / unit * unit;
-  pl.chunk_elems = (int)chunk_elems;
-  pl.chunks = (int)((vocab + chunk_elems - 1) / chunk_elems);
+  int chunk_elems = kUnroll * unit;
+  const int want_blocks = 4 * sm_count();
+  while (chunk_elems > unit && (int64_t)rows * ((vocab + chunk_elems - 1) / chunk_elems) < want_blocks)
+    chunk_elems >>= 1;
+  if (const char* e = getenv("CLV_ARGMAX_CHUNK")) chunk_elems = atoi(e) / unit * unit > 0 ? atoi(e) / unit * unit : chunk_elems;
+  pl.chunk_elems = chunk_elems;
+  pl.chunks = (vocab + chunk_elems - 1) / chunk_elems;
   pl.scratch_bytes = pl.chunks > 1 ? sizeof(unsigned long long) * (size_t)rows * pl.chunks : 0;
   return pl;
 }
