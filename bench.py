@@ -231,16 +231,31 @@ def run_clv(args):
 
     # ---- each call alone, back to back over the rotating sets (same stream) -----------------
     def time_call(name, n):
+        """Microseconds per launch of one call, back to back over the rotating input sets.  The
+        launches are replayed from a CUDA graph (one launch per input set) so that host launch
+        overhead does not set the pace of the short kernels."""
         for i in range(3):
             getattr(sets[i % ROTATE], name)()
+        torch.cuda.synchronize()
+        if args.no_graph:
+            run, per = (lambda: [getattr(sets[i], name)() for i in range(ROTATE)]), ROTATE
+        else:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(ROTATE):
+                    getattr(sets[i], name)()
+            run, per = g.replay, ROTATE
+        run()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        cur = torch.cuda.current_stream()
         torch.cuda.synchronize()
-        a.record(stream)
-        for i in range(n):
-            getattr(sets[i % ROTATE], name)()
-        b.record(stream)
+        a.record(cur)
+        reps = max(1, n // per)
+        for _ in range(reps):
+            run()
+        b.record(cur)
         torch.cuda.synchronize()
-        return a.elapsed_time(b) / n * 1e3          # microseconds per launch
+        return a.elapsed_time(b) / (reps * per) * 1e3
     n_k = max(20, min(args.steps, 400))
     call_us = {k: time_call(k, n_k) for k in ("tree_attn", "accept_argmax", "accept_walk", "kv_commit")}
 
