@@ -6,7 +6,6 @@
 // "higher value first, then lower index", and the last block to arrive for a row takes the
 // maximum key.  The result is independent of the chunking and of block scheduling.
 #include <limits.h>
-#include <stdlib.h>
 
 #include "clv_internal.cuh"
 
@@ -158,14 +157,14 @@ __global__ void __launch_bounds__(kThreads) argmax_kernel(Params p) {
 ArgmaxPlan argmax_plan(int rows, int vocab) {
   ArgmaxPlan pl;
   pl.rows = rows;
-  // 16384 logits (32 KB) per block = one batch of kUnroll loads per thread, all in flight at
-  // once; fewer, smaller pieces only when there are too few rows to cover the machine.
+  // 32768 logits (64 KB) per block = two batches of kUnroll loads per thread (measured best on
+  // 128256-wide rows: 1024 blocks = one wave of 7 blocks per SM); fewer, smaller pieces only when
+  // there are too few rows to cover the machine.
   const int unit = kThreads * 8;  // elements one pass of the block covers
-  int chunk_elems = kUnroll * unit;
+  int chunk_elems = 2 * kUnroll * unit;
   const int want_blocks = 4 * sm_count();
   while (chunk_elems > unit && (int64_t)rows * ((vocab + chunk_elems - 1) / chunk_elems) < want_blocks)
     chunk_elems >>= 1;
-  if (const char* e = getenv("CLV_ARGMAX_CHUNK")) chunk_elems = atoi(e) / unit * unit > 0 ? atoi(e) / unit * unit : chunk_elems;
   pl.chunk_elems = chunk_elems;
   pl.chunks = (vocab + chunk_elems - 1) / chunk_elems;
   pl.scratch_bytes = pl.chunks > 1 ? sizeof(unsigned long long) * (size_t)rows * pl.chunks : 0;
