@@ -31,6 +31,9 @@ METRIC = "verify-step achieved HBM GB/s (algorithmic bytes / step time)"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 ROTATE = 4   # distinct input sets cycled between steps: 4 x 138 MB > 2 x L2 (126 MB)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/verify_step_C3.md; valid for the kernels as they were when that capture was taken
+NCU_TRAFFIC = {("C3", "tree_attn"): 72.6e6, ("C3", "accept_argmax"): 65.9e6}
 
 
 def measured_peaks():
@@ -167,6 +170,19 @@ def workload_config(w):
                             % ROTATE}
 
 
+def reduce_over_ranks(dist, device, step_ms, e2e_ms, local_bytes):
+    """Whole-job figures from per-rank ones: the slowest rank sets the time (max), the bytes of all
+    ranks add up (every rank runs its own batch; there is no other exchange)."""
+    if dist is None:
+        return step_ms, e2e_ms, local_bytes
+    import torch
+    t = torch.tensor([step_ms, e2e_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    tot = torch.tensor([local_bytes], device=device, dtype=torch.float64)
+    dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(tot[0])
+
+
 # ----------------------------------------------------------------------------- device arm
 def run_clv(args):
     import torch
@@ -298,15 +314,7 @@ def run_clv(args):
         e2e_ms = e0.elapsed_time(e1) / n_e2e
 
     # ---- max over ranks ------------------------------------------------------------------------
-    if dist is not None:
-        t = torch.tensor([step_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms, e2e_ms = float(t[0]), float(t[1])
-        tot = torch.tensor([float(nbytes["total"])], device=dev, dtype=torch.float64)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-        job_bytes = float(tot[0])
-    else:
-        job_bytes = float(nbytes["total"])
+    step_ms, e2e_ms, job_bytes = reduce_over_ranks(dist, dev, step_ms, e2e_ms, float(nbytes["total"]))
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -330,7 +338,7 @@ def run_clv(args):
         "algorithmic_bytes": nbytes,
         "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak,
                      "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None},
+                     "traffic": NCU_TRAFFIC.get((args.workload, dom))},
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
