@@ -576,24 +576,35 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
       };
-      float mx = -INFINITY;
+      // One pass with the reference maximum as it stands: exponentiate, pack P (kept in registers)
+      // and track the true row maximum on the way.  The reference is only replaced when the
+      // maximum has outgrown it by more than the gap - rare after the first tile - and then the
+      // tile is redone from the scores, which are still intact because P is stored last.
+      uint32_t pk[NH * 32];
+      float mx = -INFINITY, sum = 0.f;
+      float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
 #pragma unroll
       for (int h = 0; h < NH; ++h) {
         load_half(h);
 #pragma unroll
-        for (int j = 0; j < 64; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
+        for (int j = 0; j < 32; ++j) {
+          const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
+          mx = fmaxf(mx, fmaxf(a0, a1));
+          const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(a1, p.scale_log2, neg_m));
+          sum += p0 + p1;
+          pk[h * 32 + j] = pack_bf16(p0, p1);
+        }
       }
       mx *= p.scale_log2;  // scale > 0; -inf stays -inf
       const bool need = mx > m_ref + kRescaleGap;  // also true for the first finite maximum
-      const bool any_need = __any_sync(0xFFFFFFFFu, need);
-
-      if (r > 0) {  // the previous P V has read P and is no longer writing O
-        ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        tc_fence_after();
-      }
-      if (any_need) {
+      if (__any_sync(0xFFFFFFFFu, need)) {
+        if (r > 0) {  // O must be at rest: the previous P V has completed
+          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+        }
         const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
         if (need) { m_ref = mx; l_run *= alpha; }
         if (r > 0) {
@@ -608,23 +619,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
           tmem_wait_st();
         }
-      }
-      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      float sum = 0.f;
+        neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+        sum = 0.f;
 #pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        if (NH > 1) load_half(h);  // with one half the scores are still in registers
-        uint32_t pk[32];
+        for (int h = 0; h < NH; ++h) {
+          load_half(h);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-          sum += p0 + p1;
-          pk[j] = pack_bf16(p0, p1);
+          for (int j = 0; j < 32; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
+          }
         }
-        // P (the A operand of P V) takes the place of score columns that have been consumed
-        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, pk);
       }
+      // P (the A operand of P V) takes the place of score columns that have been consumed.  The
+      // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
       tmem_wait_st();
       l_run += sum;
 
