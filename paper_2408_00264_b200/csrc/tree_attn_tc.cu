@@ -465,11 +465,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   } else if (warp == 1) {
     // =========================== MMA issuer ===================================================
-    // The whole warp walks through the issue loops (so that descriptors and loop state can live in
-    // uniform registers); only the tcgen05 instructions themselves are issued by one lane.
-    const bool leader = lane == 0;
-    if (n_tiles > 0) {
-      bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_q, 0, abort_flag));
+    if (lane == 0 && n_tiles > 0) {
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
       tc_fence_after();
       auto local_tile = [&](int s, int r) { return (MT == 2) ? r : 2 * r + s; };
       // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
@@ -479,7 +476,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
       auto issue_qk = [&](int s, int r) -> bool {
         const int i = local_tile(s, r), st = i % NST;
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag))) return false;
+        if (!mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
@@ -487,13 +484,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int ks = 0; ks < HD / 16; ++ks) {
           const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
           const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
-          if (leader) umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
+          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
         }
-        if (leader) {
-          umma_commit(bar_s_full(s));
-          if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
-        }
-        __syncwarp();
+        umma_commit(bar_s_full(s));
+        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
         return true;
       };
       const int rounds[2] = {rounds0, rounds1};
@@ -502,23 +496,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int r = 0; r < rounds0 && ok; ++r) {
         for (int s = 0; s < 2 && ok; ++s) {
           if (r >= rounds[s]) continue;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_full(s), r & 1, abort_flag));
+          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
           if (!ok) break;
           const int i = local_tile(s, r), st = i % NST;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag));
+          ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
           for (int kk = 0; kk < BN / 16; ++kk) {
-            if (leader) umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                          (r > 0 || kk > 0) ? 1u : 0u);
           }
-          if (leader) {
-            umma_commit(bar_pv_done(s));
-            if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
-          }
-          __syncwarp();
+          umma_commit(bar_pv_done(s));
+          if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
           if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
         }
       }
