@@ -48,8 +48,8 @@ constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: abo
 
 template <int MT>
 struct Cfg {
-  static constexpr int BN = (MT == 2) ? 128 : 64;        // keys per tile
-  static constexpr int kStages = (MT == 2) ? 2 : 5;      // ring depth, K and V each
+  static constexpr int BN = 128;                         // keys per tile
+  static constexpr int kStages = (MT == 2) ? 2 : 3;      // ring depth, K and V each
   static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
   static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kTile + 1024;
 };
@@ -269,6 +269,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
   __shared__ __align__(8) unsigned long long s_bar[4 * NST + 8];
+  __shared__ int s_tile_ok[Cfg<MT>::kStages];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
@@ -415,6 +416,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           page_cache = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
         }
         int row0[PPT];   // first source row of each piece, -1: piece not present
+        int tile_ok = 1;
         const CUtensorMap *mk, *mv;
         if (t < t_cache) {
           mk = &tm_kc; mv = &tm_vc;
@@ -422,7 +424,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int j = 0; j < PPT; ++j) {
             const int pc = t * PPT + j;
             int pg = __shfl_sync(0xFFFFFFFFu, page_cache, (i % kBatch) * PPT + j);
-            if (pg < 0 || pg >= p.n_pages) pg = 0;  // flagged by the reporter; its keys get masked
+            if (pc < p_cache && (pg < 0 || pg >= p.n_pages)) tile_ok = 0;  // flagged by the reporter
+            if (pg < 0 || pg >= p.n_pages) pg = 0;  // the keys of such a tile get masked
             row0[j] = (pc >= p_cache) ? -1 : (p.paged ? pg * PG : b * p.cap_tokens + pc * PG);
           }
         } else {
@@ -450,6 +453,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (i >= NST) ok = mbar_wait(bar_v_empty(st), ((i / NST) - 1) & 1, abort_flag);
           }
           if (ok) {
+            s_tile_ok[st] = tile_ok;  // read by the softmax threads after this V barrier completes
             mbar_expect_tx(bar_v_full(st), bytes);
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
@@ -527,18 +531,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // allowed columns of this row in this tile, and how many V rows of the tile are real
       uint32_t allow[BN / 32];
       int v_rows;
+      bool cache_tile = false;
       if (t < t_cache) {
         v_rows = min(BN, L - t * BN);
-        if (p.paged) {
-#pragma unroll
-          for (int j = 0; j < PPT; ++j) {
-            const int pc = t * PPT + j;
-            if (pc < p_cache) {
-              const int pg = p.block_table[(int64_t)b * p.max_pages + pc];
-              if (pg < 0 || pg >= p.n_pages) v_rows = 0;  // sequence is flagged; hide the tile
-            }
-          }
-        }
+        cache_tile = true;
 #pragma unroll
         for (int w = 0; w < BN / 32; ++w) {
           const int left = v_rows - 32 * w;
@@ -550,6 +546,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
         for (int w = 0; w < BN / 32; ++w) allow[w] = s_anc[node][tt * (BN / 32) + w];
       }
+      ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      if (p.paged && cache_tile) {
+        // the producer's verdict on this tile's pages, written before it armed the V barrier (the
+        // V stage is not reused before this tile's P V, so the flag is stable)
+        ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (!*(volatile int*)&s_tile_ok[st]) {  // sequence is flagged; hide the whole tile
+          v_rows = 0;
+#pragma unroll
+          for (int w = 0; w < BN / 32; ++w) allow[w] = 0;
+        }
+      }
+
       bool full = row_valid;
 #pragma unroll
       for (int w = 0; w < BN / 32; ++w) {
@@ -557,11 +570,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         full = full && (allow[w] == 0xFFFFFFFFu);
       }
       const bool all_full = __all_sync(0xFFFFFFFFu, full);
-
-      ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag);
-      ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) break;
-      tc_fence_after();
 
       uint32_t sv[64];
       // loads half h of the row and replaces the scores of columns that are not allowed by -inf
