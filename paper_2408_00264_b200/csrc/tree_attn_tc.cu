@@ -49,7 +49,7 @@ constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: abo
 template <int MT>
 struct Cfg {
   static constexpr int BN = 128;                         // keys per tile
-  static constexpr int kStages = (MT == 2) ? 2 : 3;      // ring depth, K and V each
+  static constexpr int kStages = 2;                      // ring depth, K and V each
   static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
   static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kTile + 1024;
 };
