@@ -216,7 +216,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the normalised weights.
 template <int NSRC, int MT>
 __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
-                                           int warp, int lane, int tile_base, int rows_total, int G,
+                                           int rot, int warp, int lane, int tile_base, int rows_total, int G,
                                            int64_t seq_row0, int Hq, int head0, uint16_t* out) {
   constexpr int RB = 16 / NSRC;
   for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
@@ -227,9 +227,10 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
       const uint32_t off = (uint32_t)(trow * HD + ((lane ^ (trow & 31)) << 2)) * 4u;
 #pragma unroll
-      for (int q = 0; q < NSRC; ++q) {
+      for (int j = 0; j < NSRC; ++j) {
+        const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
         const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-        x[u * NSRC + q] = dsmem_ld16(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 4) + off, qc));
+        x[u * NSRC + j] = dsmem_ld16(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 4) + off, qc));
       }
     }
 #pragma unroll
@@ -241,9 +242,9 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
       if (rg >= rows_total) continue;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int q = 0; q < NSRC; ++q) {
-        const float wq = w[k * NSRC + q];
-        const float4 v = x[u * NSRC + q];
+      for (int j = 0; j < NSRC; ++j) {
+        const float wq = w[k * NSRC + ((j + rot) & (NSRC - 1))];
+        const float4 v = x[u * NSRC + j];
         acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
       }
       const int onode = rg / G, ogq = rg - onode * G;
@@ -785,13 +786,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncthreads();
     // (b) weighted sums, rows spread over the warps
     const uint32_t sO_addr = smem_u32(sO);
+    const int rot = (split + 1) * (MT == 1 ? 2 : 1);  // first source read: the next block's
     uint16_t* outp = p.out;
     const int64_t seq_row0 = (int64_t)b * N;
     switch (n_src) {
-      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
