@@ -13,9 +13,10 @@
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
 //   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
 //           accumulators are merged like split-KV partials.
-// Split-KV: the blocks that share a row tile form a thread-block cluster; each stages its
-// accumulators in its own shared memory and every block finalises a share of the rows by reading
-// its peers' staging areas (distributed shared memory), so no partial result touches global memory.
+// Split-KV: the blocks that share a row tile form a thread-block cluster; every block finalises
+// a share of the rows, and each block stores its accumulator rows straight into the shared
+// memory of the block that finalises them (distributed shared memory; stores, unlike remote
+// loads, do not wait for their round trip), so no partial result touches global memory.
 // Per slot and key tile:  S = Q K^T (tcgen05.mma -> TMEM)  ->  softmax thread reads its row of S,
 // masks, exponentiates against a lazily updated reference maximum, writes P (bf16) back to tensor
 // memory  ->  O += P V (tcgen05.mma with A from TMEM, accumulator stays in TMEM).  While one slot is in its softmax
@@ -180,25 +181,19 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 }
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
 
-// Distributed shared memory: address of the same variable in block `rank` of the cluster, and a
-// 16-byte load from it.  The loads are volatile asm so that a batch of them is issued back to back
-// (all in flight together) before the first result is used.
+// Distributed shared memory: address of the same variable in block `rank` of the cluster, and
+// stores to it.
 __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(addr));
-  return v;
+__device__ __forceinline__ void dsmem_st16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
+               : "memory");
 }
-__device__ __forceinline__ float2 dsmem_ld8(uint32_t addr) {
-  float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
-  return v;
+__device__ __forceinline__ void dsmem_st8(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -211,46 +206,29 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Final combination of NSRC accumulators per output row, for the rows [k_begin, k_end) that this
-// block finalises.  One warp takes 16 / NSRC rows at a time (16 remote 16-byte loads in flight
-// per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the normalised weights.
-template <int NSRC, int MT>
-__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
-                                           int rot, int warp, int lane, int tile_base, int rows_total, int G,
+// Final combination of NSRC accumulators per output row, for the per_rank rows this block owns.
+// Its peers have written their accumulators for these rows into this block's own shared memory
+// ([source][row][128] fp32, 16-byte chunk c of row k stored at chunk c ^ (k & 31)), so every load
+// is local.  One warp per row, lane j owns output columns 4j .. 4j+3; w[] = normalised weights.
+template <int NSRC>
+__device__ __forceinline__ void merge_rows(const float* recv, const float* w, int first_row, int per_rank,
+                                           int warp, int lane, int tile_base, int rows_total, int G,
                                            int64_t seq_row0, int Hq, int head0, uint16_t* out) {
-  constexpr int RB = 16 / NSRC;
-  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
-    float4 x[RB * NSRC];
+  for (int k = warp; k < per_rank; k += kThreads / 32) {
+    const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+    const int rg = (tile_base + tile) * BM + trow;
+    if (rg >= rows_total) continue;
+    const float* src = recv + (size_t)k * HD + ((lane ^ (k & 31)) << 2);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int u = 0; u < RB; ++u) {
-      const int k = min(k0 + u, per_rank - 1);
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const uint32_t off = (uint32_t)(trow * HD + ((lane ^ (trow & 31)) << 2)) * 4u;
-#pragma unroll
-      for (int j = 0; j < NSRC; ++j) {
-        const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
-        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-        x[u * NSRC + j] = dsmem_ld16(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 4) + off, qc));
-      }
+    for (int q = 0; q < NSRC; ++q) {
+      const float wq = w[k * NSRC + q];
+      const float4 v = *reinterpret_cast<const float4*>(src + (size_t)q * per_rank * HD);
+      acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
     }
-#pragma unroll
-    for (int u = 0; u < RB; ++u) {
-      if (k0 + u >= per_rank) continue;
-      const int k = k0 + u;
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const int rg = (tile_base + tile) * BM + trow;
-      if (rg >= rows_total) continue;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int j = 0; j < NSRC; ++j) {
-        const float wq = w[k * NSRC + ((j + rot) & (NSRC - 1))];
-        const float4 v = x[u * NSRC + j];
-        acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
-      }
-      const int onode = rg / G, ogq = rg - onode * G;
-      uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
-      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-    }
+    const int onode = rg / G, ogq = rg - onode * G;
+    uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
   }
 }
 
@@ -702,6 +680,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // both conflict free.  It reuses the tile memory, which nothing reads any more.
   float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));
 
+  // With a split, every block sends each accumulator row to the block that finalises it, straight
+  // into that block's shared memory (the tile memory, which is dead once ALL blocks of the
+  // cluster are past their loops - hence the cluster barrier first).  Remote stores do not wait
+  // for their round trip, unlike remote loads.
+  const int per_rank = MT * BM / p.splits;   // rows each block finalises; per_rank * n_src = 256
+  if (n_src > 1) cg::this_cluster().sync();
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
       // only accumulator of these rows: normalise and store
@@ -727,7 +711,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (p.lse != nullptr && row_valid)
         p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
     } else {
-      float* orow = sO + ((size_t)slot * BM + row) * HD;
+      const int rr = ((MT == 2) ? slot * BM : 0) + row;       // row within the block's row tile(s)
+      const int owner = rr / per_rank, k = rr - owner * per_rank;
+      const int q = (MT == 2) ? split : split * 2 + slot;     // which source this accumulator is
+      const uint32_t orow = dsmem_addr(smem_u32(sO) + (uint32_t)((q * per_rank + k) * HD) * 4u, owner);
 #pragma unroll 1
       for (int c = 0; c < HD; c += 32) {
         uint32_t ov[32];
@@ -741,11 +728,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
         for (int q4 = 0; q4 < 8; ++q4) {
           const int chunk = (c >> 2) + q4;
-          *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 31)) << 2)) =
-              make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]);
+          dsmem_st16(orow + (uint32_t)((chunk ^ (k & 31)) << 4), ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2],
+                     ov[q4 * 4 + 3]);
         }
       }
-      s_ml[slot][row] = make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f);
+      dsmem_st8(dsmem_addr(smem_u32(&s_ml[0][0]) + (uint32_t)(q * per_rank + k) * 8u, owner),
+                my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f);
     }
   }
   tc_fence_before();
@@ -754,22 +742,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (aborted && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
   if (n_src == 1) return;  // such a block is its own cluster
 
-  // ---- merge across the cluster (the split-KV blocks of one row tile) through distributed
-  //      shared memory: rank j finalises rows [j, j+1) * rows/splits of the tile(s) ------------
+  // ---- merge: every block combines the n_src accumulators of its own rows, all in local memory --
   cg::cluster_group cluster = cg::this_cluster();
-  cluster.sync();  // every block's staging area is complete (also reached by an aborted block)
+  cluster.sync();  // all accumulators have arrived (also reached by an aborted block)
   if (!aborted) {
-    // Every rank finalises per_rank rows; per_rank * n_src is 256 whatever the split count.
-    const int per_rank = MT * BM / p.splits;
     const int first_row = split * per_rank;
-    // (a) thread (k, q) fetches the (maximum, sum) pair of source q of row k; the n_src lanes of a
-    //     row sit side by side in one warp, so the normalised weights come from shuffles.
-    //     Source q is (block q, slot `tile`) when MT == 2 and (block q / 2, slot q % 2) when MT == 1.
+    const float2* mlr = &s_ml[0][0];  // [source][row of this rank]
+    // (a) thread (k, q): the n_src lanes of a row sit side by side, weights come from shuffles
     if (tid < 2 * BM) {
       const int k = tid / n_src, q = tid - k * n_src;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-      const float2 ml = dsmem_ld8(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
+      const float2 ml = mlr[q * per_rank + k];
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
@@ -784,19 +767,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
     }
     __syncthreads();
-    // (b) weighted sums, rows spread over the warps
-    const uint32_t sO_addr = smem_u32(sO);
-    const int rot = (split + 1) * (MT == 1 ? 2 : 1);  // first source read: the next block's
-    uint16_t* outp = p.out;
+    // (b) weighted sums, one warp per row
     const int64_t seq_row0 = (int64_t)b * N;
     switch (n_src) {
-      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 2: merge_rows<2>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      case 4: merge_rows<4>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      case 8: merge_rows<8>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      default: merge_rows<16>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
     }
   }
-  cluster.sync();  // no block may leave while a peer still reads its shared memory
 }
 
 // ------------------------------------------------------------------------------------ host side
