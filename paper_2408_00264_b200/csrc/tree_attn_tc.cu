@@ -13,10 +13,9 @@
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
 //   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
 //           accumulators are merged like split-KV partials.
-// Split-KV: the blocks that share a row tile form a thread-block cluster; every block finalises
-// a share of the rows, and each block stores its accumulator rows straight into the shared
-// memory of the block that finalises them (distributed shared memory; stores, unlike remote
-// loads, do not wait for their round trip), so no partial result touches global memory.
+// Split-KV: the blocks that share a row tile form a thread-block cluster (so that they run
+// together and can use the cluster barrier); every block finalises a share of the rows, and the
+// accumulator rows travel to the finalising block through an L2-resident exchange area.
 // Per slot and key tile:  S = Q K^T (tcgen05.mma -> TMEM)  ->  softmax thread reads its row of S,
 // masks, exponentiates against a lazily updated reference maximum, writes P (bf16) back to tensor
 // memory  ->  O += P V (tcgen05.mma with A from TMEM, accumulator stays in TMEM).  While one slot is in its softmax
@@ -62,6 +61,7 @@ struct Params {
   uint16_t* out;
   float* lse;
   int32_t* status;
+  float* part;     // split-KV exchange area: [row-tile block][owner][source][row][128] fp32, then (m, l) pairs
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
   int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
@@ -181,21 +181,6 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 }
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
 
-// Distributed shared memory: address of the same variable in block `rank` of the cluster, and
-// stores to it.
-__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void dsmem_st16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
-               : "memory");
-}
-__device__ __forceinline__ void dsmem_st8(uint32_t addr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
-}
-
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -207,9 +192,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Final combination of NSRC accumulators per output row, for the per_rank rows this block owns.
-// Its peers have written their accumulators for these rows into this block's own shared memory
-// ([source][row][128] fp32, 16-byte chunk c of row k stored at chunk c ^ (k & 31)), so every load
-// is local.  One warp per row, lane j owns output columns 4j .. 4j+3; w[] = normalised weights.
+// recv = this block's part of the exchange area ([source][row][128] fp32, L2 resident).  One warp
+// per row, lane j owns output columns 4j .. 4j+3, the NSRC loads of a row are independent;
+// w[] = normalised weights.
 template <int NSRC>
 __device__ __forceinline__ void merge_rows(const float* recv, const float* w, int first_row, int per_rank,
                                            int warp, int lane, int tile_base, int rows_total, int G,
@@ -218,13 +203,16 @@ __device__ __forceinline__ void merge_rows(const float* recv, const float* w, in
     const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
     const int rg = (tile_base + tile) * BM + trow;
     if (rg >= rows_total) continue;
-    const float* src = recv + (size_t)k * HD + ((lane ^ (k & 31)) << 2);
+    const float* src = recv + (size_t)k * HD + lane * 4;
+    float4 v[NSRC];
+#pragma unroll
+    for (int q = 0; q < NSRC; ++q)
+      v[q] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)q * per_rank * HD));
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int q = 0; q < NSRC; ++q) {
       const float wq = w[k * NSRC + q];
-      const float4 v = *reinterpret_cast<const float4*>(src + (size_t)q * per_rank * HD);
-      acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
+      acc.x += wq * v[q].x; acc.y += wq * v[q].y; acc.z += wq * v[q].z; acc.w += wq * v[q].w;
     }
     const int onode = rg / G, ogq = rg - onode * G;
     uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
@@ -251,7 +239,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ int s_tile_ok[Cfg<MT>::kStages];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
   __shared__ float s_w[2 * BM];    // merge: normalised weight of every (row of this rank, source)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -675,17 +662,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const bool aborted = *abort_flag != 0;
   const int n_src = p.splits * (MT == 1 ? 2 : 1);  // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
-  // staging area for the merge: O of both slots as fp32 [slot][128 rows][128], 16-byte chunk c of
-  // row r stored at chunk (c ^ (r & 31)) so that row-per-thread writes and row-per-warp reads are
-  // both conflict free.  It reuses the tile memory, which nothing reads any more.
-  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));
-
-  // With a split, every block sends each accumulator row to the block that finalises it, straight
-  // into that block's shared memory (the tile memory, which is dead once ALL blocks of the
-  // cluster are past their loops - hence the cluster barrier first).  Remote stores do not wait
-  // for their round trip, unlike remote loads.
+  // With a split, every block hands each accumulator row to the block that finalises it through
+  // the exchange area in global memory (it stays in L2).  Measured on this part: distributed shared
+  // memory moves only about 15 bytes per clock per SM in either direction, several times less
+  // than L2, and this exchange is 128 KB per block.
   const int per_rank = MT * BM / p.splits;   // rows each block finalises; per_rank * n_src = 256
-  if (n_src > 1) cg::this_cluster().sync();
+  float* const xch = p.part + (size_t)blockIdx.x * p.splits * (2 * BM) * (HD + 2);  // this cluster's area
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
       // only accumulator of these rows: normalise and store
@@ -714,7 +696,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int rr = ((MT == 2) ? slot * BM : 0) + row;       // row within the block's row tile(s)
       const int owner = rr / per_rank, k = rr - owner * per_rank;
       const int q = (MT == 2) ? split : split * 2 + slot;     // which source this accumulator is
-      const uint32_t orow = dsmem_addr(smem_u32(sO) + (uint32_t)((q * per_rank + k) * HD) * 4u, owner);
+      float* orow = xch + ((size_t)owner * (2 * BM) + q * per_rank + k) * HD;
 #pragma unroll 1
       for (int c = 0; c < HD; c += 32) {
         uint32_t ov[32];
@@ -728,12 +710,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
         for (int q4 = 0; q4 < 8; ++q4) {
           const int chunk = (c >> 2) + q4;
-          dsmem_st16(orow + (uint32_t)((chunk ^ (k & 31)) << 4), ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2],
-                     ov[q4 * 4 + 3]);
+          __stcg(reinterpret_cast<uint4*>(orow + (chunk << 2)),
+                 make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]));
         }
       }
-      dsmem_st8(dsmem_addr(smem_u32(&s_ml[0][0]) + (uint32_t)(q * per_rank + k) * 8u, owner),
-                my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f);
+      float* mlx = xch + (size_t)p.splits * (2 * BM) * HD;   // (m, l) pairs behind the accumulators
+      __stcg(reinterpret_cast<float2*>(mlx + ((size_t)owner * (2 * BM) + q * per_rank + k) * 2),
+             make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f));
+      __threadfence();
     }
   }
   tc_fence_before();
@@ -744,15 +728,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   // ---- merge: every block combines the n_src accumulators of its own rows, all in local memory --
   cg::cluster_group cluster = cg::this_cluster();
-  cluster.sync();  // all accumulators have arrived (also reached by an aborted block)
+  cluster.sync();  // all accumulators are in the exchange area (also reached by an aborted block)
   if (!aborted) {
     const int first_row = split * per_rank;
-    const float2* mlr = &s_ml[0][0];  // [source][row of this rank]
+    const float* recv = xch + (size_t)split * (2 * BM) * HD;
+    const float2* mlr = reinterpret_cast<const float2*>(xch + (size_t)p.splits * (2 * BM) * HD) + split * (2 * BM);
     // (a) thread (k, q): the n_src lanes of a row sit side by side, weights come from shuffles
     if (tid < 2 * BM) {
       const int k = tid / n_src, q = tid - k * n_src;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const float2 ml = mlr[q * per_rank + k];
+      const float2 ml = __ldcg(mlr + q * per_rank + k);
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
@@ -770,10 +755,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // (b) weighted sums, one warp per row
     const int64_t seq_row0 = (int64_t)b * N;
     switch (n_src) {
-      case 2: merge_rows<2>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-      case 4: merge_rows<4>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-      case 8: merge_rows<8>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-      default: merge_rows<16>(sO, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      case 2: merge_rows<2>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      case 4: merge_rows<4>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      case 8: merge_rows<8>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      default: merge_rows<16>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
     }
   }
 }
@@ -841,7 +826,8 @@ AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
     splits *= 2;
   pl.splits = splits;
   pl.tickets = 0;
-  pl.scratch_bytes = 0;  // nothing goes through global memory
+  const int n_src = splits * (mt == 1 ? 2 : 1);
+  pl.scratch_bytes = n_src > 1 ? (size_t)ctas * splits * (2 * BM) * (HD + 2) * sizeof(float) : 0;
   return pl;
 }
 
@@ -850,7 +836,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
                                 cudaStream_t stream) {
-  (void)tickets; (void)scratch;
+  (void)tickets;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = G * s.n_nodes;
   const int mt = rows > BM ? 2 : 1;
@@ -881,6 +867,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.status = status;
+  p.part = static_cast<float*>(scratch);
   const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
   p.B = s.batch; p.N = s.n_nodes; p.Hq = s.n_q_heads; p.Hkv = s.n_kv_heads; p.G = G;
   p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
