@@ -199,24 +199,34 @@ template <int NSRC>
 __device__ __forceinline__ void merge_rows(const float* recv, const float* w, int first_row, int per_rank,
                                            int warp, int lane, int tile_base, int rows_total, int G,
                                            int64_t seq_row0, int Hq, int head0, uint16_t* out) {
-  for (int k = warp; k < per_rank; k += kThreads / 32) {
-    const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-    const int rg = (tile_base + tile) * BM + trow;
-    if (rg >= rows_total) continue;
-    const float* src = recv + (size_t)k * HD + lane * 4;
-    float4 v[NSRC];
+  constexpr int RB = 16 / NSRC;  // rows per warp pass: 16 independent 16-byte loads per lane
+  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
+    float4 v[RB * NSRC];
 #pragma unroll
-    for (int q = 0; q < NSRC; ++q)
-      v[q] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)q * per_rank * HD));
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int u = 0; u < RB; ++u) {
+      const int k = min(k0 + u, per_rank - 1);
 #pragma unroll
-    for (int q = 0; q < NSRC; ++q) {
-      const float wq = w[k * NSRC + q];
-      acc.x += wq * v[q].x; acc.y += wq * v[q].y; acc.z += wq * v[q].z; acc.w += wq * v[q].w;
+      for (int q = 0; q < NSRC; ++q)
+        v[u * NSRC + q] = __ldcg(reinterpret_cast<const float4*>(recv + ((size_t)q * per_rank + k) * HD + lane * 4));
     }
-    const int onode = rg / G, ogq = rg - onode * G;
-    uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      const int k = k0 + u;
+      if (k >= per_rank) continue;
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const int rg = (tile_base + tile) * BM + trow;
+      if (rg >= rows_total) continue;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int q = 0; q < NSRC; ++q) {
+        const float wq = w[k * NSRC + q];
+        const float4 x = v[u * NSRC + q];
+        acc.x += wq * x.x; acc.y += wq * x.y; acc.z += wq * x.z; acc.w += wq * x.w;
+      }
+      const int onode = rg / G, ogq = rg - onode * G;
+      uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+    }
   }
 }
 
@@ -667,6 +677,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // memory moves only about 15 bytes per clock per SM in either direction, several times less
   // than L2, and this exchange is 128 KB per block.
   const int per_rank = MT * BM / p.splits;   // rows each block finalises; per_rank * n_src = 256
+  // Step 1: thread-per-row copy of O out of TMEM into this block's (now idle) tile memory, 16-byte
+  // chunk c of row r at chunk c ^ (r & 31) (conflict free for these writes and for the row-wise
+  // reads of step 2).  Step 2: whole rows go out to the exchange area, 512 contiguous bytes per
+  // warp instruction.  (Writing rows to global memory straight from the thread-per-row layout
+  // costs 32 separate 16-byte transactions per instruction and was 6 times slower.)
+  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));  // [slot][128][128]
   float* const xch = p.part + (size_t)blockIdx.x * p.splits * (2 * BM) * (HD + 2);  // this cluster's area
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
@@ -696,7 +712,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int rr = ((MT == 2) ? slot * BM : 0) + row;       // row within the block's row tile(s)
       const int owner = rr / per_rank, k = rr - owner * per_rank;
       const int q = (MT == 2) ? split : split * 2 + slot;     // which source this accumulator is
-      float* orow = xch + ((size_t)owner * (2 * BM) + q * per_rank + k) * HD;
+      float* orow = sO + ((size_t)slot * BM + row) * HD;
 #pragma unroll 1
       for (int c = 0; c < HD; c += 32) {
         uint32_t ov[32];
@@ -710,19 +726,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
         for (int q4 = 0; q4 < 8; ++q4) {
           const int chunk = (c >> 2) + q4;
-          __stcg(reinterpret_cast<uint4*>(orow + (chunk << 2)),
-                 make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]));
+          *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 31)) << 2)) =
+              make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]);
         }
       }
       float* mlx = xch + (size_t)p.splits * (2 * BM) * HD;   // (m, l) pairs behind the accumulators
       __stcg(reinterpret_cast<float2*>(mlx + ((size_t)owner * (2 * BM) + q * per_rank + k) * 2),
              make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f));
-      __threadfence();
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+  if (!aborted && n_src > 1) {
+    for (int lr = warp; lr < 2 * BM; lr += kThreads / 32) {  // local row = slot * 128 + row
+      const int sl = lr / BM, rw = lr % BM;
+      const int rr = ((MT == 2) ? sl * BM : 0) + rw;
+      const int owner = rr / per_rank, k = rr - owner * per_rank;
+      const int q = (MT == 2) ? split : split * 2 + sl;
+      const float4 x = *reinterpret_cast<const float4*>(sO + (size_t)lr * HD + ((lane ^ (rw & 31)) << 2));
+      __stcg(reinterpret_cast<float4*>(xch + ((size_t)owner * (2 * BM) + q * per_rank + k) * HD + lane * 4), x);
+    }
+    __threadfence();
+  }
   if (aborted && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
   if (n_src == 1) return;  // such a block is its own cluster
 
