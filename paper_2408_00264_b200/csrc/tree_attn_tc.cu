@@ -13,9 +13,9 @@
 //   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
 //   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
 //           accumulators are merged like split-KV partials.
-// Split-KV: the blocks that share a row tile form a thread-block cluster (so that they run
-// together and can use the cluster barrier); every block finalises a share of the rows, and the
-// accumulator rows travel to the finalising block through an L2-resident exchange area.
+// Split-KV: the blocks that share a row tile form a thread-block cluster; each stages its
+// accumulators in its own shared memory and every block finalises a share of the rows by reading
+// its peers' staging areas (distributed shared memory), so no partial result touches global memory.
 // Per slot and key tile:  S = Q K^T (tcgen05.mma -> TMEM)  ->  softmax thread reads its row of S,
 // masks, exponentiates against a lazily updated reference maximum, writes P (bf16) back to tensor
 // memory  ->  O += P V (tcgen05.mma with A from TMEM, accumulator stays in TMEM).  While one slot is in its softmax
@@ -61,7 +61,6 @@ struct Params {
   uint16_t* out;
   float* lse;
   int32_t* status;
-  float* part;     // split-KV exchange area: [row-tile block][owner][source][row][128] fp32, then (m, l) pairs
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
   int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
@@ -181,6 +180,27 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 }
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
 
+// Distributed shared memory: address of the same variable in block `rank` of the cluster, and a
+// 16-byte load from it.  The loads are volatile asm so that a batch of them is issued back to back
+// (all in flight together) before the first result is used.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 dsmem_ld8(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -191,37 +211,41 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Final combination of NSRC accumulators per output row, for the per_rank rows this block owns.
-// recv = this block's part of the exchange area ([source][row][128] fp32, L2 resident).  One warp
-// per row, lane j owns output columns 4j .. 4j+3, the NSRC loads of a row are independent;
-// w[] = normalised weights.
-template <int NSRC>
-__device__ __forceinline__ void merge_rows(const float* recv, const float* w, int first_row, int per_rank,
-                                           int warp, int lane, int tile_base, int rows_total, int G,
+// Final combination of NSRC accumulators per output row, for the rows [k_begin, k_end) that this
+// block finalises.  One warp takes 16 / NSRC rows at a time (16 remote 16-byte loads in flight
+// per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the normalised weights.
+template <int NSRC, int MT>
+__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
+                                           int rot, int warp, int lane, int tile_base, int rows_total, int G,
                                            int64_t seq_row0, int Hq, int head0, uint16_t* out) {
-  constexpr int RB = 16 / NSRC;  // rows per warp pass: 16 independent 16-byte loads per lane
+  constexpr int RB = 16 / NSRC;
   for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
-    float4 v[RB * NSRC];
+    float4 x[RB * NSRC];
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
       const int k = min(k0 + u, per_rank - 1);
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const uint32_t off = (uint32_t)(trow * HD + ((lane ^ (trow & 31)) << 2)) * 4u;
 #pragma unroll
-      for (int q = 0; q < NSRC; ++q)
-        v[u * NSRC + q] = __ldcg(reinterpret_cast<const float4*>(recv + ((size_t)q * per_rank + k) * HD + lane * 4));
+      for (int j = 0; j < NSRC; ++j) {
+        const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
+        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+        x[u * NSRC + j] = dsmem_ld16(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 4) + off, qc));
+      }
     }
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
+      if (k0 + u >= per_rank) continue;
       const int k = k0 + u;
-      if (k >= per_rank) continue;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
       const int rg = (tile_base + tile) * BM + trow;
       if (rg >= rows_total) continue;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int q = 0; q < NSRC; ++q) {
-        const float wq = w[k * NSRC + q];
-        const float4 x = v[u * NSRC + q];
-        acc.x += wq * x.x; acc.y += wq * x.y; acc.z += wq * x.z; acc.w += wq * x.w;
+      for (int j = 0; j < NSRC; ++j) {
+        const float wq = w[k * NSRC + ((j + rot) & (NSRC - 1))];
+        const float4 v = x[u * NSRC + j];
+        acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
       }
       const int onode = rg / G, ogq = rg - onode * G;
       uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
@@ -249,6 +273,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ int s_tile_ok[Cfg<MT>::kStages];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
+  __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
   __shared__ float s_w[2 * BM];    // merge: normalised weight of every (row of this rank, source)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -672,18 +697,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const bool aborted = *abort_flag != 0;
   const int n_src = p.splits * (MT == 1 ? 2 : 1);  // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
-  // With a split, every block hands each accumulator row to the block that finalises it through
-  // the exchange area in global memory (it stays in L2).  Measured on this part: distributed shared
-  // memory moves only about 15 bytes per clock per SM in either direction, several times less
-  // than L2, and this exchange is 128 KB per block.
-  const int per_rank = MT * BM / p.splits;   // rows each block finalises; per_rank * n_src = 256
-  // Step 1: thread-per-row copy of O out of TMEM into this block's (now idle) tile memory, 16-byte
-  // chunk c of row r at chunk c ^ (r & 31) (conflict free for these writes and for the row-wise
-  // reads of step 2).  Step 2: whole rows go out to the exchange area, 512 contiguous bytes per
-  // warp instruction.  (Writing rows to global memory straight from the thread-per-row layout
-  // costs 32 separate 16-byte transactions per instruction and was 6 times slower.)
-  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));  // [slot][128][128]
-  float* const xch = p.part + (size_t)blockIdx.x * p.splits * (2 * BM) * (HD + 2);  // this cluster's area
+  // staging area for the merge: O of both slots as fp32 [slot][128 rows][128], 16-byte chunk c of
+  // row r stored at chunk (c ^ (r & 31)) so that row-per-thread writes and row-per-warp reads are
+  // both conflict free.  It reuses the tile memory, which nothing reads any more.
+  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));
+
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
       // only accumulator of these rows: normalise and store
@@ -709,9 +727,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (p.lse != nullptr && row_valid)
         p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
     } else {
-      const int rr = ((MT == 2) ? slot * BM : 0) + row;       // row within the block's row tile(s)
-      const int owner = rr / per_rank, k = rr - owner * per_rank;
-      const int q = (MT == 2) ? split : split * 2 + slot;     // which source this accumulator is
       float* orow = sO + ((size_t)slot * BM + row) * HD;
 #pragma unroll 1
       for (int c = 0; c < HD; c += 32) {
@@ -730,40 +745,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]);
         }
       }
-      float* mlx = xch + (size_t)p.splits * (2 * BM) * HD;   // (m, l) pairs behind the accumulators
-      __stcg(reinterpret_cast<float2*>(mlx + ((size_t)owner * (2 * BM) + q * per_rank + k) * 2),
-             make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f));
+      s_ml[slot][row] = make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f);
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-  if (!aborted && n_src > 1) {
-    for (int lr = warp; lr < 2 * BM; lr += kThreads / 32) {  // local row = slot * 128 + row
-      const int sl = lr / BM, rw = lr % BM;
-      const int rr = ((MT == 2) ? sl * BM : 0) + rw;
-      const int owner = rr / per_rank, k = rr - owner * per_rank;
-      const int q = (MT == 2) ? split : split * 2 + sl;
-      const float4 x = *reinterpret_cast<const float4*>(sO + (size_t)lr * HD + ((lane ^ (rw & 31)) << 2));
-      __stcg(reinterpret_cast<float4*>(xch + ((size_t)owner * (2 * BM) + q * per_rank + k) * HD + lane * 4), x);
-    }
-    __threadfence();
-  }
   if (aborted && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
   if (n_src == 1) return;  // such a block is its own cluster
 
-  // ---- merge: every block combines the n_src accumulators of its own rows, all in local memory --
+  // ---- merge across the cluster (the split-KV blocks of one row tile) through distributed
+  //      shared memory: rank j finalises rows [j, j+1) * rows/splits of the tile(s) ------------
   cg::cluster_group cluster = cg::this_cluster();
-  cluster.sync();  // all accumulators are in the exchange area (also reached by an aborted block)
+  cluster.sync();  // every block's staging area is complete (also reached by an aborted block)
   if (!aborted) {
+    // Every rank finalises per_rank rows; per_rank * n_src is 256 whatever the split count.
+    const int per_rank = MT * BM / p.splits;
     const int first_row = split * per_rank;
-    const float* recv = xch + (size_t)split * (2 * BM) * HD;
-    const float2* mlr = reinterpret_cast<const float2*>(xch + (size_t)p.splits * (2 * BM) * HD) + split * (2 * BM);
-    // (a) thread (k, q): the n_src lanes of a row sit side by side, weights come from shuffles
+    // (a) thread (k, q) fetches the (maximum, sum) pair of source q of row k; the n_src lanes of a
+    //     row sit side by side in one warp, so the normalised weights come from shuffles.
+    //     Source q is (block q, slot `tile`) when MT == 2 and (block q / 2, slot q % 2) when MT == 1.
     if (tid < 2 * BM) {
       const int k = tid / n_src, q = tid - k * n_src;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const float2 ml = __ldcg(mlr + q * per_rank + k);
+      const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+      const float2 ml = dsmem_ld8(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
@@ -778,15 +784,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
     }
     __syncthreads();
-    // (b) weighted sums, one warp per row
+    // (b) weighted sums, rows spread over the warps
+    const uint32_t sO_addr = smem_u32(sO);
+    const int rot = (split + 1) * (MT == 1 ? 2 : 1);  // first source read: the next block's
+    uint16_t* outp = p.out;
     const int64_t seq_row0 = (int64_t)b * N;
     switch (n_src) {
-      case 2: merge_rows<2>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-      case 4: merge_rows<4>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-      case 8: merge_rows<8>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-      default: merge_rows<16>(recv, s_w, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
     }
   }
+  cluster.sync();  // no block may leave while a peer still reads its shared memory
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -852,8 +862,7 @@ AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
     splits *= 2;
   pl.splits = splits;
   pl.tickets = 0;
-  const int n_src = splits * (mt == 1 ? 2 : 1);
-  pl.scratch_bytes = n_src > 1 ? (size_t)ctas * splits * (2 * BM) * (HD + 2) * sizeof(float) : 0;
+  pl.scratch_bytes = 0;  // nothing goes through global memory
   return pl;
 }
 
@@ -862,7 +871,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
                                 cudaStream_t stream) {
-  (void)tickets;
+  (void)tickets; (void)scratch;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = G * s.n_nodes;
   const int mt = rows > BM ? 2 : 1;
@@ -893,7 +902,6 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.status = status;
-  p.part = static_cast<float*>(scratch);
   const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
   p.B = s.batch; p.N = s.n_nodes; p.Hq = s.n_q_heads; p.Hkv = s.n_kv_heads; p.G = G;
   p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
