@@ -130,6 +130,36 @@ def test_attention_special_trees_and_paging(clv, oracle, tree, paged):
     check_attention(oracle, w, st)
 
 
+@pytest.mark.parametrize("hq,hkv", [(6, 2), (12, 2), (5, 1)])
+def test_attention_group_sizes_that_do_not_divide_128(clv, oracle, hq, hkv):
+    # these shapes are served by the warp-level MMA kernel (a 128-row tile must hold whole nodes)
+    cfg = W.small_config(batch=2, n_q_heads=hq, n_kv_heads=hkv, ctx=(30, 500), n_nodes=37, vocab=64,
+                         seed=W.BASE_SEED + hq)
+    w = W.generate(cfg)
+    st = make_step(w)
+    st.tree_attn()
+    torch.cuda.synchronize()
+    check_attention(oracle, w, st)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_attention_both_kernels_agree_with_the_checker(clv, oracle, paged, monkeypatch):
+    # CLV_ATTN_PATH=mma forces the warp-level kernel on a shape the tcgen05 kernel normally serves
+    cfg = W.small_config(batch=3, n_q_heads=8, n_kv_heads=2, ctx=(100, 900), n_nodes=64, vocab=64,
+                         paged=paged, seed=W.BASE_SEED + 21)
+    w = W.generate(cfg)
+    outs = []
+    for path in ("tc", "mma"):
+        monkeypatch.setenv("CLV_ATTN_PATH", path)
+        st = make_step(w)
+        st.tree_attn()
+        torch.cuda.synchronize()
+        check_attention(oracle, w, st)
+        outs.append(W.bf16_bits_to_f64(bits(st.out)))
+    monkeypatch.delenv("CLV_ATTN_PATH")
+    assert np.abs(outs[0] - outs[1]).max() < 1e-2
+
+
 def test_attention_many_splits_and_ragged(clv, oracle):
     # few (sequence, head) units and a long context: the key axis is split many ways; one
     # sequence is much shorter than max_ctx_len so some splits of it are empty
