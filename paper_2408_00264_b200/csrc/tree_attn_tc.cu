@@ -282,7 +282,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int b = unit / p.Hkv, kvh = unit - b * p.Hkv;
   const int N = p.N, G = p.G, rows_total = G * N;
 
-  // ---- per-sequence checks (same verdict in every block of the sequence) ------------------
+  // ---- set-up and per-sequence checks in one go: while thread 0 initialises the barriers and
+  //      warp 1 allocates tensor memory, everybody reads parent[] and the context length; the one
+  //      block-wide synchronisation below publishes all of it -------------------------------------
+  constexpr int NSTc = Cfg<MT>::kStages;
+  const uint32_t bar0 = smem_u32(&s_bar[0]);
+  if (tid == 0) {
+    for (int i = 0; i < 4 * NSTc; ++i) mbar_init(bar0 + 8u * i, 1);                 // K/V rings
+    mbar_init(bar0 + 8u * (4 * NSTc), 1);                                           // Q
+    for (int s2 = 0; s2 < 2; ++s2) {
+      mbar_init(bar0 + 8u * (4 * NSTc + 1 + s2), 1);                                // S ready
+      mbar_init(bar0 + 8u * (4 * NSTc + 3 + s2), BM);                               // P ready
+      mbar_init(bar0 + 8u * (4 * NSTc + 5 + s2), 1);                                // P V done
+    }
+    mbar_init(bar0 + 8u * (4 * NSTc + 7), 1);                                       // drain
+    s_abort = 0;
+    fence_barrier_init();
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
   const int L = p.ctx_len[b];
   bool bad = false;
   for (int i = tid; i < N; i += kThreads) {
@@ -294,30 +312,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int p_cache = L > 0 ? (L + PG - 1) / PG : 0;  // 64-key pieces (pages) of the context
   if (p.paged) bad |= (p_cache > p.max_pages);
   else bad |= (L > p.cap_tokens);
-  const int seq_bad = __syncthreads_or(bad ? 1 : 0);
+  tc_fence_before();
+  const int seq_bad = __syncthreads_or(bad ? 1 : 0);  // same verdict in every block of the sequence
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
   const bool reporter = (row_cta == 0 && split == 0 && kvh == 0);
-  if (reporter) {
-    bool pbad = false;
-    if (p.paged && !seq_bad) {
-      for (int pg = tid; pg < p_cache; pg += kThreads) {
-        const int e = p.block_table[(int64_t)b * p.max_pages + pg];
-        pbad |= (e < 0 || e >= p.n_pages);
-      }
-    }
-    const int page_bad = __syncthreads_or(pbad ? 1 : 0);
-    if (tid == 0) p.status[b] = (seq_bad || page_bad) ? CLV_ERR_TREE : CLV_OK;
-  }
-  if (seq_bad) return;  // before any barrier or TMEM exists; the whole cluster leaves together
-
-  // ancestor bitsets: row i of the tree's topology matrix
-  for (int i = tid; i < N; i += kThreads) {
-    uint32_t w[4] = {0, 0, 0, 0};
-    int j = i;
-    for (int hop = 0; hop < N && j >= 0; ++hop) {
-      w[j >> 5] |= 1u << (j & 31);
-      j = s_parent[j];
-    }
-    s_anc[i][0] = w[0]; s_anc[i][1] = w[1]; s_anc[i][2] = w[2]; s_anc[i][3] = w[3];
+  if (seq_bad) {  // the whole cluster leaves together; nothing has been issued yet
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (reporter && tid == 0) p.status[b] = CLV_ERR_TREE;
+    return;
   }
 
   // ---- tile range and per-slot rounds -------------------------------------------------------
@@ -338,7 +341,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t sV = sK + NST * kTile;      // ring of NST V tiles
   uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
 
-  const uint32_t bar0 = smem_u32(&s_bar[0]);
   auto bar_k_full = [&](int st) { return bar0 + 8u * st; };
   auto bar_k_empty = [&](int st) { return bar0 + 8u * (NST + st); };
   auto bar_v_full = [&](int st) { return bar0 + 8u * (2 * NST + st); };
@@ -349,24 +351,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto bar_pv_done = [&](int s) { return bar0 + 8u * (4 * NST + 5 + s); };
   const uint32_t bar_drain = bar0 + 8u * (4 * NST + 7);
 
-  if (tid == 0) {
-    for (int i = 0; i < 4 * NST; ++i) mbar_init(bar0 + 8u * i, 1);
-    mbar_init(bar_q, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar_s_full(s), 1);
-      mbar_init(bar_p_full(s), BM);
-      mbar_init(bar_pv_done(s), 1);
-    }
-    mbar_init(bar_drain, 1);
-    s_abort = 0;
-    fence_barrier_init();
-    fence_async_smem();
-  }
-  if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = s_tmem;
   volatile int* abort_flag = &s_abort;
   // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
   // the scores have been read); O of slot s at 2 BN + 128 s
@@ -524,6 +508,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     constexpr int NH = BN / 64;   // the row of S is taken in 64-column halves (register budget)
     const int rounds = my_rounds;
     bool ok = true;
+    // ancestor bitsets (row i of the tree's topology matrix), built by the softmax warps while
+    // the first tiles are on their way; the 256 threads meet at a named barrier of their own
+    for (int i = tid - 64; i < N; i += 2 * BM) {
+      uint32_t w[4] = {0, 0, 0, 0};
+      int j = i;
+      for (int hop = 0; hop < N && j >= 0; ++hop) {
+        w[j >> 5] |= 1u << (j & 31);
+        j = s_parent[j];
+      }
+      s_anc[i][0] = w[0]; s_anc[i][1] = w[1]; s_anc[i][2] = w[2]; s_anc[i][3] = w[3];
+    }
+    if (reporter && warp == 2) {  // one warp per sequence reports: block table of the context
+      bool pbad = false;
+      if (p.paged) {
+        for (int pg = lane; pg < p_cache; pg += 32) {
+          const int e = p.block_table[(int64_t)b * p.max_pages + pg];
+          pbad |= (e < 0 || e >= p.n_pages);
+        }
+      }
+      pbad = __any_sync(0xFFFFFFFFu, pbad);
+      if (lane == 0) p.status[b] = pbad ? CLV_ERR_TREE : CLV_OK;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
 
     for (int r = 0; r < rounds && ok; ++r) {
       const int i = (MT == 2) ? r : 2 * r + slot;
