@@ -301,6 +301,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     fence_async_smem();
   }
   if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+  if (tid == 64) {
+    tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
+    tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
+  }
   const int L = p.ctx_len[b];
   bool bad = false;
   for (int i = tid; i < N; i += kThreads) {
@@ -375,21 +379,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (warp == 0) {
     // =========================== TMA producer ===============================================
-    if (lane == 0) {
-      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
-      tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
-    }
     if (n_tiles > 0) {
-      if (lane == 0) {
-        mbar_expect_tx(bar_q, MT * kQTile);
-        const int nodes_per_tile = BM / G;
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-          const int node0 = b * N + (row_cta * MT + m) * nodes_per_tile;
-          tma_load_3d(sQ + m * kQTile, &tm_q, 0, kvh * G, node0, bar_q);
-          tma_load_3d(sQ + m * kQTile + kQTile / 2, &tm_q, 64, kvh * G, node0, bar_q);
-        }
-      }
       constexpr int kBatch = 32 / PPT;  // tiles whose page numbers one warp-wide fetch covers
       int page_cache = 0;               // lane j: pool page of piece (batch base * PPT + j)
       bool ok = true;
@@ -508,6 +498,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     constexpr int NH = BN / 64;   // the row of S is taken in 64-column halves (register budget)
     const int rounds = my_rounds;
     bool ok = true;
+    if (warp == 2 && n_tiles > 0) {  // the Q tile(s): issued here so that the producer starts with K/V
+      if (lane == 0) {
+        mbar_expect_tx(bar_q, MT * kQTile);
+        const int nodes_per_tile = BM / G;
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          const int node0 = b * N + (row_cta * MT + m) * nodes_per_tile;
+          tma_load_3d(sQ + m * kQTile, &tm_q, 0, kvh * G, node0, bar_q);
+          tma_load_3d(sQ + m * kQTile + kQTile / 2, &tm_q, 64, kvh * G, node0, bar_q);
+        }
+      }
+    }
     // ancestor bitsets (row i of the tree's topology matrix), built by the softmax warps while
     // the first tiles are on their way; the 256 threads meet at a named barrier of their own
     for (int i = tid - 64; i < N; i += 2 * BM) {
