@@ -599,6 +599,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // maximum has outgrown it by more than the gap - rare after the first tile - and then the
       // tile is redone from the scores, which are still intact because P is stored last.
       uint32_t pk[NH * 32];
+      if (r == 0) {  // no reference yet: take the first tile's row maximum (a cheap extra pass)
+        float m0 = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          load_half(h);
+#pragma unroll
+          for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
+        }
+        m_ref = m0 * p.scale_log2;  // stays -inf for a row without any allowed key
+      }
       float mx = -INFINITY, sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
 #pragma unroll
