@@ -328,12 +328,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
 
   // ---- tile range and per-slot rounds -------------------------------------------------------
-  const int t_cache = (p_cache + PPT - 1) / PPT;
-  const int t_tree = (N + BN - 1) / BN;
-  const int t_total = t_cache + t_tree;
-  const int t_begin = (int)((int64_t)split * t_total / p.splits);
-  const int t_end = (int)((int64_t)(split + 1) * t_total / p.splits);
-  const int n_tiles = t_end - t_begin;
+  // The key axis is cut in 64-key pieces: p_cache pieces of context, then the tree's own pieces.
+  // A block takes a contiguous range of pieces (so the split balances to one piece) and walks it
+  // in tiles of PPT pieces; a tile may end early or mix context and tree pieces.
+  const int p_total = p_cache + (N + PG - 1) / PG;
+  const int pc_begin = (int)((int64_t)split * p_total / p.splits);
+  const int pc_end = (int)((int64_t)(split + 1) * p_total / p.splits);
+  const int n_tiles = (pc_end - pc_begin + PPT - 1) / PPT;
   // local tile index of round r of slot s: MT == 2: r;  MT == 1: 2 r + s
   const int rounds0 = (MT == 2) ? n_tiles : (n_tiles + 1) / 2;
   const int rounds1 = (MT == 2) ? n_tiles : n_tiles / 2;
@@ -380,35 +381,34 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     // =========================== TMA producer ===============================================
     if (n_tiles > 0) {
-      constexpr int kBatch = 32 / PPT;  // tiles whose page numbers one warp-wide fetch covers
-      int page_cache = 0;               // lane j: pool page of piece (batch base * PPT + j)
+      int page_cache = 0;   // lane j: pool page of context piece (page_base + j)
+      int page_base = -64;
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
-        const int t = t_begin + i;
         const int st = i % NST;
-        if (p.paged && (i % kBatch) == 0) {
-          const int pc = t * PPT + lane;
+        const int g0 = pc_begin + i * PPT;  // first piece of this tile
+        if (p.paged && g0 < p_cache && g0 + PPT > page_base + 32) {  // warp-uniform refill
+          page_base = g0;
+          const int pc = g0 + lane;
           page_cache = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
         }
-        int row0[PPT];   // first source row of each piece, -1: piece not present
+        int row0[PPT];          // first source row of each piece, -1: piece not present
+        bool is_tree[PPT];
         int tile_ok = 1;
-        const CUtensorMap *mk, *mv;
-        if (t < t_cache) {
-          mk = &tm_kc; mv = &tm_vc;
 #pragma unroll
-          for (int j = 0; j < PPT; ++j) {
-            const int pc = t * PPT + j;
-            int pg = __shfl_sync(0xFFFFFFFFu, page_cache, (i % kBatch) * PPT + j);
-            if (pc < p_cache && (pg < 0 || pg >= p.n_pages)) tile_ok = 0;  // flagged by the reporter
-            if (pg < 0 || pg >= p.n_pages) pg = 0;  // the keys of such a tile get masked
-            row0[j] = (pc >= p_cache) ? -1 : (p.paged ? pg * PG : b * p.cap_tokens + pc * PG);
-          }
-        } else {
-          mk = &tm_kt; mv = &tm_vt;
-#pragma unroll
-          for (int j = 0; j < PPT; ++j) {
-            const int j0 = (t - t_cache) * BN + j * PG;
-            row0[j] = (j0 < N) ? b * N + j0 : -1;
+        for (int j = 0; j < PPT; ++j) {
+          const int g = g0 + j;
+          int pg = __shfl_sync(0xFFFFFFFFu, page_cache, (g - page_base) & 31);
+          is_tree[j] = g >= p_cache;
+          if (g >= pc_end) {
+            row0[j] = -1;
+          } else if (is_tree[j]) {
+            row0[j] = b * N + (g - p_cache) * PG;
+          } else if (p.paged) {
+            if (pg < 0 || pg >= p.n_pages) { tile_ok = 0; pg = 0; }  // flagged by the reporter; masked
+            row0[j] = pg * PG;
+          } else {
+            row0[j] = b * p.cap_tokens + g * PG;
           }
         }
         if (lane == 0) {
@@ -422,6 +422,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
+              const CUtensorMap* mk = is_tree[j] ? &tm_kt : &tm_kc;
               tma_load_3d(sK + st * kTile + j * kPiece, mk, 0, kvh, row0[j], bar_k_full(st));
               tma_load_3d(sK + st * kTile + kHalf + j * kPiece, mk, 64, kvh, row0[j], bar_k_full(st));
             }
@@ -433,6 +434,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
+              const CUtensorMap* mv = is_tree[j] ? &tm_vt : &tm_vc;
               tma_load_3d(sV + st * kTile + j * kPiece, mv, 0, kvh, row0[j], bar_v_full(st));
               tma_load_3d(sV + st * kTile + kHalf + j * kPiece, mv, 64, kvh, row0[j], bar_v_full(st));
             }
@@ -536,25 +538,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     for (int r = 0; r < rounds && ok; ++r) {
       const int i = (MT == 2) ? r : 2 * r + slot;
-      const int t = t_begin + i;
       const int st = i % NST;
-      // allowed columns of this row in this tile, and how many V rows of the tile are real
+      // allowed columns of this row in this tile (64 per piece), and how many rows of each V
+      // piece are real keys
       uint32_t allow[BN / 32];
-      int v_rows;
-      bool cache_tile = false;
-      if (t < t_cache) {
-        v_rows = min(BN, L - t * BN);
-        cache_tile = true;
+      int valid[PPT];
+      bool cache_tile = false, short_tile = false;
 #pragma unroll
-        for (int w = 0; w < BN / 32; ++w) {
-          const int left = v_rows - 32 * w;
-          allow[w] = left >= 32 ? 0xFFFFFFFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
+      for (int j = 0; j < PPT; ++j) {
+        const int g = pc_begin + i * PPT + j;
+        if (g >= pc_end) {                 // the range ended inside this tile
+          valid[j] = 0;
+          allow[2 * j] = allow[2 * j + 1] = 0;
+        } else if (g < p_cache) {          // context piece: everything up to the context length
+          cache_tile = true;
+          valid[j] = min(PG, L - g * PG);
+          const uint64_t bits = valid[j] >= 64 ? ~0ull : ((1ull << valid[j]) - 1ull);
+          allow[2 * j] = (uint32_t)bits; allow[2 * j + 1] = (uint32_t)(bits >> 32);
+        } else {                           // tree piece: the node's ancestors (itself included)
+          const int tp = g - p_cache;
+          valid[j] = min(PG, N - tp * PG);
+          allow[2 * j] = s_anc[node][2 * tp]; allow[2 * j + 1] = s_anc[node][2 * tp + 1];
         }
-      } else {
-        const int tt = t - t_cache;
-        v_rows = min(BN, N - tt * BN);
-#pragma unroll
-        for (int w = 0; w < BN / 32; ++w) allow[w] = s_anc[node][tt * (BN / 32) + w];
+        short_tile |= valid[j] < PG;
       }
       ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
@@ -567,7 +573,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         if (!*(volatile int*)&s_tile_ok[st]) {  // sequence is flagged; hide the whole tile
-          v_rows = 0;
+          short_tile = true;
+#pragma unroll
+          for (int j = 0; j < PPT; ++j) valid[j] = 0;
 #pragma unroll
           for (int w = 0; w < BN / 32; ++w) allow[w] = 0;
         }
@@ -669,18 +677,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       tmem_wait_st();
       l_run += sum;
 
-      if (v_rows < BN) {
-        // Rows of the V tile beyond the real keys hold whatever lies behind them in memory (or were
+      if (short_tile) {
+        // Rows of a V piece beyond its real keys hold whatever lies behind them in memory (or were
         // never loaded); their probabilities are exactly 0, but 0 * NaN would poison O: clear them.
         ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         uint8_t* vt = sV_gen + st * kTile;
-        const int per_half = (BN - v_rows) * 8;  // 16-byte chunks per half of the head dimension
-        for (int c = (warp - 2 - slot * 4) * 32 + lane; c < 2 * per_half; c += BM) {
-          const int half = c / per_half, rem = c - half * per_half;
-          const int vr = v_rows + (rem >> 3), ch = rem & 7;
-          *reinterpret_cast<uint4*>(vt + half * kHalf + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+        const int me = (warp - 2 - slot * 4) * 32 + lane;   // 0 .. 127 within the softmax group
+#pragma unroll
+        for (int j = 0; j < PPT; ++j) {
+          const int per_half = (PG - valid[j]) * 8;  // 16-byte chunks per half of the head dimension
+          for (int c = me; c < 2 * per_half; c += BM) {
+            const int half = c / per_half, rem = c - half * per_half;
+            const int vr = j * PG + valid[j] + (rem >> 3), ch = rem & 7;
+            *reinterpret_cast<uint4*>(vt + half * kHalf + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+          }
         }
         fence_async_smem();   // cleared V rows visible to the tensor core's reads
       }
