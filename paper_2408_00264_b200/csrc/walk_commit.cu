@@ -16,6 +16,11 @@ __global__ void __launch_bounds__(32) walk_kernel(int N, int path_cap, const int
   __shared__ int sp[CLV_MAX_NODES], st[CLV_MAX_NODES], si[CLV_MAX_NODES], path[CLV_MAX_NODES];
   const int b = blockIdx.x, lane = threadIdx.x;
   const int64_t o = (int64_t)b * N;
+  // Launched with programmatic stream serialisation: this grid may be set up while the previous
+  // kernel of the stream is still draining, so wait for that kernel's results here, and let the
+  // next kernel (the commit) start its own set-up right away.
+  cudaGridDependencySynchronize();
+  cudaTriggerProgrammaticLaunchCompletion();
   bool bad = false;
   for (int i = lane; i < N; i += 32) {
     const int p = parent[o + i];
@@ -76,6 +81,7 @@ __global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
   __shared__ long long s_dst[CLV_MAX_NODES];  // destination token row (global row index)
   __shared__ int s_ok;
   const int b = blockIdx.x, tid = threadIdx.x;
+  cudaGridDependencySynchronize();  // programmatic launch: the walk's outputs are complete after this
   const int L = p.ctx_len[b];
   const int len = p.accept_len[b];
   if (tid == 0) s_ok = (L >= 0 && len >= 0 && len <= p.path_cap && len <= CLV_MAX_NODES) ? 1 : 0;
@@ -121,9 +127,17 @@ __global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
 cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
                         const int32_t* ids, int32_t* accept_len, int32_t* accept_idx,
                         int32_t* next_token, int32_t* status, cudaStream_t stream) {
-  walk_kernel<<<s.batch, 32, 0, stream>>>(s.n_nodes, s.path_cap, parent, tokens, ids, accept_len,
-                                          accept_idx, next_token, status);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)s.batch, 1, 1);
+  cfg.blockDim = dim3(32, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, walk_kernel, (int)s.n_nodes, (int)s.path_cap, parent, tokens, ids, accept_len,
+                            accept_idx, next_token, status);
 }
 
 cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void* k_tree,
@@ -148,8 +162,16 @@ cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void*
   p.n_pages = c.n_pages;
   p.max_pages = c.max_pages_per_seq;
   p.row_vec = s.n_kv_heads * CLV_HEAD_DIM * 2 / 16;
-  commit_kernel<<<s.batch, 256, 0, stream>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)s.batch, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, commit_kernel, p);
 }
 
 }  // namespace clv
