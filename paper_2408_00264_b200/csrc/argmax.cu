@@ -85,6 +85,9 @@ __global__ void __launch_bounds__(kThreads) argmax_kernel(Params p) {
   const int nvec = (end - begin) >> 3;
   const uint4* vp = reinterpret_cast<const uint4*>(base + begin);
   const int tid = threadIdx.x;
+  // programmatic launch: the grid may be set up while the previous kernel of the stream drains;
+  // nothing is read or written before that kernel's results are complete
+  cudaGridDependencySynchronize();
 
   Track trk;
   track_init(trk);
@@ -182,8 +185,16 @@ cudaError_t launch_argmax(const ArgmaxPlan& plan, const void* logits, int64_t ld
   p.ids = ids;
   p.tickets = tickets;
   p.partial = static_cast<unsigned long long*>(scratch);
-  argmax_kernel<<<(unsigned)((int64_t)plan.rows * plan.chunks), kThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((int64_t)plan.rows * plan.chunks), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, argmax_kernel, p);
 }
 
 // ---- variant whose scratch lives in the library image ------------------------------------------
