@@ -63,6 +63,7 @@ struct Params {
   int32_t* status;
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
+  int longest_first;  // hand out sequences in order of decreasing context length
   int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
   int splits;      // thread blocks along the key axis = cluster size (1, 2, 4 or 8)
   float scale_log2;
@@ -279,8 +280,28 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.x / p.row_ctas, row_cta = blockIdx.x - unit * p.row_ctas;
   const int split = blockIdx.y;
-  const int b = unit / p.Hkv, kvh = unit - b * p.Hkv;
+  int b = unit / p.Hkv;
+  const int kvh = unit - b * p.Hkv;
   const int N = p.N, G = p.G, rows_total = G * N;
+  if (p.longest_first) {
+    // More blocks than SMs and contexts of different lengths (ragged batch): hand the sequences
+    // out longest first, so that the block scheduler packs the short ones into the gaps.  Block
+    // group `b` takes the sequence whose length has rank b (ties by index); every thread ranks
+    // at most one sequence.
+    __shared__ int s_seq;
+    const int want = b;
+    for (int i = tid; i < p.B; i += kThreads) {
+      const int Li = p.ctx_len[i];
+      int rank = 0;
+      for (int j = 0; j < p.B; ++j) {
+        const int Lj = __ldg(p.ctx_len + j);
+        rank += (Lj > Li) || (Lj == Li && j < i);
+      }
+      if (rank == want) s_seq = i;
+    }
+    __syncthreads();
+    b = s_seq;
+  }
 
   // ---- set-up and per-sequence checks in one go: while thread 0 initialises the barriers and
   //      warp 1 allocates tensor memory, everybody reads parent[] and the context length; the one
@@ -938,6 +959,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
   p.row_ctas = plan.m_tiles;
   p.splits = plan.splits;
+  p.longest_first = (ctas > sm_count() && s.batch > 1 && s.batch <= 256) ? 1 : 0;
   p.scale_log2 = scale * 1.4426950408889634f;
 
   cudaLaunchConfig_t cfg = {};
