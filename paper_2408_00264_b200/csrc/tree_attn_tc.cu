@@ -656,16 +656,29 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int h = 0; h < NH; ++h) {
         load_half(h);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
-          mx = fmaxf(mx, fmaxf(a0, a1));
-          const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
-          // every fourth exponential goes to the FMA pipe when no column is masked (-inf inputs
-          // are left to the special-function unit, which returns an exact zero for them)
-          const float x1 = fmaf(a1, p.scale_log2, neg_m);
-          const float p1 = (all_full && (j & 1)) ? ex2_fma(x1) : ex2(x1);
-          sum += p0 + p1;
-          pk[h * 32 + j] = pack_bf16(p0, p1);
+        if (all_full) {
+          // no masked column: every fourth exponential goes to the FMA pipe (-inf inputs are
+          // left to the special-function unit, which returns an exact zero for them)
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
+            mx = fmaxf(mx, fmaxf(a0, a1));
+            const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
+            const float x1 = fmaf(a1, p.scale_log2, neg_m);
+            const float p1 = (j & 1) ? ex2_fma(x1) : ex2(x1);
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
+            mx = fmaxf(mx, fmaxf(a0, a1));
+            const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(a1, p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
+          }
         }
       }
       mx *= p.scale_log2;  // scale > 0; -inf stays -inf
