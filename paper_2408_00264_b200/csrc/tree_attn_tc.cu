@@ -207,18 +207,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// 2^x on the FMA pipe (round-to-integer by the magic-number add, cubic for the fraction in
-// [-0.5, 0.5], exponent added as an integer); relative error 8e-5, for finite x.  Used for a
-// share of the exponentials because the softmax is bound by the special-function unit.
-__device__ __forceinline__ float ex2_fma(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;        // 1.5 * 2^23: the integer part lands in the low mantissa bits
-  const float r = x - (t - 12582912.f);
-  float q = fmaf(r, 0.05508868f, 0.24260405f);
-  q = fmaf(r, q, 0.69327623f);
-  q = fmaf(r, q, 0.99992895f);
-  return __uint_as_float(__float_as_uint(q) + (__float_as_uint(t) << 23));
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -656,29 +644,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int h = 0; h < NH; ++h) {
         load_half(h);
 #pragma unroll
-        if (all_full) {
-          // no masked column: every fourth exponential goes to the FMA pipe (-inf inputs are
-          // left to the special-function unit, which returns an exact zero for them)
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
-            mx = fmaxf(mx, fmaxf(a0, a1));
-            const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
-            const float x1 = fmaf(a1, p.scale_log2, neg_m);
-            const float p1 = (j & 1) ? ex2_fma(x1) : ex2(x1);
-            sum += p0 + p1;
-            pk[h * 32 + j] = pack_bf16(p0, p1);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
-            mx = fmaxf(mx, fmaxf(a0, a1));
-            const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(a1, p.scale_log2, neg_m));
-            sum += p0 + p1;
-            pk[h * 32 + j] = pack_bf16(p0, p1);
-          }
+        for (int j = 0; j < 32; ++j) {
+          const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
+          mx = fmaxf(mx, fmaxf(a0, a1));
+          const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(a1, p.scale_log2, neg_m));
+          sum += p0 + p1;
+          pk[h * 32 + j] = pack_bf16(p0, p1);
         }
       }
       mx *= p.scale_log2;  // scale > 0; -inf stays -inf
