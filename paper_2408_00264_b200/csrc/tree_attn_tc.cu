@@ -43,7 +43,7 @@ constexpr int kThreads = 320;
 constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
 constexpr uint32_t kTmemCols = 512;
-constexpr float kRescaleGap = 8.0f;           // log2 units: P stays below 2^8
+constexpr float kRowSumLimit = 256.0f;        // a row of P may sum to 2^8 before the reference is replaced
 constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: about a second
 
 template <int MT>
@@ -624,11 +624,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       };
       // One pass with the reference maximum as it stands: exponentiate, pack P (kept in registers)
-      // and track the true row maximum on the way.  The reference is only replaced when the
-      // maximum has outgrown it by more than the gap - rare after the first tile - and then the
-      // tile is redone from the scores, which are still intact because P is stored last.
+      // and add up the row.  No per-element maximum is tracked (the softmax threads are bound by
+      // instruction issue): a row sum of at most 2^8 proves that no probability exceeded 2^8,
+      // i.e. that the reference is still good.  Otherwise (rare after the first tile; inf or NaN
+      // from an overflow also lands here) the true maximum is taken from the scores - still
+      // intact, because P is stored last - the reference replaced, O rescaled and the tile redone.
       uint32_t pk[NH * 32];
-      if (r == 0) {  // no reference yet: take the first tile's row maximum (a cheap extra pass)
+      auto row_max = [&]() {
         float m0 = -INFINITY;
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
@@ -636,26 +638,30 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
         }
-        m_ref = m0 * p.scale_log2;  // stays -inf for a row without any allowed key
-      }
-      float mx = -INFINITY, sum = 0.f;
+        return m0 * p.scale_log2;  // scale > 0; -inf (no allowed key) stays -inf
+      };
+      if (r == 0) m_ref = row_max();  // no reference yet: a cheap extra pass instead of a redo
+      float sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      auto exp_pass = [&]() {
+        sum = 0.f;
 #pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        load_half(h);
+        for (int h = 0; h < NH; ++h) {
+          load_half(h);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float a0 = __uint_as_float(sv[2 * j]), a1 = __uint_as_float(sv[2 * j + 1]);
-          mx = fmaxf(mx, fmaxf(a0, a1));
-          const float p0 = ex2(fmaf(a0, p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(a1, p.scale_log2, neg_m));
-          sum += p0 + p1;
-          pk[h * 32 + j] = pack_bf16(p0, p1);
+          for (int j = 0; j < 32; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
+          }
         }
-      }
-      mx *= p.scale_log2;  // scale > 0; -inf stays -inf
-      const bool need = mx > m_ref + kRescaleGap;  // also true for the first finite maximum
-      if (__any_sync(0xFFFFFFFFu, need)) {
+      };
+      exp_pass();
+      const bool suspect = !(sum <= kRowSumLimit);  // also catches inf and NaN
+      if (__any_sync(0xFFFFFFFFu, suspect)) {
+        const float mx = suspect ? row_max() : m_ref;
+        const bool need = mx > m_ref;
         if (r > 0) {  // O must be at rest: the previous P V has completed
           ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
           ok = __all_sync(0xFFFFFFFFu, ok);
@@ -677,18 +683,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tmem_wait_st();
         }
         neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-        sum = 0.f;
-#pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          load_half(h);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-            sum += p0 + p1;
-            pk[h * 32 + j] = pack_bf16(p0, p1);
-          }
-        }
+        exp_pass();
       }
       // P (the A operand of P V) takes the place of score columns that have been consumed.  The
       // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
