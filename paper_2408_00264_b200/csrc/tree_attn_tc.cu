@@ -270,7 +270,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
-  __shared__ __align__(8) unsigned long long s_bar[4 * NST + 12];
+  __shared__ __align__(8) unsigned long long s_bar[4 * NST + 8];
   __shared__ int s_tile_ok[Cfg<MT>::kStages];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -317,10 +317,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_init(bar0 + 8u * (4 * NSTc + 5 + s2), 1);                                // P V done
     }
     mbar_init(bar0 + 8u * (4 * NSTc + 7), 1);                                       // drain
-    for (int s2 = 0; s2 < 2; ++s2) {
-      mbar_init(bar0 + 8u * (4 * NSTc + 8 + s2), BM);                               // first half of P ready
-      mbar_init(bar0 + 8u * (4 * NSTc + 10 + s2), 1);                               // first half of P V done
-    }
     s_abort = 0;
     fence_barrier_init();
     fence_async_smem();
@@ -380,8 +376,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto bar_p_full = [&](int s) { return bar0 + 8u * (4 * NST + 3 + s); };
   auto bar_pv_done = [&](int s) { return bar0 + 8u * (4 * NST + 5 + s); };
   const uint32_t bar_drain = bar0 + 8u * (4 * NST + 7);
-  auto bar_p_half = [&](int s) { return bar0 + 8u * (4 * NST + 8 + s); };
-  auto bar_pvh_done = [&](int s) { return bar0 + 8u * (4 * NST + 10 + s); };
 
   volatile int* abort_flag = &s_abort;
   // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
@@ -504,9 +498,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int r = 0; r < rounds0 && ok; ++r) {
         for (int s = 0; s < 2 && ok; ++s) {
           if (r >= rounds[s]) continue;
-          // P arrives in two halves of 64 keys: the first half of P V runs while the softmax
-          // threads are still exponentiating the second
-          ok = mbar_wait(bar_p_half(s), r & 1, abort_flag);
+          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
           if (!ok) break;
           const int i = local_tile(s, r), st = i % NST;
           ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
@@ -514,17 +506,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < BN / 32; ++kk) {
+          for (int kk = 0; kk < BN / 16; ++kk) {
             umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                          (r > 0 || kk > 0) ? 1u : 0u);
-          }
-          umma_commit(bar_pvh_done(s));
-          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int kk = BN / 32; kk < BN / 16; ++kk) {
-            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV, 1u);
           }
           umma_commit(bar_pv_done(s));
           if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
@@ -639,6 +623,76 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
       };
+      // One pass with the reference maximum as it stands: exponentiate, pack P (kept in registers)
+      // and add up the row.  No per-element maximum is tracked (the softmax threads are bound by
+      // instruction issue): a row sum of at most 2^8 proves that no probability exceeded 2^8,
+      // i.e. that the reference is still good.  Otherwise (rare after the first tile; inf or NaN
+      // from an overflow also lands here) the true maximum is taken from the scores - still
+      // intact, because P is stored last - the reference replaced, O rescaled and the tile redone.
+      uint32_t pk[NH * 32];
+      auto row_max = [&]() {
+        float m0 = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          load_half(h);
+#pragma unroll
+          for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
+        }
+        return m0 * p.scale_log2;  // scale > 0; -inf (no allowed key) stays -inf
+      };
+      if (r == 0) m_ref = row_max();  // no reference yet: a cheap extra pass instead of a redo
+      float sum = 0.f;
+      float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      auto exp_pass = [&]() {
+        sum = 0.f;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          load_half(h);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
+          }
+        }
+      };
+      exp_pass();
+      const bool suspect = !(sum <= kRowSumLimit);  // also catches inf and NaN
+      if (__any_sync(0xFFFFFFFFu, suspect)) {
+        const float mx = suspect ? row_max() : m_ref;
+        const bool need = mx > m_ref;
+        if (r > 0) {  // O must be at rest: the previous P V has completed
+          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
+        if (need) { m_ref = mx; l_run *= alpha; }
+        if (r > 0) {
+#pragma unroll 1
+          for (int c = 0; c < HD; c += 32) {
+            uint32_t ov[32];
+            tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+            tmem_st_x32(tmem_O(slot) + lane_addr + c, ov);
+          }
+          tmem_wait_st();
+        }
+        neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+        exp_pass();
+      }
+      // P (the A operand of P V) takes the place of score columns that have been consumed.  The
+      // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
+      tmem_wait_st();
+      l_run += sum;
+
       if (short_tile) {
         // Rows of a V piece beyond its real keys hold whatever lies behind them in memory (or were
         // never loaded); their probabilities are exactly 0, but 0 * NaN would poison O: clear them.
@@ -658,103 +712,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         fence_async_smem();   // cleared V rows visible to the tensor core's reads
       }
-
-      // The row is exponentiated against the reference maximum as it stands, in two halves of 64
-      // keys; P of the first half goes to the tensor core while the second is computed.  No
-      // per-element maximum is tracked (these threads are bound by instruction issue): a row sum
-      // of at most 2^8 proves that no probability exceeded 2^8, i.e. that the reference is still
-      // good.  Otherwise (rare after the first tile; inf or NaN from an overflow also lands here)
-      // the true maximum is taken from the scores, the reference replaced and O rescaled.
-      static_assert(NH == 2, "the row is processed as two 64-column halves");
-      uint32_t pk[32];
-      float sum0 = 0.f, sum1 = 0.f;
-      auto half_max = [&]() {  // maximum of the half that is in sv
-        float m0 = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
-        return m0 * p.scale_log2;  // scale > 0; -inf (no allowed key) stays -inf
-      };
-      auto exp_half = [&](float neg_m) {  // sv -> pk, returns the sum of the 64 probabilities
-        float acc = 0.f;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-          acc += p0 + p1;
-          pk[j] = pack_bf16(p0, p1);
-        }
-        return acc;
-      };
-      auto rescale_o = [&](float alpha) {  // O must be at rest
-#pragma unroll 1
-        for (int c = 0; c < HD; c += 32) {
-          uint32_t ov[32];
-          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-          tmem_st_x32(tmem_O(slot) + lane_addr + c, ov);
-        }
-        tmem_wait_st();
-      };
-      if (r == 0) {  // no reference yet: the first tile's row maximum (a cheap extra pass)
-        load_half(0);
-        const float ma = half_max();
-        load_half(1);
-        m_ref = fmaxf(ma, half_max());
-      }
-      // ---- first half
-      load_half(0);
-      sum0 = exp_half((m_ref == -INFINITY) ? 0.f : -m_ref);
-      const bool suspect0 = !(sum0 <= kRowSumLimit);  // also catches inf and NaN
-      if (__any_sync(0xFFFFFFFFu, suspect0)) {
-        // nothing of this tile has been handed over yet: take the row maximum, move the reference
-        float mx = m_ref;
-        if (suspect0) {
-          mx = half_max();
-          load_half(1);
-          mx = fmaxf(mx, half_max());
-        }
-        if (r > 0) {  // O must be at rest: the previous P V has completed
-          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
-          ok = __all_sync(0xFFFFFFFFu, ok);
-          if (!ok) break;
-          tc_fence_after();
-        }
-        const bool need = mx > m_ref;
-        const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
-        if (need) { m_ref = mx; l_run *= alpha; }
-        if (r > 0) rescale_o(alpha);
-        load_half(0);
-        sum0 = exp_half((m_ref == -INFINITY) ? 0.f : -m_ref);
-      }
-      // P (the A operand of P V) takes the place of score columns that have been consumed.  The
-      // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
-      tmem_st_x32(tmem_P(slot) + lane_addr, pk);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p_half(slot));
-      // ---- second half
-      load_half(1);
-      sum1 = exp_half((m_ref == -INFINITY) ? 0.f : -m_ref);
-      const bool suspect1 = !(sum0 + sum1 <= kRowSumLimit);
-      if (__any_sync(0xFFFFFFFFu, suspect1)) {
-        // The first half is already with the tensor core: wait until that part of P V has landed
-        // in O, then move the reference; what the first half contributed is rescaled with O.
-        const float mx = suspect1 ? fmaxf(m_ref, half_max()) : m_ref;
-        ok = mbar_wait(bar_pvh_done(slot), r & 1, abort_flag);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        tc_fence_after();
-        const bool need = mx > m_ref;
-        const float alpha = need ? ex2(m_ref - mx) : 1.0f;
-        if (need) { m_ref = mx; l_run *= alpha; sum0 *= alpha; }
-        rescale_o(alpha);
-        sum1 = exp_half((m_ref == -INFINITY) ? 0.f : -m_ref);
-      }
-      tmem_st_x32(tmem_P(slot) + lane_addr + 32, pk);
-      tmem_wait_st();
-      l_run += sum0 + sum1;
       tc_fence_before();
       mbar_arrive(bar_p_full(slot));
     }
