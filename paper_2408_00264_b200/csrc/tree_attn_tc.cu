@@ -266,10 +266,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   constexpr int NST = Cfg<MT>::kStages;
   constexpr uint32_t kTile = Cfg<MT>::kTile;
   constexpr uint32_t kHalf = kTile / 2;    // one 64-wide half of the head dimension: [BN keys][64 d]
-  constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);
-  // V buffers are handed back by the softmax threads (one round later, no commit) or by a commit
-  // of the issuer right after the P V that read them
-  constexpr bool kSoftVRelease = (MT == 2);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
+  constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
@@ -491,11 +488,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
           umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
         }
-        // The one commit of the loop.  It completes when everything issued so far has finished:
-        // this Q K^T, the other row tile's Q K^T on the same K buffer, and the P V before them.
-        // The softmax threads that see it hand the K (and the previous V) buffer back themselves:
-        // a commit costs the tensor pipe as much as an MMA.
         umma_commit(bar_s_full(s));
+        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
         return true;
       };
       const int rounds[2] = {rounds0, rounds1};
@@ -516,9 +510,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                          (r > 0 || kk > 0) ? 1u : 0u);
           }
-          if (!kSoftVRelease && (MT == 1 || s == 1)) umma_commit(bar_v_empty(st));  // last reader of this V buffer
+          umma_commit(bar_pv_done(s));
+          if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
           if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
-          else umma_commit(bar_pv_done(s));  // the slot's last P V: O is final when this completes
         }
       }
     }
@@ -593,13 +587,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      // Everything the issuer queued before this tile's commit has completed: the last Q K^T on
-      // this K buffer and the previous round's P V of this slot (so O is at rest while these
-      // threads work on the tile).  The group that reads a buffer last gives it back.
-      if ((MT == 1 || slot == 1) && quarter == 0 && lane == 0) {
-        mbar_arrive(bar_k_empty(st));
-        if (kSoftVRelease && r > 0) mbar_arrive(bar_v_empty(((MT == 2) ? r - 1 : 2 * (r - 1) + slot) % NST));
-      }
       if (p.paged && cache_tile) {
         // the producer's verdict on this tile's pages, written before it armed the V barrier (the
         // V stage is not reused before this tile's P V, so the flag is stable)
@@ -675,6 +662,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (__any_sync(0xFFFFFFFFu, suspect)) {
         const float mx = suspect ? row_max() : m_ref;
         const bool need = mx > m_ref;
+        if (r > 0) {  // O must be at rest: the previous P V has completed
+          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+        }
         const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
         if (need) { m_ref = mx; l_run *= alpha; }
         if (r > 0) {
@@ -724,7 +717,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 
     if (ok && rounds > 0) {  // the last P V of this slot has landed in O
-      ok = mbar_wait(bar_pv_done(slot), 0, abort_flag);
+      ok = mbar_wait(bar_pv_done(slot), (rounds - 1) & 1, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
     }
   }
