@@ -49,9 +49,10 @@ constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: abo
 template <int MT>
 struct Cfg {
   static constexpr int BN = 128;                         // keys per tile
-  static constexpr int kStages = 2;                      // ring depth, K and V each
+  static constexpr int kStagesK = (MT == 1) ? 3 : 2;     // depth of the K ring
+  static constexpr int kStagesV = 2;                     // depth of the V ring
   static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
-  static constexpr uint32_t kSmem = MT * kQTile + kStages * 2 * kTile + 1024;
+  static constexpr uint32_t kSmem = MT * kQTile + (kStagesK + kStagesV) * kTile + 1024;
 };
 
 struct Params {
@@ -263,15 +264,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const __grid_constant__ CUtensorMap tm_vt, const Params p) {
   constexpr int BN = Cfg<MT>::BN;          // keys per tile
   constexpr int PPT = BN / PG;             // 64-key pieces per tile
-  constexpr int NST = Cfg<MT>::kStages;
+  constexpr int KST = Cfg<MT>::kStagesK, VST = Cfg<MT>::kStagesV;
   constexpr uint32_t kTile = Cfg<MT>::kTile;
   constexpr uint32_t kHalf = kTile / 2;    // one 64-wide half of the head dimension: [BN keys][64 d]
   constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
-  __shared__ __align__(8) unsigned long long s_bar[4 * NST + 8];
-  __shared__ int s_tile_ok[Cfg<MT>::kStages];  // paged cache: every page of the tile in this V stage is valid
+  __shared__ __align__(8) unsigned long long s_bar[2 * KST + 2 * VST + 8];
+  __shared__ int s_tile_ok[VST];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
@@ -306,17 +307,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // ---- set-up and per-sequence checks in one go: while thread 0 initialises the barriers and
   //      warp 1 allocates tensor memory, everybody reads parent[] and the context length; the one
   //      block-wide synchronisation below publishes all of it -------------------------------------
-  constexpr int NSTc = Cfg<MT>::kStages;
+  constexpr int NRING = 2 * KST + 2 * VST;
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   if (tid == 0) {
-    for (int i = 0; i < 4 * NSTc; ++i) mbar_init(bar0 + 8u * i, 1);                 // K/V rings
-    mbar_init(bar0 + 8u * (4 * NSTc), 1);                                           // Q
+    for (int i = 0; i < NRING; ++i) mbar_init(bar0 + 8u * i, 1);                 // K/V rings
+    mbar_init(bar0 + 8u * (NRING), 1);                                           // Q
     for (int s2 = 0; s2 < 2; ++s2) {
-      mbar_init(bar0 + 8u * (4 * NSTc + 1 + s2), 1);                                // S ready
-      mbar_init(bar0 + 8u * (4 * NSTc + 3 + s2), BM);                               // P ready
-      mbar_init(bar0 + 8u * (4 * NSTc + 5 + s2), 1);                                // P V done
+      mbar_init(bar0 + 8u * (NRING + 1 + s2), 1);                                // S ready
+      mbar_init(bar0 + 8u * (NRING + 3 + s2), BM);                               // P ready
+      mbar_init(bar0 + 8u * (NRING + 5 + s2), 1);                                // P V done
     }
-    mbar_init(bar0 + 8u * (4 * NSTc + 7), 1);                                       // drain
+    mbar_init(bar0 + 8u * (NRING + 7), 1);                                       // drain
     s_abort = 0;
     fence_barrier_init();
     fence_async_smem();
@@ -363,19 +364,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem_base;
-  const uint32_t sK = sQ + MT * kQTile;      // ring of NST K tiles
-  const uint32_t sV = sK + NST * kTile;      // ring of NST V tiles
+  const uint32_t sK = sQ + MT * kQTile;      // ring of KST K tiles
+  const uint32_t sV = sK + KST * kTile;      // ring of VST V tiles
   uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
 
   auto bar_k_full = [&](int st) { return bar0 + 8u * st; };
-  auto bar_k_empty = [&](int st) { return bar0 + 8u * (NST + st); };
-  auto bar_v_full = [&](int st) { return bar0 + 8u * (2 * NST + st); };
-  auto bar_v_empty = [&](int st) { return bar0 + 8u * (3 * NST + st); };
-  const uint32_t bar_q = bar0 + 8u * (4 * NST);
-  auto bar_s_full = [&](int s) { return bar0 + 8u * (4 * NST + 1 + s); };
-  auto bar_p_full = [&](int s) { return bar0 + 8u * (4 * NST + 3 + s); };
-  auto bar_pv_done = [&](int s) { return bar0 + 8u * (4 * NST + 5 + s); };
-  const uint32_t bar_drain = bar0 + 8u * (4 * NST + 7);
+  auto bar_k_empty = [&](int st) { return bar0 + 8u * (KST + st); };
+  auto bar_v_full = [&](int st) { return bar0 + 8u * (2 * KST + st); };
+  auto bar_v_empty = [&](int st) { return bar0 + 8u * (2 * KST + VST + st); };
+  const uint32_t bar_q = bar0 + 8u * NRING;
+  auto bar_s_full = [&](int s) { return bar0 + 8u * (NRING + 1 + s); };
+  auto bar_p_full = [&](int s) { return bar0 + 8u * (NRING + 3 + s); };
+  auto bar_pv_done = [&](int s) { return bar0 + 8u * (NRING + 5 + s); };
+  const uint32_t bar_drain = bar0 + 8u * (NRING + 7);
 
   volatile int* abort_flag = &s_abort;
   // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
@@ -384,7 +385,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto tmem_P = [&](int s) { return tmem + (uint32_t)(s * BN); };
   auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + s * HD); };
 
-  int issued_tiles = 0;  // producer bookkeeping for the drain
+  int issued_k = 0, issued_v = 0;  // producer bookkeeping for the drain
 
   // per-thread state of the softmax groups (warps 2..9); declared here because the epilogue runs
   // after block-wide synchronisation points that all roles must reach together
@@ -406,7 +407,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       int page_base = -64;
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
-        const int st = i % NST;
+        const int ks = i % KST, vs = i % VST;
         const int g0 = pc_begin + i * PPT;  // first piece of this tile
         if (p.paged && g0 < p_cache && g0 + PPT > page_base + 32) {  // warp-uniform refill
           page_base = g0;
@@ -437,29 +438,30 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
           const uint32_t bytes = (uint32_t)n_pieces * 2u * kPiece;  // both halves of the head dim
-          if (i >= NST) ok = mbar_wait(bar_k_empty(st), ((i / NST) - 1) & 1, abort_flag);
+          if (i >= KST) ok = mbar_wait(bar_k_empty(ks), ((i / KST) - 1) & 1, abort_flag);
           if (ok) {
-            mbar_expect_tx(bar_k_full(st), bytes);
+            mbar_expect_tx(bar_k_full(ks), bytes);
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
               const CUtensorMap* mk = is_tree[j] ? &tm_kt : &tm_kc;
-              tma_load_3d(sK + st * kTile + j * kPiece, mk, 0, kvh, row0[j], bar_k_full(st));
-              tma_load_3d(sK + st * kTile + kHalf + j * kPiece, mk, 64, kvh, row0[j], bar_k_full(st));
+              tma_load_3d(sK + ks * kTile + j * kPiece, mk, 0, kvh, row0[j], bar_k_full(ks));
+              tma_load_3d(sK + ks * kTile + kHalf + j * kPiece, mk, 64, kvh, row0[j], bar_k_full(ks));
             }
-            if (i >= NST) ok = mbar_wait(bar_v_empty(st), ((i / NST) - 1) & 1, abort_flag);
+            issued_k = i + 1;
+            if (i >= VST) ok = mbar_wait(bar_v_empty(vs), ((i / VST) - 1) & 1, abort_flag);
           }
           if (ok) {
-            s_tile_ok[st] = tile_ok;  // read by the softmax threads after this V barrier completes
-            mbar_expect_tx(bar_v_full(st), bytes);
+            s_tile_ok[vs] = tile_ok;  // read by the softmax threads after this V barrier completes
+            mbar_expect_tx(bar_v_full(vs), bytes);
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
               const CUtensorMap* mv = is_tree[j] ? &tm_vt : &tm_vc;
-              tma_load_3d(sV + st * kTile + j * kPiece, mv, 0, kvh, row0[j], bar_v_full(st));
-              tma_load_3d(sV + st * kTile + kHalf + j * kPiece, mv, 64, kvh, row0[j], bar_v_full(st));
+              tma_load_3d(sV + vs * kTile + j * kPiece, mv, 0, kvh, row0[j], bar_v_full(vs));
+              tma_load_3d(sV + vs * kTile + kHalf + j * kPiece, mv, 64, kvh, row0[j], bar_v_full(vs));
             }
-            issued_tiles = i + 1;
+            issued_v = i + 1;
           }
         }
         ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
@@ -477,8 +479,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint64_t k_desc = smem_desc(sK, 16, 1024);
       const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
       auto issue_qk = [&](int s, int r) -> bool {
-        const int i = local_tile(s, r), st = i % NST;
-        if (!mbar_wait(bar_k_full(st), (i / NST) & 1, abort_flag)) return false;
+        const int i = local_tile(s, r), st = i % KST;
+        if (!mbar_wait(bar_k_full(st), (i / KST) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
@@ -500,8 +502,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (r >= rounds[s]) continue;
           ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
           if (!ok) break;
-          const int i = local_tile(s, r), st = i % NST;
-          ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+          const int i = local_tile(s, r), st = i % VST;
+          ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
@@ -559,7 +561,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     for (int r = 0; r < rounds && ok; ++r) {
       const int i = (MT == 2) ? r : 2 * r + slot;
-      const int st = i % NST;
+      const int st = i % VST;   // these threads only touch the V ring
       // allowed columns of this row in this tile (64 per piece), and how many rows of each V
       // piece are real keys
       uint32_t allow[BN / 32];
@@ -590,7 +592,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (p.paged && cache_tile) {
         // the producer's verdict on this tile's pages, written before it armed the V barrier (the
         // V stage is not reused before this tile's P V, so the flag is stable)
-        ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         if (!*(volatile int*)&s_tile_ok[st]) {  // sequence is flagged; hide the whole tile
@@ -696,7 +698,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (short_tile) {
         // Rows of a V piece beyond its real keys hold whatever lies behind them in memory (or were
         // never loaded); their probabilities are exactly 0, but 0 * NaN would poison O: clear them.
-        ok = mbar_wait(bar_v_full(st), (i / NST) & 1, abort_flag);
+        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         uint8_t* vt = sV_gen + st * kTile;
@@ -727,10 +729,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (*abort_flag) {
     if (warp == 0 && lane == 0) {
       // TMA copies that were issued land on their own; wait for the newest phase of each stage
-      for (int i = max(0, issued_tiles - NST); i < issued_tiles; ++i) {
-        mbar_drain(bar_k_full(i % NST), (i / NST) & 1);
-        mbar_drain(bar_v_full(i % NST), (i / NST) & 1);
-      }
+      for (int i = max(0, issued_k - KST); i < issued_k; ++i) mbar_drain(bar_k_full(i % KST), (i / KST) & 1);
+      for (int i = max(0, issued_v - VST); i < issued_v; ++i) mbar_drain(bar_v_full(i % VST), (i / VST) & 1);
       if (n_tiles > 0) mbar_drain(bar_q, 0);
     }
     if (warp == 1 && lane == 0) {
