@@ -218,7 +218,7 @@ def run_clv(args):
 
     # ---- whole step, inputs resident -------------------------------------------------------
     for i in range(max(args.warmup, 3)):
-        sets[i % ROTATE].run(overlap=not args.no_overlap)
+        sets[i % ROTATE].run()
     torch.cuda.synchronize()
     graphs = None
     if not args.no_graph:
@@ -226,7 +226,7 @@ def run_clv(args):
         for s in sets:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                s.run(overlap=not args.no_overlap)
+                s.run()
             graphs.append(g)
         for i in range(max(args.warmup, 3)):
             graphs[i % ROTATE].replay()
@@ -240,7 +240,7 @@ def run_clv(args):
                 graphs[i % ROTATE].replay()
         else:
             for i in range(args.steps):
-                sets[i % ROTATE].run(overlap=not args.no_overlap)
+                sets[i % ROTATE].run()
         e1.record(stream)
         barrier()
     step_ms = e0.elapsed_time(e1) / args.steps
@@ -335,8 +335,6 @@ def run_clv(args):
         "frac_of_hbm_peak": {"of_%s_%.0f_GBps" % (peak_kind, peak): value / world / peak,
                              "of_nominal_8000_GBps": value / world / NOMINAL_HBM_GBS},
         "call_us": call_us, "launch_mode": "per-call" if graphs is None else "cuda-graph replay",
-        "step_schedule": ("tree_attn, accept_argmax, accept_walk, kv_commit on one stream" if args.no_overlap
-                          else "accept_argmax on a second stream beside tree_attn, joined before accept_walk, kv_commit"),
         "algorithmic_bytes": nbytes,
         "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak,
                      "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
@@ -366,8 +364,6 @@ def main():
     ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--impl", default="clv", choices=["clv", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch the four calls per step directly")
-    ap.add_argument("--no-overlap", action="store_true",
-                    help="run the argmax after the attention on one stream instead of beside it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiling runs)")
     args = ap.parse_args()

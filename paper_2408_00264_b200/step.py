@@ -19,12 +19,8 @@ def bits_of(t: torch.Tensor) -> np.ndarray:
 
 
 class VerifyStep:
-    """Holds the inputs of a workload on one GPU plus every output buffer, and runs the four calls
-    of a verify step.  clv_tree_attn and clv_accept_argmax read disjoint inputs and write disjoint
-    outputs, so `run` launches the argmax on a second stream beside the attention (each with a
-    workspace of its own) and joins before clv_accept_walk -> clv_kv_commit; the attention
-    leaves most of the HBM bandwidth unused and the argmax is a pure stream, so the two overlap
-    almost completely.  The fork and join are events, so the step can be captured in a CUDA graph.
+    """Holds the inputs of a workload on one GPU plus every output buffer, and runs
+    clv_tree_attn -> clv_accept_argmax -> clv_accept_walk -> clv_kv_commit on the current stream.
     """
 
     def __init__(self, w, device="cuda", with_lse: bool = True, logits: bool = True):
@@ -49,9 +45,6 @@ class VerifyStep:
         self.shape = clv.make_shape(B, N, c.n_q_heads, c.n_kv_heads, c.vocab, w.path_cap)
         self.cache = clv.make_cache(self.k_cache, self.v_cache, self.block_table)
         self.workspace = clv.new_workspace(self.shape, self.cache, self.max_ctx_len, device)
-        # the argmax gets its own arrival counters and scratch: it may run beside the attention
-        self.workspace_argmax = clv.new_workspace(self.shape, self.cache, self.max_ctx_len, device)
-        self._side = None   # second stream and fork/join events, created on first use
         i32 = dict(dtype=torch.int32, device=device)
         self.out = torch.empty_like(self.q)
         self.lse = torch.empty(B, N, c.n_q_heads, dtype=torch.float32, device=device) if with_lse else None
@@ -68,8 +61,7 @@ class VerifyStep:
                           self.status[0], self.workspace, stream)
 
     def accept_argmax(self, stream=None):
-        clv.clv_accept_argmax(self.shape, self.logits, self.ld, self.ids, self.workspace_argmax,
-                              stream)
+        clv.clv_accept_argmax(self.shape, self.logits, self.ld, self.ids, self.workspace, stream)
 
     def accept_walk(self, stream=None):
         clv.clv_accept_walk(self.shape, self.parent, self.tokens, self.ids, self.accept_len,
@@ -81,24 +73,9 @@ class VerifyStep:
                           self.ctx_len_out if ctx_len_out is None else ctx_len_out,
                           self.status[2], stream)
 
-    def run(self, stream=None, overlap: bool = True):
-        """One whole verify step (four launches).  With `overlap` the argmax runs on a second
-        stream beside the attention; the walk and the commit follow on `stream` after both."""
-        main = torch.cuda.current_stream(self.device) if stream is None else stream
-        if overlap:
-            if self._side is None:
-                self._side = (torch.cuda.Stream(self.device), torch.cuda.Event(), torch.cuda.Event())
-            side, fork, join = self._side
-            fork.record(main)
-            side.wait_event(fork)
-            # the attention first: its blocks need a whole SM's shared memory each, the argmax
-            # blocks then settle beside them
-            self.tree_attn(main)
-            self.accept_argmax(side)
-            join.record(side)
-            main.wait_event(join)
-        else:
-            self.tree_attn(main)
-            self.accept_argmax(main)
-        self.accept_walk(main)
-        self.kv_commit(main)
+    def run(self, stream=None):
+        """One whole verify step (four launches, stream-ordered)."""
+        self.tree_attn(stream)
+        self.accept_argmax(stream)
+        self.accept_walk(stream)
+        self.kv_commit(stream)
