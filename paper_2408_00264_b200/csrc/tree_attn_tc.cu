@@ -480,8 +480,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
       auto issue_qk = [&](int s, int r) -> bool {
         const int i = local_tile(s, r), st = i % KST;
-        if (!mbar_wait(bar_k_full(st), (i / KST) & 1, abort_flag)) return false;
-        tc_fence_after();
+        // with two row tiles, slot 1 uses the K tile that slot 0 has just waited for
+        if (MT == 1 || s == 0) {
+          if (!mbar_wait(bar_k_full(st), (i / KST) & 1, abort_flag)) return false;
+          tc_fence_after();
+        }
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
@@ -503,8 +506,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
           if (!ok) break;
           const int i = local_tile(s, r), st = i % VST;
-          ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
-          if (!ok) break;
+          if (MT == 1 || s == 0) {  // likewise the V tile
+            ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
+            if (!ok) break;
+          }
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
