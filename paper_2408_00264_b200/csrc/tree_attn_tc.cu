@@ -94,10 +94,22 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // never suspends
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
 // try_wait itself suspends the thread for a hardware-bounded time, so the first polls need no
 // clock; after that the SM clock (cheap to read, unlike the global timer) bounds the wait.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_test(bar, parity)) return true;  // the common case in steady state: already complete
 #pragma unroll 1
   for (int spin = 0; spin < 32; ++spin)
     if (mbar_try(bar, parity)) return true;
