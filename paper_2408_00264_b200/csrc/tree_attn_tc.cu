@@ -26,6 +26,7 @@
 // CLV_ERR_TIMEOUT is reported for the sequence.
 #include <cooperative_groups.h>
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <math.h>
 
 #include "clv_internal.cuh"
@@ -209,11 +210,6 @@ __device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
                : "r"(addr));
   return v;
 }
-__device__ __forceinline__ float2 dsmem_ld8(uint32_t addr) {
-  float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
-  return v;
-}
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -225,26 +221,37 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ uint2 dsmem_ld8u(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared::cluster.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 half2_bits_to_float2(uint32_t u) {
+  return __half22float2(*reinterpret_cast<const __half2*>(&u));
+}
+
 // Final combination of NSRC accumulators per output row, for the rows [k_begin, k_end) that this
-// block finalises.  One warp takes 16 / NSRC rows at a time (16 remote 16-byte loads in flight
-// per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the normalised weights.
+// block finalises.  The staged accumulators are fp16 (each row scaled by a power of two of its
+// own, which the weight undoes), 256 bytes per row.  One warp takes 32 / NSRC rows at a time (32
+// remote 8-byte loads in flight per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the
+// normalised weights divided by the rows' scales.
 template <int NSRC, int MT>
 __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
                                            int rot, int warp, int lane, int tile_base, int rows_total, int G,
                                            int64_t seq_row0, int Hq, int head0, uint16_t* out) {
-  constexpr int RB = 16 / NSRC;
+  constexpr int RB = 32 / NSRC;
   for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
-    float4 x[RB * NSRC];
+    uint2 x[RB * NSRC];
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
       const int k = min(k0 + u, per_rank - 1);
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const uint32_t off = (uint32_t)(trow * HD + ((lane ^ (trow & 31)) << 2)) * 4u;
+      const uint32_t off = (uint32_t)(trow * (HD * 2) + (((lane >> 1) ^ (trow & 15)) << 4) + ((lane & 1) << 3));
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
         const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
         const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-        x[u * NSRC + j] = dsmem_ld16(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 4) + off, qc));
+        x[u * NSRC + j] = dsmem_ld8u(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 2) + off, qc));
       }
     }
 #pragma unroll
@@ -258,8 +265,8 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
         const float wq = w[k * NSRC + ((j + rot) & (NSRC - 1))];
-        const float4 v = x[u * NSRC + j];
-        acc.x += wq * v.x; acc.y += wq * v.y; acc.z += wq * v.z; acc.w += wq * v.w;
+        const float2 lo = half2_bits_to_float2(x[u * NSRC + j].x), hi = half2_bits_to_float2(x[u * NSRC + j].y);
+        acc.x += wq * lo.x; acc.y += wq * lo.y; acc.z += wq * hi.x; acc.w += wq * hi.y;
       }
       const int onode = rg / G, ogq = rg - onode * G;
       uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
@@ -287,7 +294,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ int s_tile_ok[VST];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ float2 s_ml[2][BM];   // (reference maximum, row sum) of both slots, for the merge
+  __shared__ float4 s_ml[2][BM];   // (reference maximum, row sum, 1 / staging scale, -) of both slots, for the merge
   __shared__ float s_w[2 * BM];    // merge: normalised weight of every (row of this rank, source)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -761,10 +768,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const bool aborted = *abort_flag != 0;
   const int n_src = p.splits * (MT == 1 ? 2 : 1);  // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
-  // staging area for the merge: O of both slots as fp32 [slot][128 rows][128], 16-byte chunk c of
-  // row r stored at chunk (c ^ (r & 31)) so that row-per-thread writes and row-per-warp reads are
-  // both conflict free.  It reuses the tile memory, which nothing reads any more.
-  float* const sO = reinterpret_cast<float*>(smem_raw + (sQ - smem_u32(smem_raw)));
+  // staging area for the merge: O of both slots as fp16 [slot][128 rows][128], every row scaled by
+  // a power of two that puts its largest magnitude in [2^13, 2^14) (half the bytes of fp32 through
+  // distributed shared memory, at a relative rounding error of 2^-11, far below that of the bf16
+  // output; the scale travels with the row's maximum and sum).  The 16-byte chunk c of row r is
+  // stored at chunk (c ^ (r & 15)) so that row-per-thread writes and row-per-warp reads are both
+  // conflict free.  The area reuses the tile memory, which nothing reads any more.
+  uint8_t* const sO = smem_raw + (sQ - smem_u32(smem_raw));
 
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
@@ -791,7 +801,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (p.lse != nullptr && row_valid)
         p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
     } else {
-      float* orow = sO + ((size_t)slot * BM + row) * HD;
+      uint8_t* orow = sO + ((size_t)slot * BM + row) * (HD * 2);
+      // first pass: the row's largest magnitude, which fixes its scale
+      float amax = 0.f;
+      if (my_rounds > 0) {
+#pragma unroll 1
+        for (int c = 0; c < HD; c += 32) {
+          uint32_t ov[32];
+          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(__uint_as_float(ov[j])));
+        }
+      }
+      // scale 2^lc with amax * 2^lc in [2^13, 2^14); lc is clamped so that the scale and its
+      // inverse are normal numbers (a zero row keeps zeros, inf or NaN stay what they are)
+      const int biased = (int)((__float_as_uint(amax) >> 23) & 255u);
+      const int lc = max(-100, min(100, 140 - biased));
+      const float cscale = __uint_as_float((uint32_t)(127 + lc) << 23);
+      const float cinv = __uint_as_float((uint32_t)(127 - lc) << 23);
 #pragma unroll 1
       for (int c = 0; c < HD; c += 32) {
         uint32_t ov[32];
@@ -803,13 +831,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int j = 0; j < 32; ++j) ov[j] = 0u;
         }
 #pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) {
-          const int chunk = (c >> 2) + q4;
-          *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 31)) << 2)) =
-              make_uint4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]);
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t h[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const __half2 v = __floats2half2_rn(__uint_as_float(ov[q4 * 8 + 2 * e]) * cscale,
+                                                __uint_as_float(ov[q4 * 8 + 2 * e + 1]) * cscale);
+            h[e] = *reinterpret_cast<const uint32_t*>(&v);
+          }
+          const int chunk = (c >> 3) + q4;
+          *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 15)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
         }
       }
-      s_ml[slot][row] = make_float2(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f);
+      s_ml[slot][row] = make_float4(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f, cinv, 0.f);
     }
   }
   tc_fence_before();
@@ -833,14 +867,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int k = tid / n_src, q = tid - k * n_src;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
       const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-      const float2 ml = dsmem_ld8(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
+      const float4 ml = dsmem_ld16(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
       const float wgt = (ml.y > 0.f) ? ex2(ml.x - mu) : 0.f;
       float lsum = wgt * ml.y;
       for (int o = 1; o < n_src; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
-      s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f);
+      s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
       const int rg = (row_cta * MT + tile) * BM + trow;
       if (q == 0 && p.lse != nullptr && rg < rows_total) {
         const int onode = rg / G, ogq = rg - onode * G;
