@@ -225,51 +225,47 @@ __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t u) {
   return __half22float2(*reinterpret_cast<const __half2*>(&u));
 }
 
-// Final combination of NSRC accumulators per output row, for the per_rank rows that this block
-// finalises.  The accumulators are fp16 rows of 256 bytes (each scaled by a power of two of its
-// own, which the weight undoes): this block's own in its staging area, the peers' in the receive
-// area ([source][row of this rank]), where their bulk copies put them.  One warp takes 32 / NSRC
-// rows at a time; lane j owns output columns 4j .. 4j+3.  w[] holds the normalised weights
-// divided by the rows' scales.
-template <int NSRC, int MT>
-__device__ __forceinline__ void merge_rows(const uint8_t* stage, const uint8_t* recv, const float* w,
+// Final combination of the n_src accumulators of every output row that this block finalises.
+// The accumulators are fp16 rows of 256 bytes (each scaled by a power of two of its own, which the
+// weight undoes): this block's own in its staging area, the peers' in the receive area
+// ([source][row of this rank]), where their bulk copies put them.  A half-warp takes one row, a
+// lane 8 of its columns.  The loops are kept rolled on purpose: this code runs once per block, so
+// its cost is the instruction fetch, not the arithmetic.  w[] holds the normalised weights divided
+// by the rows' scales.
+template <int MT>
+__device__ __forceinline__ void merge_rows(const uint8_t* stage, const uint8_t* recv, const float* w, int n_src,
                                            int split, int first_row, int per_rank, int warp, int lane,
                                            int tile_base, int rows_total, int G, int64_t seq_row0, int Hq,
                                            int head0, uint16_t* out) {
-  constexpr int RB = 32 / NSRC;
-  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
-    uint2 x[RB * NSRC];
+  const int hl = lane & 15;
+#pragma unroll 1
+  for (int k = warp * 2 + (lane >> 4); k < per_rank; k += 2 * (kThreads / 32)) {
+    const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+    const int rg = (tile_base + tile) * BM + trow;
+    if (rg >= rows_total) continue;
+    const uint32_t off = (uint32_t)((hl ^ (trow & 15)) << 4);
+    float acc[8];
 #pragma unroll
-    for (int u = 0; u < RB; ++u) {
-      const int k = min(k0 + u, per_rank - 1);
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const uint32_t off = (uint32_t)((((lane >> 1) ^ (trow & 15)) << 4) + ((lane & 1) << 3));
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll 2
+    for (int j = 0; j < n_src; ++j) {
+      const int qc = (MT == 2) ? j : j >> 1, qs = (MT == 2) ? tile : j & 1;
+      const uint8_t* src = (qc == split) ? stage + (size_t)(qs * BM + trow) * (HD * 2)
+                                         : recv + (size_t)(j * per_rank + k) * (HD * 2);
+      const uint4 x = *reinterpret_cast<const uint4*>(src + off);
+      const float wq = w[k * n_src + j];
+      const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-      for (int j = 0; j < NSRC; ++j) {
-        const int qc = (MT == 2) ? j : j >> 1, qs = (MT == 2) ? tile : j & 1;
-        const uint8_t* src = (qc == split) ? stage + (size_t)(qs * BM + trow) * (HD * 2)
-                                           : recv + (size_t)(j * per_rank + k) * (HD * 2);
-        x[u * NSRC + j] = *reinterpret_cast<const uint2*>(src + off);
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = half2_bits_to_float2(xs[e]);
+        acc[2 * e] += wq * f.x;
+        acc[2 * e + 1] += wq * f.y;
       }
     }
-#pragma unroll
-    for (int u = 0; u < RB; ++u) {
-      if (k0 + u >= per_rank) continue;
-      const int k = k0 + u;
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const int rg = (tile_base + tile) * BM + trow;
-      if (rg >= rows_total) continue;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int j = 0; j < NSRC; ++j) {
-        const float wq = w[k * NSRC + j];
-        const float2 lo = half2_bits_to_float2(x[u * NSRC + j].x), hi = half2_bits_to_float2(x[u * NSRC + j].y);
-        acc.x += wq * lo.x; acc.y += wq * lo.y; acc.z += wq * hi.x; acc.w += wq * hi.y;
-      }
-      const int onode = rg / G, ogq = rg - onode * G;
-      uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
-      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-    }
+    const int onode = rg / G, ogq = rg - onode * G;
+    uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + hl * 8;
+    *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]),
+                                                pack_bf16(acc[4], acc[5]), pack_bf16(acc[6], acc[7]));
   }
 }
 
@@ -920,12 +916,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // (b) weighted sums, rows spread over the warps
     uint16_t* outp = p.out;
     const int64_t seq_row0 = (int64_t)b * N;
-    switch (n_src) {
-      case 2: merge_rows<2, MT>(sO, sRecv, s_w, split, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 4: merge_rows<4, MT>(sO, sRecv, s_w, split, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 8: merge_rows<8, MT>(sO, sRecv, s_w, split, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      default: merge_rows<16, MT>(sO, sRecv, s_w, split, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-    }
+    merge_rows<MT>(sO, sRecv, s_w, n_src, split, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G,
+                   seq_row0, p.Hq, kvh * G, outp);
   }
   // Nobody leaves before every block has received its rows: a block's staging area is the source
   // of copies that complete on the peers' barriers.
