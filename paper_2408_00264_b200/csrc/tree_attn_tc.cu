@@ -196,19 +196,19 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
 
 // Distributed shared memory: address of the same variable in block `rank` of the cluster, and a
-// bulk copy from this block's shared memory into a peer's, which counts its bytes on a barrier of
-// the peer (both destination addresses are cluster addresses of the same block).
+// 16-byte load from it.  The loads are volatile asm so that a batch of them is issued back to back
+// (all in flight together) before the first result is used.
 __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void dsmem_push(uint32_t dst_cluster, uint32_t src_local, uint32_t bytes,
-                                           uint32_t bar_cluster) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(dst_cluster), "r"(src_local), "r"(bytes), "r"(bar_cluster)
-      : "memory");
+__device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
+  return v;
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -221,51 +221,57 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ uint2 dsmem_ld8u(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared::cluster.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t u) {
   return __half22float2(*reinterpret_cast<const __half2*>(&u));
 }
 
-// Final combination of the n_src accumulators of every output row that this block finalises.
-// The accumulators are fp16 rows of 256 bytes (each scaled by a power of two of its own, which the
-// weight undoes): this block's own in its staging area, the peers' in the receive area
-// ([source][row of this rank]), where their bulk copies put them.  A half-warp takes one row, a
-// lane 8 of its columns.  The loops are kept rolled on purpose: this code runs once per block, so
-// its cost is the instruction fetch, not the arithmetic.  w[] holds the normalised weights divided
-// by the rows' scales.
-template <int MT>
-__device__ __forceinline__ void merge_rows(const uint8_t* stage, const uint8_t* recv, const float* w, int n_src,
-                                           int split, int first_row, int per_rank, int warp, int lane,
-                                           int tile_base, int rows_total, int G, int64_t seq_row0, int Hq,
-                                           int head0, uint16_t* out) {
-  const int hl = lane & 15;
-#pragma unroll 1
-  for (int k = warp * 2 + (lane >> 4); k < per_rank; k += 2 * (kThreads / 32)) {
-    const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-    const int rg = (tile_base + tile) * BM + trow;
-    if (rg >= rows_total) continue;
-    const uint32_t off = (uint32_t)((hl ^ (trow & 15)) << 4);
-    float acc[8];
+// Final combination of NSRC accumulators per output row, for the rows [k_begin, k_end) that this
+// block finalises.  The staged accumulators are fp16 (each row scaled by a power of two of its
+// own, which the weight undoes), 256 bytes per row.  One warp takes 32 / NSRC rows at a time (32
+// remote 8-byte loads in flight per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the
+// normalised weights divided by the rows' scales.
+template <int NSRC, int MT>
+__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
+                                           int rot, int warp, int lane, int tile_base, int rows_total, int G,
+                                           int64_t seq_row0, int Hq, int head0, uint16_t* out) {
+  constexpr int RB = 32 / NSRC;
+  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
+    uint2 x[RB * NSRC];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#pragma unroll 2
-    for (int j = 0; j < n_src; ++j) {
-      const int qc = (MT == 2) ? j : j >> 1, qs = (MT == 2) ? tile : j & 1;
-      const uint8_t* src = (qc == split) ? stage + (size_t)(qs * BM + trow) * (HD * 2)
-                                         : recv + (size_t)(j * per_rank + k) * (HD * 2);
-      const uint4 x = *reinterpret_cast<const uint4*>(src + off);
-      const float wq = w[k * n_src + j];
-      const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+    for (int u = 0; u < RB; ++u) {
+      const int k = min(k0 + u, per_rank - 1);
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const uint32_t off = (uint32_t)(trow * (HD * 2) + (((lane >> 1) ^ (trow & 15)) << 4) + ((lane & 1) << 3));
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = half2_bits_to_float2(xs[e]);
-        acc[2 * e] += wq * f.x;
-        acc[2 * e + 1] += wq * f.y;
+      for (int j = 0; j < NSRC; ++j) {
+        const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
+        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
+        x[u * NSRC + j] = dsmem_ld8u(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 2) + off, qc));
       }
     }
-    const int onode = rg / G, ogq = rg - onode * G;
-    uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + hl * 8;
-    *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]),
-                                                pack_bf16(acc[4], acc[5]), pack_bf16(acc[6], acc[7]));
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      if (k0 + u >= per_rank) continue;
+      const int k = k0 + u;
+      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const int rg = (tile_base + tile) * BM + trow;
+      if (rg >= rows_total) continue;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < NSRC; ++j) {
+        const float wq = w[k * NSRC + ((j + rot) & (NSRC - 1))];
+        const float2 lo = half2_bits_to_float2(x[u * NSRC + j].x), hi = half2_bits_to_float2(x[u * NSRC + j].y);
+        acc.x += wq * lo.x; acc.y += wq * lo.y; acc.z += wq * hi.x; acc.w += wq * hi.y;
+      }
+      const int onode = rg / G, ogq = rg - onode * G;
+      uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+    }
   }
 }
 
@@ -284,7 +290,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
-  __shared__ __align__(8) unsigned long long s_bar[2 * KST + 2 * VST + 9];
+  __shared__ __align__(8) unsigned long long s_bar[2 * KST + 2 * VST + 8];
   __shared__ int s_tile_ok[VST];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -331,7 +337,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_init(bar0 + 8u * (NRING + 5 + s2), 1);                                // P V done
     }
     mbar_init(bar0 + 8u * (NRING + 7), 1);                                       // drain
-    mbar_init(bar0 + 8u * (NRING + 8), 1);                                       // merge: peers' rows received
     s_abort = 0;
     fence_barrier_init();
     fence_async_smem();
@@ -391,7 +396,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto bar_p_full = [&](int s) { return bar0 + 8u * (NRING + 3 + s); };
   auto bar_pv_done = [&](int s) { return bar0 + 8u * (NRING + 5 + s); };
   const uint32_t bar_drain = bar0 + 8u * (NRING + 7);
-  const uint32_t bar_recv = bar0 + 8u * (NRING + 8);
 
   volatile int* abort_flag = &s_abort;
   // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
@@ -769,14 +773,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // distributed shared memory, at a relative rounding error of 2^-11, far below that of the bf16
   // output; the scale travels with the row's maximum and sum).  The 16-byte chunk c of row r is
   // stored at chunk (c ^ (r & 15)) so that row-per-thread writes and row-per-warp reads are both
-  // conflict free.  The area reuses the tile memory, which nothing reads any more; behind it lie
-  // the receive areas for the peers' rows and their (maximum, sum, scale) records.
+  // conflict free.  The area reuses the tile memory, which nothing reads any more.
   uint8_t* const sO = smem_raw + (sQ - smem_u32(smem_raw));
-  constexpr uint32_t kStageBytes = 2 * BM * HD * 2;          // 64 KB: both slots
-  constexpr uint32_t kRecvBytes = 2 * BM * HD * 2;           // n_src * per_rank = 256 rows whatever the split
-  uint8_t* const sRecv = sO + kStageBytes;
-  float4* const sRecvMl = reinterpret_cast<float4*>(sRecv + kRecvBytes);   // 256 records
-  static_assert(kStageBytes + kRecvBytes + 2 * BM * 16 <= Cfg<MT>::kSmem - 1024, "merge areas exceed the tile memory");
 
   if (!aborted && warp >= 2) {
     if (n_src == 1) {
@@ -846,7 +844,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
       s_ml[slot][row] = make_float4(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f, cinv, 0.f);
-      fence_async_smem();  // the staged rows are read by bulk copies
     }
   }
   tc_fence_before();
@@ -855,50 +852,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (aborted && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
   if (n_src == 1) return;  // such a block is its own cluster
 
-  // ---- merge across the cluster (the split-KV blocks of one row tile): rank j finalises rows
-  //      [j, j+1) * rows/splits of the tile(s).  Once every block has staged its accumulators,
-  //      each pushes the rows the others finalise into their receive areas with bulk copies
-  //      through distributed shared memory (a handful of copies of 4 to 32 KB per block; pulling
-  //      the same rows with loads was bound by the number of remote requests, not by bytes) ------
+  // ---- merge across the cluster (the split-KV blocks of one row tile) through distributed
+  //      shared memory: rank j finalises rows [j, j+1) * rows/splits of the tile(s) ------------
   cg::cluster_group cluster = cg::this_cluster();
-  constexpr int kSlotsPerBlock = (MT == 1) ? 2 : 1;   // sources that one block contributes to a row
-  const int per_rank = MT * BM / p.splits;            // rows each rank finalises; per_rank * n_src = 256
-  const int first_row = split * per_rank;
-  if (tid == 0)  // bytes this block will receive: rows and records from every other block
-    mbar_expect_tx(bar_recv, (uint32_t)((p.splits - 1) * kSlotsPerBlock * per_rank * (HD * 2 + 16)));
-  cluster.sync();  // every block's staging area is complete and its tile memory idle (also reached by
-                   // an aborted block, which pushes whatever it has so that nobody waits for it)
-  if (tid == 0) {
-    const uint32_t stage_addr = smem_u32(sO), recv_addr = smem_u32(sRecv), recvml_addr = smem_u32(sRecvMl);
-    for (int d = 1; d < p.splits; ++d) {
-      const int peer = (split + d) % p.splits;          // every block starts with a different peer
-      const uint32_t peer_bar = dsmem_addr(bar_recv, peer);
-#pragma unroll
-      for (int sl = 0; sl < kSlotsPerBlock; ++sl) {
-        // rows of `peer` in my staging area; my source number at the peer
-        const int src_row = (MT == 2) ? peer * per_rank : sl * BM + peer * per_rank;
-        const int j = split * kSlotsPerBlock + sl;
-        dsmem_push(dsmem_addr(recv_addr + (uint32_t)(j * per_rank) * (HD * 2), peer),
-                   stage_addr + (uint32_t)src_row * (HD * 2), (uint32_t)per_rank * (HD * 2), peer_bar);
-        dsmem_push(dsmem_addr(recvml_addr + (uint32_t)(j * per_rank) * 16u, peer),
-                   smem_u32(&s_ml[0][0]) + (uint32_t)src_row * 16u, (uint32_t)per_rank * 16u, peer_bar);
-      }
-    }
-  }
-  bool got = false;
-  if (aborted) mbar_drain(bar_recv, 0);  // result unused, but no copy may still be on its way in
-  else got = mbar_wait(bar_recv, 0, abort_flag);
-  got = __syncthreads_and(got ? 1 : 0) != 0;
-  if (!aborted && !got && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
-  if (got) {
-    // (a) thread (k, q) takes the (maximum, sum, scale) record of source q of row k; the n_src
-    //     lanes of a row sit side by side in one warp, so the normalised weights come from shuffles.
+  cluster.sync();  // every block's staging area is complete (also reached by an aborted block)
+  if (!aborted) {
+    // Every rank finalises per_rank rows; per_rank * n_src is 256 whatever the split count.
+    const int per_rank = MT * BM / p.splits;
+    const int first_row = split * per_rank;
+    // (a) thread (k, q) fetches the (maximum, sum) pair of source q of row k; the n_src lanes of a
+    //     row sit side by side in one warp, so the normalised weights come from shuffles.
     //     Source q is (block q, slot `tile`) when MT == 2 and (block q / 2, slot q % 2) when MT == 1.
     if (tid < 2 * BM) {
       const int k = tid / n_src, q = tid - k * n_src;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
       const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-      const float4 ml = (qc == split) ? s_ml[qs][trow] : sRecvMl[q * per_rank + k];
+      const float4 ml = dsmem_ld16(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
@@ -914,14 +883,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
     __syncthreads();
     // (b) weighted sums, rows spread over the warps
+    const uint32_t sO_addr = smem_u32(sO);
+    const int rot = (split + 1) * (MT == 1 ? 2 : 1);  // first source read: the next block's
     uint16_t* outp = p.out;
     const int64_t seq_row0 = (int64_t)b * N;
-    merge_rows<MT>(sO, sRecv, s_w, n_src, split, first_row, per_rank, warp, lane, row_cta * MT, rows_total, G,
-                   seq_row0, p.Hq, kvh * G, outp);
+    switch (n_src) {
+      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+    }
   }
-  // Nobody leaves before every block has received its rows: a block's staging area is the source
-  // of copies that complete on the peers' barriers.
-  cluster.sync();
+  cluster.sync();  // no block may leave while a peer still reads its shared memory
 }
 
 // ------------------------------------------------------------------------------------ host side
