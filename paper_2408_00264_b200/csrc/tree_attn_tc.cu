@@ -44,7 +44,6 @@ constexpr int kThreads = 320;
 constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
 constexpr uint32_t kTmemCols = 512;
-constexpr int kFmaPairs = 3;                   // of every 8 pairs of exponentials, those computed on the FMA pipe
 constexpr float kRowSumLimit = 256.0f;        // a row of P may sum to 2^8 before the reference is replaced
 constexpr long long kWaitLimitCycles = 2000000000ll;  // SM cycles per wait: about a second
 
@@ -216,39 +215,6 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-// 2^x for two arguments on the FMA pipe, with the packed two-float instructions: round to the
-// nearest integer by adding 1.5 * 2^23, a cubic for 2^r on r in [-0.5, 0.5] (relative error 8e-5,
-// far below the bf16 rounding of P), and the integer part added to the exponent field.  For
-// finite arguments; below -126 the result is clamped to 2^-126.  The special-function unit
-// delivers one exponential per lane every eight cycles per scheduler and is what the softmax
-// threads wait for, so a share of the exponentials is computed here instead.
-__device__ __forceinline__ void ex2_fma_pair(float x0, float x1, float& y0, float& y1) {
-  x0 = fmaxf(x0, -126.f);
-  x1 = fmaxf(x1, -126.f);
-  uint32_t q0, q1, t0, t1;
-  asm("{\n\t.reg .b64 X, M, T, R, Q, C;\n\t"
-      "mov.b64 X, {%4, %5};\n\t"
-      "mov.b64 M, {%6, %6};\n\t"
-      "add.rn.f32x2 T, X, M;\n\t"
-      "mov.b64 M, {%7, %7};\n\t"
-      "add.rn.f32x2 R, T, M;\n\t"
-      "mov.b64 C, {%8, %8};\n\t"
-      "fma.rn.f32x2 R, R, C, X;\n\t"
-      "mov.b64 C, {%9, %9};\n\t"
-      "mov.b64 Q, {%10, %10};\n\t"
-      "fma.rn.f32x2 Q, R, C, Q;\n\t"
-      "mov.b64 C, {%11, %11};\n\t"
-      "fma.rn.f32x2 Q, R, Q, C;\n\t"
-      "mov.b64 C, {%12, %12};\n\t"
-      "fma.rn.f32x2 Q, R, Q, C;\n\t"
-      "mov.b64 {%0, %1}, Q;\n\t"
-      "mov.b64 {%2, %3}, T;\n\t}"
-      : "=r"(q0), "=r"(q1), "=r"(t0), "=r"(t1)
-      : "f"(x0), "f"(x1), "f"(12582912.f), "f"(-12582912.f), "f"(-1.f), "f"(0.05508868f), "f"(0.24260405f),
-        "f"(0.69327623f), "f"(0.99992895f));
-  y0 = __uint_as_float(q0 + (t0 << 23));
-  y1 = __uint_as_float(q1 + (t1 << 23));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -708,31 +674,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
           load_half(h);
-          if (all_full) {
-            // unmasked tile: kFmaPairs of every 8 pairs go to the FMA pipe (-inf scores of masked
-            // tiles are left to the special-function unit, which returns an exact zero)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float x0 = fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m);
-              const float x1 = fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m);
-              float p0, p1;
-              if ((j & 7) < kFmaPairs) {
-                ex2_fma_pair(x0, x1, p0, p1);
-              } else {
-                p0 = ex2(x0);
-                p1 = ex2(x1);
-              }
-              sum += p0 + p1;
-              pk[h * 32 + j] = pack_bf16(p0, p1);
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-              const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-              sum += p0 + p1;
-              pk[h * 32 + j] = pack_bf16(p0, p1);
-            }
+          for (int j = 0; j < 32; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
           }
         }
       };
