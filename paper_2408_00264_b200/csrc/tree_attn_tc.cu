@@ -669,40 +669,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (r == 0) m_ref = row_max();  // no reference yet: a cheap extra pass instead of a redo
       float sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      // The row is taken in quarters of 32 columns, the load of the next quarter in flight while
-      // this one is exponentiated (a tensor-memory load takes a few hundred cycles to return).
-      auto exp_quarter = [&](int qt, uint32_t (&x)[32]) {
-        if (!all_full) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (!((allow[qt] >> j) & 1u)) x[j] = 0xFF800000u;  // -inf
-        }
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float p0 = ex2(fmaf(__uint_as_float(x[2 * j]), p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(x[2 * j + 1]), p.scale_log2, neg_m));
-          sum += p0 + p1;
-          pk[qt * 16 + j] = pack_bf16(p0, p1);
-        }
-      };
       auto exp_pass = [&]() {
-        static_assert(BN == 128, "four quarters of 32 columns");
         sum = 0.f;
-        uint32_t (&xa)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sv[0]);
-        uint32_t (&xb)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sv[32]);
-        const uint32_t s_addr = tmem_S(slot) + lane_addr;
-        tmem_ld_x32(s_addr, xa);
-        tmem_wait_ld_for(xa);
-        tmem_ld_x32(s_addr + 32, xb);
-        exp_quarter(0, xa);
-        tmem_wait_ld_for(xb);
-        tmem_ld_x32(s_addr + 64, xa);
-        exp_quarter(1, xb);
-        tmem_wait_ld_for(xa);
-        tmem_ld_x32(s_addr + 96, xb);
-        exp_quarter(2, xa);
-        tmem_wait_ld_for(xb);
-        exp_quarter(3, xb);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          load_half(h);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[h * 32 + j] = pack_bf16(p0, p1);
+          }
+        }
       };
       exp_pass();
       const bool suspect = !(sum <= kRowSumLimit);  // also catches inf and NaN
