@@ -175,6 +175,43 @@ def test_attention_many_splits_and_ragged(clv, oracle):
     check_attention(oracle, w, st)
 
 
+def _scale_bf16_by_pow2(bits_arr, k):
+    """bf16 bit patterns times 2^k, exactly (normal numbers; zeros stay zeros)."""
+    b = bits_arr.astype(np.int64)
+    expo = (b >> 7) & 0xFF
+    new = np.clip(expo + k, 1, 254)
+    out = (b & ~(0xFF << 7)) | (new << 7)
+    return np.where(expo == 0, b, out).astype(np.uint16)
+
+
+@pytest.mark.parametrize("k_lo,k_hi", [(40, 40), (-40, -40), (30, -30), (-30, 30)])
+def test_attention_value_magnitudes_across_splits(clv, oracle, k_lo, k_hi):
+    # The split-KV partial sums travel between blocks in fp16, every row scaled by its own power of
+    # two.  Values far outside the fp16 range, and key ranges whose values differ by 2^60, must
+    # come out as the checker computes them (relative to each output row's scale: the absolute
+    # tolerance presupposes values of order one and is not applied here).
+    from parity_util import attn_errors, ATTN_MAX_REL
+    cfg = W.small_config(batch=2, n_q_heads=8, n_kv_heads=2, ctx=(1500, 2300), n_nodes=48, vocab=64,
+                         seed=W.BASE_SEED + 77)
+    w = W.generate(cfg)
+    half = w.v_cache.shape[1] // 2 if w.v_cache.ndim == 4 else None
+    assert half is not None
+    w.v_cache[:, :half] = _scale_bf16_by_pow2(w.v_cache[:, :half], k_lo)
+    w.v_cache[:, half:] = _scale_bf16_by_pow2(w.v_cache[:, half:], k_hi)
+    w.v_tree[:] = _scale_bf16_by_pow2(w.v_tree, k_hi)
+    st = make_step(w)
+    st.tree_attn()
+    torch.cuda.synchronize()
+    ref, _, lse, status = oracle.tree_attn(w.q, w.k_cache, w.v_cache, w.k_tree, w.v_tree, w.parent,
+                                           w.ctx_len, w.scale, block_table=w.block_table)
+    got = bits(st.out)
+    assert np.array_equal(st.status[0].cpu().numpy(), status)
+    assert np.isfinite(W.bf16_bits_to_f64(got)).all()
+    _, rel = attn_errors(got, ref)
+    assert rel <= ATTN_MAX_REL, rel
+    assert np.abs(st.lse.cpu().numpy().astype(np.float64) - lse).max() < 2e-3
+
+
 def test_attention_mask_exactness_on_device(clv, oracle):
     # overwriting K/V of nodes that are not ancestors must not change a node's output at all
     cfg = W.small_config(batch=1, n_q_heads=4, n_kv_heads=2, ctx=100, n_nodes=24, vocab=64)
