@@ -303,29 +303,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   int b = unit / p.Hkv;
   const int kvh = unit - b * p.Hkv;
   const int N = p.N, G = p.G, rows_total = G * N;
-  if (p.longest_first) {
-    // More blocks than SMs and contexts of different lengths (ragged batch): hand the sequences
-    // out longest first, so that the block scheduler packs the short ones into the gaps.  Block
-    // group `b` takes the sequence whose length has rank b (ties by index); every thread ranks
-    // at most one sequence.
-    __shared__ int s_seq;
-    const int want = b;
-    for (int i = tid; i < p.B; i += kThreads) {
-      const int Li = p.ctx_len[i];
-      int rank = 0;
-      for (int j = 0; j < p.B; ++j) {
-        const int Lj = __ldg(p.ctx_len + j);
-        rank += (Lj > Li) || (Lj == Li && j < i);
-      }
-      if (rank == want) s_seq = i;
-    }
-    __syncthreads();
-    b = s_seq;
-  }
-
-  // ---- set-up and per-sequence checks in one go: while thread 0 initialises the barriers and
-  //      warp 1 allocates tensor memory, everybody reads parent[] and the context length; the one
-  //      block-wide synchronisation below publishes all of it -------------------------------------
+  // ---- set-up that reads no global memory: barriers, tensor memory, descriptor prefetch.  The
+  //      kernel is launched with programmatic stream serialisation, so this part may run while the
+  //      previous kernel of the stream drains; everything after the grid dependency wait sees that
+  //      kernel's results.  Dependents are released at once: they wait for this grid themselves.
   constexpr int NRING = 2 * KST + 2 * VST;
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   if (tid == 0) {
@@ -346,6 +327,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
     tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
   }
+  cudaGridDependencySynchronize();
+  cudaTriggerProgrammaticLaunchCompletion();
+
+  if (p.longest_first) {
+    // More blocks than SMs and contexts of different lengths (ragged batch): hand the sequences
+    // out longest first, so that the block scheduler packs the short ones into the gaps.  Block
+    // group `b` takes the sequence whose length has rank b (ties by index); every thread ranks
+    // at most one sequence.
+    __shared__ int s_seq;
+    const int want = b;
+    for (int i = tid; i < p.B; i += kThreads) {
+      const int Li = p.ctx_len[i];
+      int rank = 0;
+      for (int j = 0; j < p.B; ++j) {
+        const int Lj = __ldg(p.ctx_len + j);
+        rank += (Lj > Li) || (Lj == Li && j < i);
+      }
+      if (rank == want) s_seq = i;
+    }
+    __syncthreads();
+    b = s_seq;
+  }
+
+  // ---- per-sequence checks: everybody reads parent[] and the context length; the one block-wide
+  //      synchronisation below publishes them together with the set-up above --------------------
   const int L = p.ctx_len[b];
   bool bad = false;
   for (int i = tid; i < N; i += kThreads) {
@@ -1013,13 +1019,15 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = mt == 1 ? Cfg<1>::kSmem : Cfg<2>::kSmem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;  // the blocks that split one row tile's keys
   attr[0].val.clusterDim.x = 1;
   attr[0].val.clusterDim.y = (unsigned)plan.splits;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up overlaps the previous kernel's tail
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   if (mt == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
   return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<2>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
 }

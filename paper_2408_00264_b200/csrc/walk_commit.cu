@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
   __shared__ int s_ok;
   const int b = blockIdx.x, tid = threadIdx.x;
   cudaGridDependencySynchronize();  // programmatic launch: the walk's outputs are complete after this
+  cudaTriggerProgrammaticLaunchCompletion();  // a following kernel may set up; it waits for this grid itself
   const int L = p.ctx_len[b];
   const int len = p.accept_len[b];
   if (tid == 0) s_ok = (L >= 0 && len >= 0 && len <= p.path_cap && len <= CLV_MAX_NODES) ? 1 : 0;
