@@ -88,7 +88,6 @@ __global__ void __launch_bounds__(kThreads) argmax_kernel(Params p) {
   // programmatic launch: the grid may be set up while the previous kernel of the stream drains;
   // nothing is read or written before that kernel's results are complete
   cudaGridDependencySynchronize();
-  cudaTriggerProgrammaticLaunchCompletion();  // the next kernel waits for this grid itself
 
   Track trk;
   track_init(trk);

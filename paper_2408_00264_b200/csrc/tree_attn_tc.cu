@@ -306,7 +306,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // ---- set-up that reads no global memory: barriers, tensor memory, descriptor prefetch.  The
   //      kernel is launched with programmatic stream serialisation, so this part may run while the
   //      previous kernel of the stream drains; everything after the grid dependency wait sees that
-  //      kernel's results.  Dependents are released at once: they wait for this grid themselves.
+  //      kernel's results.
   constexpr int NRING = 2 * KST + 2 * VST;
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   if (tid == 0) {
@@ -328,7 +328,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
   }
   cudaGridDependencySynchronize();
-  cudaTriggerProgrammaticLaunchCompletion();
 
   if (p.longest_first) {
     // More blocks than SMs and contexts of different lengths (ragged batch): hand the sequences
