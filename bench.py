@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 ROTATE = 4   # distinct input sets cycled between steps: 4 x 138 MB > 2 x L2 (126 MB)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
 # profiles/verify_step_C3.md; valid for the kernels as they were when that capture was taken
-NCU_TRAFFIC = {("C3", "tree_attn"): 71.8e6, ("C3", "accept_argmax"): 65.8e6}
+NCU_TRAFFIC = {("C3", "tree_attn"): 71.7e6, ("C3", "accept_argmax"): 65.9e6}
 
 
 def measured_peaks():
