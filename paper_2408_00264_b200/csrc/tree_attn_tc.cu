@@ -216,12 +216,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Two non-negative floats to a bf16 pair, rounded to nearest (ties up) with integer instructions.
-// The conversion instruction shares the special-function pipe with the exponentials, which is
-// what the softmax threads wait for; adds and a byte permute run beside it.
-__device__ __forceinline__ uint32_t pack_bf16_pos(float lo, float hi) {
-  return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -690,7 +684,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
             const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
             sum += p0 + p1;
-            pk[h * 32 + j] = pack_bf16_pos(p0, p1);
+            pk[h * 32 + j] = pack_bf16(p0, p1);
           }
         }
       };
