@@ -160,6 +160,30 @@ clv_status clv_accept_argmax_noalloc(const clv_shape* shape,
                                      void* cuda_stream);
 
 /*
+ * LM head fused with the greedy choice (Sec. 3.1: the target's final norm and LM head produce the
+ * logits of every tree node; Sec. 4.2: greedy decoding at temperature 0):
+ *   argmax_ids[r] = the lowest v that maximises round_bf16(sum_k hidden[r][k] * weight[v][k]),
+ * the products accumulated in fp32 and the logit rounded to bf16 (round to nearest even) before
+ * the comparison, as a bf16 logits tensor would hold it.  The logits are never written to memory.
+ * hidden: device, bf16 [rows, ld_hidden], already normalised; weight: device, bf16
+ * [vocab, ld_weight] (one row per vocabulary entry); hidden_dim must be a multiple of 64, both
+ * row strides multiples of 8 elements, both bases 16-byte aligned.  rows <= 32767.
+ * status: device, one int32: CLV_OK, or CLV_ERR_TIMEOUT if a bounded wait inside the kernel ran
+ * out (argmax_ids is then unspecified).  workspace: as returned by clv_workspace_bytes for any
+ * shape, initialised with clv_workspace_init; the caller owns every buffer.  NaN logits are
+ * ignored; a row without any finite or infinite logit gives 0.
+ * Errors: CLV_ERR_NULL, CLV_ERR_SHAPE, CLV_ERR_ALIGN, CLV_ERR_UNSUPPORTED (hidden_dim not a
+ * multiple of 64, too many rows, no tensor-map support in the driver), CLV_ERR_WORKSPACE,
+ * CLV_ERR_CUDA.  Nothing is launched on an error.
+ */
+clv_status clv_lm_head_argmax(const void* hidden, int64_t ld_hidden,
+                              const void* weight, int64_t ld_weight,
+                              int32_t rows, int32_t hidden_dim, int32_t vocab,
+                              int32_t* argmax_ids,   /* [rows] */
+                              int32_t* status,       /* [1]    */
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Greedy acceptance walk (Sec. 2.1 verification phase; Sec. 4.1).  Start at the root; at node cur
  * the target wants argmax_ids[cur]; the child of cur whose drafted token equals it (the lowest
  * index if siblings repeat a token) is accepted and becomes cur; otherwise stop.

@@ -116,6 +116,26 @@ def argmax(logits: np.ndarray, vocab: int) -> np.ndarray:
     return ids.reshape(lead)
 
 
+def lm_head_argmax(hidden: np.ndarray, weight: np.ndarray, rows=None, want_logits: bool = False):
+    """Greedy choice from the LM head (Sec. 3.1 + Sec. 4.2): hidden [M, K] and weight [V, K] bf16
+    bits; logits in float64, rounded to bf16, first strict maximum.  Returns ids [n] (and the
+    unrounded float64 logits [n, V] if asked) for the selected rows (all if ``rows`` is None)."""
+    lib = _load()
+    h = _c(hidden, np.uint16)
+    w = _c(weight, np.uint16)
+    M, K = h.shape
+    V = w.shape[0]
+    assert w.shape[1] == K
+    sel = None if rows is None else _c(np.asarray(rows), np.int32)
+    n = M if sel is None else len(sel)
+    ids = np.empty(n, dtype=np.int32)
+    z = np.empty((n, V), dtype=np.float64) if want_logits else None
+    rc = lib.orc_lm_head_argmax(ctypes.c_int(n), _p(sel), ctypes.c_int(K), ctypes.c_int(V),
+                                ctypes.c_int64(K), ctypes.c_int64(K), _p(h), _p(w), _p(z), _p(ids))
+    assert rc == 0
+    return (ids, z) if want_logits else ids
+
+
 def accept_walk(parent, tokens, ids, path_cap: int):
     """Greedy acceptance walk; returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
     status [B])."""

@@ -15,6 +15,8 @@
  *                       tree's topology matrix (a node sees the committed context and its own
  *                       ancestors, itself included).
  *   orc_argmax        - Sec. 4.2 (Table 1 note): temperature 0 is greedy decoding of the target.
+ *   orc_lm_head_argmax - Sec. 3.1 (final norm + LM head give the logits) followed by Sec. 4.2's
+ *                       greedy choice, the logit held in bf16 like a logits tensor.
  *   orc_accept_walk   - Sec. 2.1 verification phase (the target filters out wrong drafted
  *                       tokens; the output equals plain decoding) with the greedy rule of the
  *                       tree-sampling algorithm Sec. 4.1 adopts.
@@ -24,7 +26,8 @@
  * Pins (tests/test_oracle_*.py): path linearisation, chain == causal prefill, star == independent
  * decodes, a float64 library attention with an explicit boolean mask, convex-hull and
  * log-sum-exp identities, mask exactness under perturbation, brute-force path enumeration,
- * numpy's first-occurrence argmax, and the commit/append equivalence.  No function here is
+ * numpy's first-occurrence argmax, the commit/append equivalence, and for the LM head a float64
+ * library matrix product, a one-hot weight matrix and planted rounding ties.  No function here is
  * "parity unpinned".
  */
 #include <math.h>
@@ -181,6 +184,41 @@ int orc_argmax(int64_t n_rows, int vocab, int64_t ld, const uint16_t *logits, in
       if (x > best) { best = x; arg = v; }
     }
     ids[r] = arg;
+  }
+  return 0;
+}
+
+/*
+ * LM head followed by the greedy choice (Sec. 3.1: the logits of a node are the LM head applied
+ * to its normalised hidden state; Sec. 4.2: temperature 0).  For each selected row r:
+ *   logit[v] = sum_k hidden[r][k] * weight[v][k]   in double, then rounded to bf16 (the precision
+ *   the logits tensor has), ids = the first strict maximum of the rounded values.
+ * logits64 (optional, [n_sel][vocab]) receives the unrounded doubles so that a test can see how
+ * close the runners-up are.  rows == NULL selects rows 0 .. n_sel-1.
+ */
+int orc_lm_head_argmax(int n_sel, const int32_t *rows, int hidden_dim, int vocab, int64_t ld_hidden,
+                       int64_t ld_weight, const uint16_t *hidden, const uint16_t *weight,
+                       double *logits64, int32_t *ids) {
+  for (int i = 0; i < n_sel; ++i) {
+    const uint16_t *h = hidden + (int64_t)(rows ? rows[i] : i) * ld_hidden;
+    double *z = (double *)malloc(sizeof(double) * (size_t)vocab);
+    if (!z) return -1;
+#pragma omp parallel for schedule(static)
+    for (int v = 0; v < vocab; ++v) {
+      const uint16_t *w = weight + (int64_t)v * ld_weight;
+      double acc = 0.0;
+      for (int k = 0; k < hidden_dim; ++k) acc += bf16_to_f64(h[k]) * bf16_to_f64(w[k]);
+      z[v] = acc;
+    }
+    double best = bf16_to_f64(f64_to_bf16(z[0]));
+    int32_t arg = 0;
+    for (int v = 1; v < vocab; ++v) {
+      double x = bf16_to_f64(f64_to_bf16(z[v]));
+      if (x > best) { best = x; arg = v; }
+    }
+    ids[i] = arg;
+    if (logits64) memcpy(logits64 + (size_t)i * vocab, z, sizeof(double) * (size_t)vocab);
+    free(z);
   }
   return 0;
 }

@@ -24,6 +24,7 @@ EXPORTS = (
     "clv_workspace_bytes", "clv_workspace_init", "clv_tree_attn", "clv_accept_argmax",
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
+    "clv_lm_head_argmax",
 )
 
 
@@ -86,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.clv_accept_argmax.argtypes = [vp, vp, i64, vp, vp, sz, vp]
         L.clv_accept_argmax_noalloc.restype = i32
         L.clv_accept_argmax_noalloc.argtypes = [vp, vp, i64, vp, vp]
+        L.clv_lm_head_argmax.restype = i32
+        L.clv_lm_head_argmax.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp]
         L.clv_accept_walk.restype = i32
         L.clv_accept_walk.argtypes = [vp] * 9
         L.clv_kv_commit.restype = i32
@@ -182,6 +185,21 @@ def clv_accept_argmax_noalloc(shape, logits, ld, argmax_ids, stream=None, check=
                                            _stream(stream))
     if check:
         _check(code, "clv_accept_argmax_noalloc")
+    return code
+
+
+def clv_lm_head_argmax(hidden, weight, argmax_ids, status, workspace, stream=None, check=True) -> int:
+    """hidden bf16 [rows, hidden_dim], weight bf16 [vocab, hidden_dim] (row strides taken from the
+    tensors), argmax_ids int32 [rows], status int32 [1]."""
+    rows, hidden_dim = hidden.shape
+    vocab = weight.shape[0]
+    code = lib().clv_lm_head_argmax(_ptr(hidden), int(hidden.stride(0)), _ptr(weight),
+                                    int(weight.stride(0)), int(rows), int(hidden_dim), int(vocab),
+                                    _ptr(argmax_ids), _ptr(status), _ptr(workspace),
+                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _stream(stream))
+    if check:
+        _check(code, "clv_lm_head_argmax")
     return code
 
 

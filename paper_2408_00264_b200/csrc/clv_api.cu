@@ -150,6 +150,24 @@ clv_status clv_accept_argmax_noalloc(const clv_shape* shape, const void* logits,
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
+clv_status clv_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight,
+                              int64_t ld_weight, int32_t rows, int32_t hidden_dim, int32_t vocab,
+                              int32_t* argmax_ids, int32_t* status, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  if (!hidden || !weight || !argmax_ids || !status) return CLV_ERR_NULL;
+  if (rows < 1 || hidden_dim < 1 || vocab < 1 || ld_hidden < hidden_dim || ld_weight < hidden_dim)
+    return CLV_ERR_SHAPE;
+  if (!aligned16(hidden) || !aligned16(weight) || (ld_hidden % 8) != 0 || (ld_weight % 8) != 0)
+    return CLV_ERR_ALIGN;
+  if (!lm_head_supported(rows, hidden_dim, vocab)) return CLV_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < kWsFixedBytes) return CLV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  cudaError_t e = launch_lm_head_argmax(hidden, ld_hidden, weight, ld_weight, rows, hidden_dim, vocab,
+                                        argmax_ids, status, ws_tickets(workspace),
+                                        static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
 clv_status clv_accept_walk(const clv_shape* shape, const int32_t* parent, const int32_t* tokens,
                            const int32_t* argmax_ids, int32_t* accept_len, int32_t* accept_idx,
                            int32_t* next_token, int32_t* status, void* cuda_stream) {

@@ -70,6 +70,12 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
                                 cudaStream_t stream);
 
+// ---- LM head fused with the argmax (tcgen05 GEMM whose logits stay in tensor memory) ---------------
+bool lm_head_supported(int rows, int hidden, int vocab);
+cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
+                                  int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
+                                  unsigned* tickets, cudaStream_t stream);
+
 int sm_count();
 
 }  // namespace clv

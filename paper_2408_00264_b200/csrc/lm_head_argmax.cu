@@ -1,0 +1,294 @@
+// LM head fused with the per-node greedy choice (Sec. 3.1: final norm and LM head of the target;
+// Sec. 4.2: greedy decoding at T = 0): ids[r] = argmax_v round_bf16(<hidden[r, :], W[v, :]>), lowest
+// v on ties.  The logits are never written: each 256 x 256 tile of them lives in tensor memory
+// only, and its row maxima go to one 64-bit key per row with atomicMax.
+//
+// A persistent block per SM walks (vocabulary tile, row block) pairs.  Warp 0 streams 64-wide
+// K chunks of the weight tile ([256 vocabulary rows][64]) and of the hidden rows ([2 x 128][64])
+// through a three-deep TMA ring, warp 1 issues tcgen05.mma (M 128, N 256, K 16; two accumulators
+// of 256 columns fill the tensor memory), warps 2..9 are the epilogue: one thread per row scans
+// the accumulator for the row's best (value, lowest index).  The weight matrix is read from HBM
+// once per row block; the hidden rows are re-read from L2 by every block.
+#include <cuda_bf16.h>
+#include <limits.h>
+#include <math.h>
+
+#include "clv_internal.cuh"
+#include "tc_ptx.cuh"
+#include "tmem_access.cuh"
+
+namespace clv {
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int BM = 128;              // rows per accumulator
+constexpr int MB = 2 * BM;           // rows per block step (two accumulators)
+constexpr int BN = 256;              // vocabulary entries per tile
+constexpr int BK = 64;               // K elements per ring stage (one 128-byte swizzle row)
+constexpr int kStages = 3;
+constexpr uint32_t kATile = BM * BK * 2;      // 16 KB
+constexpr uint32_t kWTile = BN * BK * 2;      // 32 KB
+constexpr uint32_t kStageBytes = 2 * kATile + kWTile;
+constexpr uint32_t kSmem = kStages * kStageBytes + 1024;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kIdesc = make_idesc(BM, BN, false);
+
+struct Params {
+  int M, K, V;
+  int n_tiles, m_blocks;
+  int32_t* ids;
+  unsigned long long* keys;   // [M], zero between calls
+  unsigned* counter;          // zero between calls
+  unsigned* aborts;           // blocks that gave up a wait; zero between calls
+  int32_t* status;            // one word: CLV_OK or CLV_ERR_TIMEOUT
+};
+
+__device__ __forceinline__ unsigned long long pack_key(float v, int i) {
+  if (v == 0.0f) v = 0.0f;  // -0 and +0 are the same value: one bit pattern
+  const uint32_t f = __float_as_uint(v);
+  const uint32_t ord = (f & 0x80000000u) ? ~f : (f | 0x80000000u);
+  return ((unsigned long long)ord << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+}
+__device__ __forceinline__ float round_bf16(float x) {
+  return __bfloat162float(__float2bfloat16_rn(x));
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                      const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) unsigned long long s_bar[2 * kStages + 3];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ int s_last;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t bar0 = smem_u32(&s_bar[0]);
+  auto bar_full = [&](int s) { return bar0 + 8u * s; };
+  auto bar_empty = [&](int s) { return bar0 + 8u * (kStages + s); };
+  const uint32_t bar_acc_full = bar0 + 8u * (2 * kStages);       // a tile's accumulators are complete
+  const uint32_t bar_acc_empty = bar0 + 8u * (2 * kStages + 1);  // the epilogue has read them
+  const uint32_t bar_drain = bar0 + 8u * (2 * kStages + 2);
+  if (tid == 0) {
+    for (int i = 0; i < 2 * kStages; ++i) mbar_init(bar0 + 8u * i, 1);
+    mbar_init(bar_acc_full, 1);
+    mbar_init(bar_acc_empty, 2 * BM);
+    mbar_init(bar_drain, 1);
+    s_abort = 0;
+    fence_barrier_init();
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+  if (tid == 64) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_w); }
+  cudaGridDependencySynchronize();  // programmatic launch: the previous kernel's results are complete
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abort_flag = &s_abort;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  auto sA = [&](int s, int mt) { return smem_base + (uint32_t)s * kStageBytes + (uint32_t)mt * kATile; };
+  auto sW = [&](int s) { return smem_base + (uint32_t)s * kStageBytes + 2 * kATile; };
+
+  // work items of this block: (vocabulary tile n, row block mb), all row blocks of a tile in a row
+  // so that the weight tile is read from HBM once and from L2 afterwards
+  const int n_items = p.n_tiles * p.m_blocks;
+  const int k_chunks = p.K / BK;
+  int issued = 0;  // ring stages filled by the producer (for the drain)
+
+  if (warp == 0) {
+    // =========================== TMA producer ===============================================
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int n = item / p.m_blocks, mb = item - n * p.m_blocks;
+        const int rows_left = p.M - mb * MB;
+        const int m_tiles = rows_left > BM ? 2 : 1;
+        for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
+          const int s = it % kStages;
+          if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(bar_full(s), kWTile + (uint32_t)m_tiles * kATile);
+          tma_load_2d(sW(s), &tm_w, kc * BK, n * BN, bar_full(s));
+          for (int mt = 0; mt < m_tiles; ++mt)
+            tma_load_2d(sA(s, mt), &tm_a, kc * BK, mb * MB + mt * BM, bar_full(s));
+          issued = it + 1;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================== MMA issuer ===================================================
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0, tile = 0;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
+        const int n = item / p.m_blocks, mb = item - n * p.m_blocks;
+        (void)n;
+        const int m_tiles = (p.M - mb * MB) > BM ? 2 : 1;
+        if (tile > 0) {  // the epilogue has taken the previous tile out of tensor memory
+          ok = mbar_wait(bar_acc_empty, (tile - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
+          const int s = it % kStages;
+          ok = mbar_wait(bar_full(s), (it / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t wd = smem_desc(sW(s), 16, 1024);
+          for (int mt = 0; mt < m_tiles; ++mt) {
+            const uint64_t ad = smem_desc(sA(s, mt), 16, 1024);
+#pragma unroll
+            for (int ks = 0; ks < BK / 16; ++ks)
+              umma_bf16(tmem + (uint32_t)(mt * BN), ad + (uint64_t)((ks * 32) >> 4), wd + (uint64_t)((ks * 32) >> 4),
+                        kIdesc, (kc > 0 || ks > 0) ? 1u : 0u);
+          }
+          umma_commit(bar_empty(s));  // the stage is free once these MMAs have read it
+        }
+        if (ok) umma_commit(bar_acc_full);
+      }
+    }
+  } else {
+    // =========================== epilogue: one thread per row ==================================
+    const int mt = (warp - 2) >> 2;          // accumulator of this group
+    const int quarter = warp & 3;            // tensor-memory lanes this warp may touch
+    const int row_in_tile = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    bool ok = true;
+    int tile = 0;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
+      const int n = item / p.m_blocks, mb = item - n * p.m_blocks;
+      const int row = mb * MB + mt * BM + row_in_tile;
+      const bool row_valid = row < p.M;
+      ok = mbar_wait(bar_acc_full, tile & 1, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool group_used = (p.M - mb * MB) > mt * BM;   // second accumulator unused for a short row block
+      float best_v = -INFINITY;
+      int best_i = INT_MAX;
+      if (group_used) {
+        const int col0 = n * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t x[32];
+          tmem_ld_x32(tmem + lane_addr + (uint32_t)(mt * BN + c), x);
+          tmem_wait_ld();
+          // rounding to bf16 is monotonic: the chunk's maximum first, the position only if it wins
+          float m = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float v = (col0 + c + j < p.V) ? __uint_as_float(x[j]) : -INFINITY;
+            x[j] = __float_as_uint(v);
+            m = fmaxf(m, v);   // NaN operands are dropped
+          }
+          const float mr = round_bf16(m);
+          if (mr > best_v) {
+            int first = 31;
+#pragma unroll
+            for (int j = 31; j >= 0; --j)
+              if (round_bf16(__uint_as_float(x[j])) == mr) first = j;
+            best_v = mr;
+            best_i = col0 + c + first;
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_acc_empty);
+      if (row_valid && best_i != INT_MAX) atomicMax(p.keys + row, pack_key(best_v, best_i));
+    }
+  }
+
+  // ---- teardown --------------------------------------------------------------------------------
+  __syncwarp();
+  if (*abort_flag) {
+    if (warp == 0 && lane == 0)
+      for (int i = max(0, issued - kStages); i < issued; ++i) mbar_drain(bar_full(i % kStages), (i / kStages) & 1);
+    if (warp == 1 && lane == 0) {
+      umma_commit(bar_drain);
+      mbar_drain(bar_drain, 0);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+  if (tid == 0) {
+    if (*abort_flag) atomicAdd(p.aborts, 1u);
+    __threadfence();
+    const unsigned arrived = atomicInc(p.counter, gridDim.x - 1);  // wraps to 0
+    s_last = (arrived == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  // the last block turns the keys into indices and leaves keys and counters zero for the next call
+  __threadfence();
+  if (tid == 0) *p.status = atomicExch(p.aborts, 0u) ? (int)CLV_ERR_TIMEOUT : (int)CLV_OK;
+  for (int r = tid; r < p.M; r += kThreads) {
+    const unsigned long long key = atomicExch(p.keys + r, 0ull);
+    const int idx = (int)(0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull));
+    p.ids[r] = (key == 0ull) ? 0 : idx;  // a row of only -inf / NaN logits: first index
+  }
+}
+
+bool make_map_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t k, int64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)k, rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool lm_head_supported(int rows, int hidden, int vocab) {
+  // keys share the zero-initialised counter area of the workspace: 2 words per row after the counter
+  return rows > 0 && vocab > 0 && hidden > 0 && (hidden % BK) == 0 && 2 * (int64_t)rows + 2 <= kTickets &&
+         encode_fn() != nullptr;
+}
+
+cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
+                                  int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
+                                  unsigned* tickets, cudaStream_t stream) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSmem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  CUtensorMap tm_a, tm_w;
+  if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, BM) ||
+      !make_map_2d(&tm_w, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN))
+    return cudaErrorInvalidValue;
+  Params p;
+  p.M = rows;
+  p.K = hidden_dim;
+  p.V = vocab;
+  p.n_tiles = (vocab + BN - 1) / BN;
+  p.m_blocks = (rows + MB - 1) / MB;
+  p.ids = ids;
+  p.counter = tickets;
+  p.aborts = tickets + 1;
+  p.keys = reinterpret_cast<unsigned long long*>(tickets + 2);
+  p.status = status;
+  const int items = p.n_tiles * p.m_blocks;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(items < sm_count() ? items : sm_count()), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, lm_head_argmax_kernel, tm_a, tm_w, p);
+}
+
+}  // namespace clv

@@ -272,6 +272,30 @@ def make_logits(rows: int, vocab: int, ld: int, winner: np.ndarray, margin: floa
     return lg
 
 
+def make_lm_head(rows: int, hidden_dim: int, vocab: int, seed: int, planted: float = 12.0):
+    """Inputs of the LM head for ``rows`` tree nodes: hidden states N(0,1) and a weight matrix
+    N(0, 1/hidden_dim) (so that logits are about N(0,1)), both rounded to bf16 and returned as bit
+    patterns [rows, hidden_dim] and [vocab, hidden_dim].  With ``planted`` > 0 every hidden row
+    gets ``planted`` times the weight row of a drawn vocabulary entry added before rounding, which
+    lifts that entry's logit about ``planted`` above the rest: ``winner`` [rows] holds the entries
+    (a clear argmax); with ``planted`` = 0 the argmax is whatever the draw gives and ``winner`` is
+    None.  Generated in slabs so that a 128256 x 4096 matrix needs no float64 copy."""
+    ss = np.random.SeedSequence(seed).spawn(3)
+    rng_w = np.random.default_rng(ss[0])
+    weight = np.empty((vocab, hidden_dim), dtype=np.uint16)
+    inv = np.float32(1.0 / np.sqrt(hidden_dim))
+    slab = max(1, (1 << 24) // hidden_dim)
+    for v0 in range(0, vocab, slab):
+        v1 = min(vocab, v0 + slab)
+        weight[v0:v1] = f32_to_bf16_bits(rng_w.standard_normal((v1 - v0, hidden_dim), dtype=np.float32) * inv)
+    hid = np.random.default_rng(ss[1]).standard_normal((rows, hidden_dim), dtype=np.float32)
+    winner = None
+    if planted > 0:
+        winner = np.random.default_rng(ss[2]).integers(0, vocab, size=rows).astype(np.int32)
+        hid += np.float32(planted) * bf16_bits_to_f32(weight[winner])
+    return f32_to_bf16_bits(hid), weight, winner
+
+
 def generate(cfg: VerifyConfig, ld_pad: int = 0, extra_cap: int = 0,
              tree_order: str = "score") -> Workload:
     """Create every input of one verify step for ``cfg`` (deterministic in ``cfg.seed``).
