@@ -36,6 +36,59 @@ ROTATE = 4   # distinct input sets cycled between steps: 4 x 138 MB > 2 x L2 (12
 NCU_TRAFFIC = {("C3", "tree_attn"): 71.7e6, ("C3", "accept_argmax"): 65.9e6}
 
 
+def time_lm_head(rows, hidden, vocab, dev, args):
+    """clv_lm_head_argmax on `rows` tree nodes: microseconds per launch (CUDA events, launches
+    replayed from a CUDA graph over two copies of the weight matrix, 2 x 1.05 GB at vocabulary
+    128256, so that no launch finds its weights in L2), with the rates against both roofs."""
+    import torch
+    from paper_2408_00264_b200 import binding as clv
+    from paper_2408_00264_b200 import workloads as W
+    h, w, win = W.make_lm_head(rows, hidden, vocab, seed=W.BASE_SEED + 77)
+    hid = W.as_torch_bf16(h).to(dev)
+    wgt = [W.as_torch_bf16(w).to(dev)]
+    wgt.append(wgt[0].clone())
+    ids = torch.zeros(rows, dtype=torch.int32, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = clv.new_workspace(clv.make_shape(1, 1, 1, 1, vocab=8), None, 0, dev)
+    for i in range(4):
+        clv.clv_lm_head_argmax(hid, wgt[i % 2], ids, st, ws)
+    torch.cuda.synchronize()
+    ok = bool((ids.cpu().numpy() == win).all()) and int(st.item()) == 0
+    if args.no_graph:
+        run = lambda: [clv.clv_lm_head_argmax(hid, wgt[i], ids, st, ws) for i in range(2)]  # noqa: E731
+    else:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(2):
+                clv.clv_lm_head_argmax(hid, wgt[i], ids, st, ws)
+        run = g.replay
+    run()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    reps = 10
+    a.record(cur)
+    for _ in range(reps):
+        run()
+    b.record(cur)
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) / (2 * reps) * 1e3
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except (OSError, ValueError):
+        pass
+    tf_peak, tf_kind = (peaks["bf16_tflops"], "measured") if "bf16_tflops" in peaks else (1590.0, "fallback")
+    bw_peak, bw_kind = measured_peaks()
+    tflops = 2.0 * rows * hidden * vocab / us / 1e6
+    gbs = (vocab + rows) * hidden * 2 / us / 1e3
+    return {"rows": rows, "hidden": hidden, "vocab": vocab, "us": us, "ids_match_planted_winners": ok,
+            "tflops": tflops, "frac_of_bf16_peak": {"of_%s_%.0f_TFLOPs" % (tf_kind, tf_peak): tflops / tf_peak},
+            "algorithmic_bytes": (vocab + rows) * hidden * 2 + rows * 4, "gbs": gbs,
+            "frac_of_hbm_peak": {"of_%s_%.0f_GBps" % (bw_kind, bw_peak): gbs / bw_peak},
+            "launches_timed": 2 * reps}
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -313,6 +366,11 @@ def run_clv(args):
         barrier()
         e2e_ms = e0.elapsed_time(e1) / n_e2e
 
+    # ---- the step before the argmax: LM head fused with the greedy choice (rank 0 only) ---------
+    lm_head = None
+    if rank == 0 and not args.no_lm_head:
+        lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
+
     # ---- max over ranks ------------------------------------------------------------------------
     step_ms, e2e_ms, job_bytes = reduce_over_ranks(dist, dev, step_ms, e2e_ms, float(nbytes["total"]))
     if rank != 0:
@@ -342,6 +400,7 @@ def run_clv(args):
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
+        "next_rows": {"lm_head_argmax": lm_head},
         "gpu_launches": 4 * args.steps,
         "clocks": clocks.summary(),
     }
@@ -365,6 +424,8 @@ def main():
     ap.add_argument("--impl", default="clv", choices=["clv", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch the four calls per step directly")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lm-head", action="store_true",
+                    help="skip the timing of clv_lm_head_argmax (hidden 4096, the workload's rows and vocabulary)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
