@@ -32,10 +32,13 @@ constexpr uint32_t kStageBytes = 2 * kATile + kWTile;
 constexpr uint32_t kSmem = kStages * kStageBytes + 1024;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kIdesc = make_idesc(BM, BN, false);
+constexpr uint32_t kIdescHalf = make_idesc(BM, BN / 2, false);
 
 struct Params {
   int M, K, V;
   int n_tiles, m_blocks;
+  int full_items;   // work items that are whole tiles; the rest are half tiles (128 vocabulary entries)
+  int n_items;
   int32_t* ids;
   unsigned long long* keys;   // [M], zero between calls
   unsigned* counter;          // zero between calls
@@ -53,9 +56,31 @@ __device__ __forceinline__ float round_bf16(float x) {
   return __bfloat162float(__float2bfloat16_rn(x));
 }
 
+// Work item -> (first vocabulary entry, entries, row block).  Items are whole tiles, all row
+// blocks of a tile in a row so that a weight tile is read from HBM once and from L2 afterwards;
+// when the last round would leave more than half of the blocks idle, its tiles are cut in two
+// halves of 128 entries so that twice as many blocks share it.
+struct Item {
+  int col0, cols, mb;
+};
+__device__ __forceinline__ Item decode_item(const Params& p, int item) {
+  int tile = item, half = -1;
+  if (item >= p.full_items) {
+    const int j = item - p.full_items;
+    tile = p.full_items + (j >> 1);
+    half = j & 1;
+  }
+  const int n = tile / p.m_blocks;
+  Item it;
+  it.mb = tile - n * p.m_blocks;
+  it.col0 = n * BN + (half > 0 ? BN / 2 : 0);
+  it.cols = half < 0 ? BN : BN / 2;
+  return it;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
-                      const Params p) {
+                      const __grid_constant__ CUtensorMap tm_w_half, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) unsigned long long s_bar[2 * kStages + 3];
   __shared__ uint32_t s_tmem;
@@ -79,7 +104,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     fence_async_smem();
   }
   if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
-  if (tid == 64) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_w); }
+  if (tid == 64) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_w); tma_prefetch_desc(&tm_w_half); }
   cudaGridDependencySynchronize();  // programmatic launch: the previous kernel's results are complete
   tc_fence_before();
   __syncthreads();
@@ -91,9 +116,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   auto sA = [&](int s, int mt) { return smem_base + (uint32_t)s * kStageBytes + (uint32_t)mt * kATile; };
   auto sW = [&](int s) { return smem_base + (uint32_t)s * kStageBytes + 2 * kATile; };
 
-  // work items of this block: (vocabulary tile n, row block mb), all row blocks of a tile in a row
-  // so that the weight tile is read from HBM once and from L2 afterwards
-  const int n_items = p.n_tiles * p.m_blocks;
+  const int n_items = p.n_items;
   const int k_chunks = p.K / BK;
   int issued = 0;  // ring stages filled by the producer (for the drain)
 
@@ -103,15 +126,17 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       bool ok = true;
       int it = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const int n = item / p.m_blocks, mb = item - n * p.m_blocks;
+        const Item wi = decode_item(p, item);
+        const int mb = wi.mb;
         const int rows_left = p.M - mb * MB;
         const int m_tiles = rows_left > BM ? 2 : 1;
+        const uint32_t w_bytes = (uint32_t)wi.cols * BK * 2;
         for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
           const int s = it % kStages;
           if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_expect_tx(bar_full(s), kWTile + (uint32_t)m_tiles * kATile);
-          tma_load_2d(sW(s), &tm_w, kc * BK, n * BN, bar_full(s));
+          mbar_expect_tx(bar_full(s), w_bytes + (uint32_t)m_tiles * kATile);
+          tma_load_2d(sW(s), wi.cols == BN ? &tm_w : &tm_w_half, kc * BK, wi.col0, bar_full(s));
           for (int mt = 0; mt < m_tiles; ++mt)
             tma_load_2d(sA(s, mt), &tm_a, kc * BK, mb * MB + mt * BM, bar_full(s));
           issued = it + 1;
@@ -124,9 +149,9 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       bool ok = true;
       int it = 0, tile = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
-        const int n = item / p.m_blocks, mb = item - n * p.m_blocks;
-        (void)n;
-        const int m_tiles = (p.M - mb * MB) > BM ? 2 : 1;
+        const Item wi = decode_item(p, item);
+        const int m_tiles = (p.M - wi.mb * MB) > BM ? 2 : 1;
+        const uint32_t idesc = wi.cols == BN ? kIdesc : kIdescHalf;
         if (tile > 0) {  // the epilogue has taken the previous tile out of tensor memory
           ok = mbar_wait(bar_acc_empty, (tile - 1) & 1, abort_flag);
           if (!ok) break;
@@ -143,7 +168,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
 #pragma unroll
             for (int ks = 0; ks < BK / 16; ++ks)
               umma_bf16(tmem + (uint32_t)(mt * BN), ad + (uint64_t)((ks * 32) >> 4), wd + (uint64_t)((ks * 32) >> 4),
-                        kIdesc, (kc > 0 || ks > 0) ? 1u : 0u);
+                        idesc, (kc > 0 || ks > 0) ? 1u : 0u);
           }
           umma_commit(bar_empty(s));  // the stage is free once these MMAs have read it
         }
@@ -159,7 +184,8 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     bool ok = true;
     int tile = 0;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
-      const int n = item / p.m_blocks, mb = item - n * p.m_blocks;
+      const Item wi = decode_item(p, item);
+      const int mb = wi.mb;
       const int row = mb * MB + mt * BM + row_in_tile;
       const bool row_valid = row < p.M;
       ok = mbar_wait(bar_acc_full, tile & 1, abort_flag);
@@ -170,9 +196,9 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       float best_v = -INFINITY;
       int best_i = INT_MAX;
       if (group_used) {
-        const int col0 = n * BN;
+        const int col0 = wi.col0;
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = 0; c < wi.cols; c += 32) {
           uint32_t x[32];
           tmem_ld_x32(tmem + lane_addr + (uint32_t)(mt * BN + c), x);
           tmem_wait_ld();
@@ -262,9 +288,10 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  CUtensorMap tm_a, tm_w;
+  CUtensorMap tm_a, tm_w, tm_w_half;
   if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, BM) ||
-      !make_map_2d(&tm_w, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN))
+      !make_map_2d(&tm_w, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN) ||
+      !make_map_2d(&tm_w_half, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN / 2))
     return cudaErrorInvalidValue;
   Params p;
   p.M = rows;
@@ -277,9 +304,14 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
   p.aborts = tickets + 1;
   p.keys = reinterpret_cast<unsigned long long*>(tickets + 2);
   p.status = status;
-  const int items = p.n_tiles * p.m_blocks;
+  const int tiles = p.n_tiles * p.m_blocks;
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const int rem = tiles % grid;   // tiles of the last, incomplete round
+  const int split = (rem > 0 && 2 * rem <= grid) ? rem : 0;
+  p.full_items = tiles - split;
+  p.n_items = tiles + split;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(items < sm_count() ? items : sm_count()), 1, 1);
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmem;
   cfg.stream = stream;
@@ -288,7 +320,7 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, lm_head_argmax_kernel, tm_a, tm_w, p);
+  return cudaLaunchKernelEx(&cfg, lm_head_argmax_kernel, tm_a, tm_w, tm_w_half, p);
 }
 
 }  // namespace clv
