@@ -165,6 +165,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   constexpr uint32_t kTile = Cfg<MT>::kTile;
   constexpr uint32_t kHalf = kTile / 2;    // one 64-wide half of the head dimension: [BN keys][64 d]
   constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
+  constexpr uint32_t kIdescQKHalf = make_idesc(BM, BN / 2, false);  // a tile that holds one 64-key piece only
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
@@ -259,6 +260,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int pc_begin = (int)((int64_t)split * p_total / p.splits);
   const int pc_end = (int)((int64_t)(split + 1) * p_total / p.splits);
   const int n_tiles = (pc_end - pc_begin + PPT - 1) / PPT;
+  // pieces in local tile i: a range with an odd number of pieces ends in a tile of one piece, which
+  // gets a round of half the size (64 score columns, half the exponentials, half of P V)
+  auto tile_pieces = [&](int i) { return min(PPT, pc_end - pc_begin - i * PPT); };
   // local tile index of round r of slot s: MT == 2: r;  MT == 1: 2 r + s
   const int rounds0 = (MT == 2) ? n_tiles : (n_tiles + 1) / 2;
   const int rounds1 = (MT == 2) ? n_tiles : n_tiles / 2;
@@ -389,11 +393,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
+        const uint32_t idesc_qk = tile_pieces(i) == PPT ? kIdescQK : kIdescQKHalf;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
           const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
           const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
-          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
+          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), idesc_qk, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar_s_full(s));
         if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
@@ -414,8 +419,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
+          const int n_keys = tile_pieces(i) * PG;
 #pragma unroll
           for (int kk = 0; kk < BN / 16; ++kk) {
+            if (kk * 16 >= n_keys) break;
             umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                          (r > 0 || kk > 0) ? 1u : 0u);
           }
@@ -474,12 +481,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       uint32_t allow[BN / 32];
       int valid[PPT];
       bool cache_tile = false, short_tile = false;
+      const int nh = tile_pieces(i);       // 64-column halves of this tile that hold keys
 #pragma unroll
       for (int j = 0; j < PPT; ++j) {
         const int g = pc_begin + i * PPT + j;
-        if (g >= pc_end) {                 // the range ended inside this tile
-          valid[j] = 0;
-          allow[2 * j] = allow[2 * j + 1] = 0;
+        if (g >= pc_end) {                 // the range ended before this piece: it does not exist
+          valid[j] = PG;                   // (nothing of it is computed, loaded or cleared)
+          allow[2 * j] = allow[2 * j + 1] = 0xFFFFFFFFu;
         } else if (g < p_cache) {          // context piece: everything up to the context length
           cache_tile = true;
           valid[j] = min(PG, L - g * PG);
@@ -543,6 +551,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         float m0 = -INFINITY;
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
+          if (h >= nh) break;
           load_half(h);
 #pragma unroll
           for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
@@ -556,6 +565,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         sum = 0.f;
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
+          if (h >= nh) break;
           load_half(h);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -598,7 +608,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
 #pragma unroll
       for (int h = 0; h < NH; ++h)
-        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
+        if (h < nh) tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
       tmem_wait_st();
       l_run += sum;
 
