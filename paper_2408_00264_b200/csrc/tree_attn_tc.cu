@@ -29,6 +29,8 @@
 #include <cuda_fp16.h>
 #include <math.h>
 
+#include <type_traits>
+
 #include "clv_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tmem_access.cuh"
@@ -420,11 +422,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
           const int n_keys = tile_pieces(i) * PG;
+          if (n_keys == BN) {
 #pragma unroll
-          for (int kk = 0; kk < BN / 16; ++kk) {
-            if (kk * 16 >= n_keys) break;
-            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
-                         (r > 0 || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < BN / 16; ++kk)
+              umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                           (r > 0 || kk > 0) ? 1u : 0u);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < BN / 32; ++kk)
+              umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                           (r > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(bar_pv_done(s));
           if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
@@ -547,25 +554,26 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // from an overflow also lands here) the true maximum is taken from the scores - still
       // intact, because P is stored last - the reference replaced, O rescaled and the tile redone.
       uint32_t pk[NH * 32];
-      auto row_max = [&]() {
+      auto row_max_n = [&](auto halves) {
         float m0 = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          if (h >= nh) break;
+        for (int h = 0; h < decltype(halves)::value; ++h) {
           load_half(h);
 #pragma unroll
           for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
         }
         return m0 * p.scale_log2;  // scale > 0; -inf (no allowed key) stays -inf
       };
+      auto row_max = [&]() {
+        return nh == NH ? row_max_n(std::integral_constant<int, NH>{}) : row_max_n(std::integral_constant<int, 1>{});
+      };
       if (r == 0) m_ref = row_max();  // no reference yet: a cheap extra pass instead of a redo
       float sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      auto exp_pass = [&]() {
+      auto exp_pass_n = [&](auto halves) {
         sum = 0.f;
 #pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          if (h >= nh) break;
+        for (int h = 0; h < decltype(halves)::value; ++h) {
           load_half(h);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -575,6 +583,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             pk[h * 32 + j] = pack_bf16(p0, p1);
           }
         }
+      };
+      auto exp_pass = [&]() {
+        if (nh == NH) exp_pass_n(std::integral_constant<int, NH>{});
+        else exp_pass_n(std::integral_constant<int, 1>{});
       };
       exp_pass();
       const bool suspect = !(sum <= kRowSumLimit);  // also catches inf and NaN
@@ -608,7 +620,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
 #pragma unroll
       for (int h = 0; h < NH; ++h)
-        if (h < nh) tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
+        if (h == 0 || nh == NH)
+          tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
       tmem_wait_st();
       l_run += sum;
 
