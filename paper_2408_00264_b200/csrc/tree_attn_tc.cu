@@ -29,8 +29,6 @@
 #include <cuda_fp16.h>
 #include <math.h>
 
-#include <type_traits>
-
 #include "clv_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tmem_access.cuh"
@@ -167,7 +165,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   constexpr uint32_t kTile = Cfg<MT>::kTile;
   constexpr uint32_t kHalf = kTile / 2;    // one 64-wide half of the head dimension: [BN keys][64 d]
   constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
-  constexpr uint32_t kIdescQKHalf = make_idesc(BM, BN / 2, false);  // a tile that holds one 64-key piece only
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
@@ -262,9 +259,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int pc_begin = (int)((int64_t)split * p_total / p.splits);
   const int pc_end = (int)((int64_t)(split + 1) * p_total / p.splits);
   const int n_tiles = (pc_end - pc_begin + PPT - 1) / PPT;
-  // pieces in local tile i: a range with an odd number of pieces ends in a tile of one piece, which
-  // gets a round of half the size (64 score columns, half the exponentials, half of P V)
-  auto tile_pieces = [&](int i) { return min(PPT, pc_end - pc_begin - i * PPT); };
   // local tile index of round r of slot s: MT == 2: r;  MT == 1: 2 r + s
   const int rounds0 = (MT == 2) ? n_tiles : (n_tiles + 1) / 2;
   const int rounds1 = (MT == 2) ? n_tiles : n_tiles / 2;
@@ -395,12 +389,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
         const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
-        const uint32_t idesc_qk = tile_pieces(i) == PPT ? kIdescQK : kIdescQKHalf;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
           const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
           const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
-          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), idesc_qk, ks > 0 ? 1u : 0u);
+          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar_s_full(s));
         if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
@@ -421,17 +414,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
           tc_fence_after();
           const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
-          const int n_keys = tile_pieces(i) * PG;
-          if (n_keys == BN) {
 #pragma unroll
-            for (int kk = 0; kk < BN / 16; ++kk)
-              umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
-                           (r > 0 || kk > 0) ? 1u : 0u);
-          } else {
-#pragma unroll
-            for (int kk = 0; kk < BN / 32; ++kk)
-              umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
-                           (r > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < BN / 16; ++kk) {
+            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                         (r > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(bar_pv_done(s));
           if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
@@ -488,13 +474,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       uint32_t allow[BN / 32];
       int valid[PPT];
       bool cache_tile = false, short_tile = false;
-      const int nh = tile_pieces(i);       // 64-column halves of this tile that hold keys
 #pragma unroll
       for (int j = 0; j < PPT; ++j) {
         const int g = pc_begin + i * PPT + j;
-        if (g >= pc_end) {                 // the range ended before this piece: it does not exist
-          valid[j] = PG;                   // (nothing of it is computed, loaded or cleared)
-          allow[2 * j] = allow[2 * j + 1] = 0xFFFFFFFFu;
+        if (g >= pc_end) {                 // the range ended inside this tile
+          valid[j] = 0;
+          allow[2 * j] = allow[2 * j + 1] = 0;
         } else if (g < p_cache) {          // context piece: everything up to the context length
           cache_tile = true;
           valid[j] = min(PG, L - g * PG);
@@ -554,26 +539,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // from an overflow also lands here) the true maximum is taken from the scores - still
       // intact, because P is stored last - the reference replaced, O rescaled and the tile redone.
       uint32_t pk[NH * 32];
-      auto row_max_n = [&](auto halves) {
+      auto row_max = [&]() {
         float m0 = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < decltype(halves)::value; ++h) {
+        for (int h = 0; h < NH; ++h) {
           load_half(h);
 #pragma unroll
           for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
         }
         return m0 * p.scale_log2;  // scale > 0; -inf (no allowed key) stays -inf
       };
-      auto row_max = [&]() {
-        return nh == NH ? row_max_n(std::integral_constant<int, NH>{}) : row_max_n(std::integral_constant<int, 1>{});
-      };
       if (r == 0) m_ref = row_max();  // no reference yet: a cheap extra pass instead of a redo
       float sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      auto exp_pass_n = [&](auto halves) {
+      auto exp_pass = [&]() {
         sum = 0.f;
 #pragma unroll
-        for (int h = 0; h < decltype(halves)::value; ++h) {
+        for (int h = 0; h < NH; ++h) {
           load_half(h);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -583,10 +565,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             pk[h * 32 + j] = pack_bf16(p0, p1);
           }
         }
-      };
-      auto exp_pass = [&]() {
-        if (nh == NH) exp_pass_n(std::integral_constant<int, NH>{});
-        else exp_pass_n(std::integral_constant<int, 1>{});
       };
       exp_pass();
       const bool suspect = !(sum <= kRowSumLimit);  // also catches inf and NaN
@@ -620,8 +598,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
 #pragma unroll
       for (int h = 0; h < NH; ++h)
-        if (h == 0 || nh == NH)
-          tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
+        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
       tmem_wait_st();
       l_run += sum;
 
