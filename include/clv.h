@@ -60,6 +60,8 @@ enum {
 };
 
 #define CLV_MAX_NODES 128
+#define CLV_TREE_MAX_CAND 128 /* clv_build_token_tree: speculated sequences per tree */
+#define CLV_TREE_MAX_LEN 16   /* clv_build_token_tree: tokens per speculated sequence */
 #define CLV_HEAD_DIM 128
 #define CLV_PAGE_SIZE 64
 
@@ -182,6 +184,30 @@ clv_status clv_lm_head_argmax(const void* hidden, int64_t ld_hidden,
                               int32_t* argmax_ids,   /* [rows] */
                               int32_t* status,       /* [1]    */
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Token tree from speculated sequences (Sec. 2.1 and the caption of Fig. 2: the speculations are
+ * merged by prefix matching into a tree).  For every sequence b, n_cand candidate continuations
+ * cand[b][c][0 .. cand_len[b][c]) of the root token are merged: a node is a distinct non-empty
+ * prefix of some candidate; node 0 is the root and carries root_token[b] with parent -1.  Nodes
+ * are numbered by depth first and, within a depth, by the lowest candidate index that contains the
+ * prefix, so parent[i] < i and the result is unique.  Siblings carry distinct tokens by
+ * construction.  Slots n_nodes[b] .. node_cap-1 are padding: parent 0, token -1 (no target token
+ * matches them), so tokens/parent can be given to clv_tree_attn / clv_accept_walk with
+ * n_nodes = node_cap unchanged.  node_of[b][c][d] = the node of candidate c's prefix of length
+ * d+1, or -1 where d >= cand_len[b][c].
+ * All pointers are device pointers; int32; layouts [B], [B, n_cand, max_len], [B, n_cand],
+ * [B, node_cap], [B, node_cap], [B], [B, n_cand, max_len], [B].
+ * status[b] = CLV_ERR_TREE if a cand_len is outside [0, max_len] or the tree needs more than
+ * node_cap nodes: then n_nodes[b] = 1, the tree is the root plus padding, node_of is all -1.
+ * Limits: 1 <= n_cand <= CLV_TREE_MAX_CAND, 1 <= max_len <= CLV_TREE_MAX_LEN,
+ * 1 <= node_cap <= CLV_MAX_NODES (CLV_ERR_UNSUPPORTED beyond).  Nothing is launched on an error.
+ */
+clv_status clv_build_token_tree(int32_t batch, int32_t n_cand, int32_t max_len, int32_t node_cap,
+                                const int32_t* root_token, const int32_t* cand,
+                                const int32_t* cand_len,
+                                int32_t* tokens, int32_t* parent, int32_t* n_nodes,
+                                int32_t* node_of, int32_t* status, void* cuda_stream);
 
 /*
  * Greedy acceptance walk (Sec. 2.1 verification phase; Sec. 4.1).  Start at the root; at node cur

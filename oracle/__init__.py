@@ -136,6 +136,46 @@ def lm_head_argmax(hidden: np.ndarray, weight: np.ndarray, rows=None, want_logit
     return (ids, z) if want_logits else ids
 
 
+def build_token_tree(root_token, cand, cand_len, node_cap: int):
+    """Token tree by prefix matching (Sec. 2.1, caption of Fig. 2), written as the definition: the
+    nodes are the distinct non-empty prefixes of the candidate sequences, node 0 is the root; they
+    are numbered by depth and then by the first candidate that contains the prefix.  Plain Python
+    over a dictionary of prefixes (the sizes are tiny).  Returns tokens, parent [B, node_cap],
+    n_nodes [B], node_of [B, C, D], status [B]; padding slots are children of the root with token
+    -1; a tree that does not fit, or a length outside [0, D], gives status 7 and the bare root."""
+    cand = np.asarray(cand)
+    B, C, D = cand.shape
+    tokens = np.full((B, node_cap), -1, dtype=np.int32)
+    parent = np.zeros((B, node_cap), dtype=np.int32)
+    n_nodes = np.ones(B, dtype=np.int32)
+    node_of = np.full((B, C, D), -1, dtype=np.int32)
+    status = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        tokens[b, 0] = root_token[b]
+        parent[b, 0] = -1
+        lens = [int(x) for x in cand_len[b]]
+        if any(l < 0 or l > D for l in lens):
+            status[b] = 7
+            continue
+        first = {}                      # prefix (tuple of tokens) -> first candidate holding it
+        for c in range(C):
+            for d in range(lens[c]):
+                first.setdefault(tuple(int(t) for t in cand[b, c, :d + 1]), c)
+        order = sorted(first, key=lambda pre: (len(pre), first[pre]))
+        if 1 + len(order) > node_cap:
+            status[b] = 7
+            continue
+        index = {pre: 1 + i for i, pre in enumerate(order)}
+        for pre, i in index.items():
+            tokens[b, i] = pre[-1]
+            parent[b, i] = index[pre[:-1]] if len(pre) > 1 else 0
+        n_nodes[b] = 1 + len(order)
+        for c in range(C):
+            for d in range(lens[c]):
+                node_of[b, c, d] = index[tuple(int(t) for t in cand[b, c, :d + 1])]
+    return tokens, parent, n_nodes, node_of, status
+
+
 def accept_walk(parent, tokens, ids, path_cap: int):
     """Greedy acceptance walk; returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
     status [B])."""

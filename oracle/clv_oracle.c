@@ -17,6 +17,8 @@
  *   orc_argmax        - Sec. 4.2 (Table 1 note): temperature 0 is greedy decoding of the target.
  *   orc_lm_head_argmax - Sec. 3.1 (final norm + LM head give the logits) followed by Sec. 4.2's
  *                       greedy choice, the logit held in bf16 like a logits tensor.
+ *   build_token_tree (in the Python wrapper, plain loops over a dictionary) - Sec. 2.1 and the
+ *                       caption of Fig. 2: speculations merged by prefix matching into a tree.
  *   orc_accept_walk   - Sec. 2.1 verification phase (the target filters out wrong drafted
  *                       tokens; the output equals plain decoding) with the greedy rule of the
  *                       tree-sampling algorithm Sec. 4.1 adopts.

@@ -24,7 +24,7 @@ EXPORTS = (
     "clv_workspace_bytes", "clv_workspace_init", "clv_tree_attn", "clv_accept_argmax",
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
-    "clv_lm_head_argmax",
+    "clv_lm_head_argmax", "clv_build_token_tree",
 )
 
 
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.clv_accept_argmax_noalloc.argtypes = [vp, vp, i64, vp, vp]
         L.clv_lm_head_argmax.restype = i32
         L.clv_lm_head_argmax.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.clv_build_token_tree.restype = i32
+        L.clv_build_token_tree.argtypes = [i32, i32, i32, i32] + [vp] * 9
         L.clv_accept_walk.restype = i32
         L.clv_accept_walk.argtypes = [vp] * 9
         L.clv_kv_commit.restype = i32
@@ -185,6 +187,19 @@ def clv_accept_argmax_noalloc(shape, logits, ld, argmax_ids, stream=None, check=
                                            _stream(stream))
     if check:
         _check(code, "clv_accept_argmax_noalloc")
+    return code
+
+
+def clv_build_token_tree(root_token, cand, cand_len, tokens, parent, n_nodes, node_of, status,
+                         stream=None, check=True) -> int:
+    """cand int32 [B, n_cand, max_len], cand_len [B, n_cand], root_token [B]; outputs tokens and
+    parent [B, node_cap], n_nodes [B], node_of [B, n_cand, max_len], status [B] (all int32)."""
+    B, C, D = cand.shape
+    code = lib().clv_build_token_tree(int(B), int(C), int(D), int(tokens.shape[1]), _ptr(root_token),
+                                      _ptr(cand), _ptr(cand_len), _ptr(tokens), _ptr(parent),
+                                      _ptr(n_nodes), _ptr(node_of), _ptr(status), _stream(stream))
+    if check:
+        _check(code, "clv_build_token_tree")
     return code
 
 

@@ -150,6 +150,20 @@ clv_status clv_accept_argmax_noalloc(const clv_shape* shape, const void* logits,
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
+clv_status clv_build_token_tree(int32_t batch, int32_t n_cand, int32_t max_len, int32_t node_cap,
+                                const int32_t* root_token, const int32_t* cand, const int32_t* cand_len,
+                                int32_t* tokens, int32_t* parent, int32_t* n_nodes, int32_t* node_of,
+                                int32_t* status, void* cuda_stream) {
+  if (!root_token || !cand || !cand_len || !tokens || !parent || !n_nodes || !node_of || !status)
+    return CLV_ERR_NULL;
+  if (batch < 1 || n_cand < 1 || max_len < 1 || node_cap < 1) return CLV_ERR_SHAPE;
+  if (n_cand > CLV_TREE_MAX_CAND || max_len > CLV_TREE_MAX_LEN || node_cap > CLV_MAX_NODES)
+    return CLV_ERR_UNSUPPORTED;
+  cudaError_t e = launch_token_tree(batch, n_cand, max_len, node_cap, root_token, cand, cand_len, tokens,
+                                    parent, n_nodes, node_of, status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
 clv_status clv_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight,
                               int64_t ld_weight, int32_t rows, int32_t hidden_dim, int32_t vocab,
                               int32_t* argmax_ids, int32_t* status, void* workspace,

@@ -76,6 +76,11 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
                                   int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
                                   unsigned* tickets, cudaStream_t stream);
 
+// ---- token tree from speculated sequences -------------------------------------------------------
+cudaError_t launch_token_tree(int batch, int n_cand, int max_len, int node_cap, const int32_t* root_token,
+                              const int32_t* cand, const int32_t* cand_len, int32_t* tokens, int32_t* parent,
+                              int32_t* n_nodes, int32_t* node_of, int32_t* status, cudaStream_t stream);
+
 int sm_count();
 
 }  // namespace clv

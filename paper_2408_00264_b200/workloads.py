@@ -272,6 +272,28 @@ def make_logits(rows: int, vocab: int, ld: int, winner: np.ndarray, margin: floa
     return lg
 
 
+def make_candidates(batch: int, n_cand: int, max_len: int, vocab: int, seed: int, p_follow: float = 0.6):
+    """Speculated sequences with shared prefixes, as a draft model's top-k expansion produces them:
+    every candidate copies a random earlier candidate of the same sequence up to a random depth
+    (with probability ``p_follow``) and continues with uniform tokens below ``vocab``; lengths are
+    uniform in [0, max_len].  Returns root_token [B], cand [B, n_cand, max_len] (unused positions
+    hold -1) and cand_len [B, n_cand], all int32."""
+    rng = np.random.default_rng(np.random.SeedSequence(seed))
+    cand = np.full((batch, n_cand, max_len), -1, dtype=np.int32)
+    lens = rng.integers(0, max_len + 1, size=(batch, n_cand)).astype(np.int32)
+    for b in range(batch):
+        for c in range(n_cand):
+            n = int(lens[b, c])
+            seq = rng.integers(0, vocab, size=n)
+            if c > 0 and rng.random() < p_follow:
+                o = int(rng.integers(0, c))
+                k = int(rng.integers(0, min(n, int(lens[b, o])) + 1))
+                seq[:k] = cand[b, o, :k]
+            cand[b, c, :n] = seq
+    root = rng.integers(0, vocab, size=batch).astype(np.int32)
+    return root, cand, lens
+
+
 def make_lm_head(rows: int, hidden_dim: int, vocab: int, seed: int, planted: float = 12.0):
     """Inputs of the LM head for ``rows`` tree nodes: hidden states N(0,1) and a weight matrix
     N(0, 1/hidden_dim) (so that logits are about N(0,1)), both rounded to bf16 and returned as bit
