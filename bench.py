@@ -36,6 +36,37 @@ ROTATE = 4   # distinct input sets cycled between steps: 4 x 138 MB > 2 x L2 (12
 NCU_TRAFFIC = {("C3", "tree_attn"): 71.7e6, ("C3", "accept_argmax"): 65.9e6}
 
 
+def time_token_tree(batch, node_cap, dev):
+    """clv_build_token_tree for `batch` sequences, 32 speculated sequences of up to 6 tokens each
+    (latency bound: one small block per sequence): microseconds per launch, replayed from a graph."""
+    import torch
+    from paper_2408_00264_b200 import binding as clv
+    from paper_2408_00264_b200 import workloads as W
+    root, cand, lens = W.make_candidates(batch, 32, 6, 6, seed=W.BASE_SEED + 9)
+    t = lambda a: torch.from_numpy(a).to(dev)  # noqa: E731
+    ins = (t(root), t(cand), t(lens))
+    outs = [torch.zeros(s, dtype=torch.int32, device=dev)
+            for s in ((batch, node_cap), (batch, node_cap), (batch,), (batch, 32, 6), (batch,))]
+    for _ in range(3):
+        clv.clv_build_token_tree(*ins, *outs)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(8):
+            clv.clv_build_token_tree(*ins, *outs)
+    g.replay()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    a.record(cur)
+    for _ in range(20):
+        g.replay()
+    b.record(cur)
+    torch.cuda.synchronize()
+    return {"batch": batch, "n_cand": 32, "max_len": 6, "node_cap": node_cap,
+            "us": a.elapsed_time(b) / 160 * 1e3, "nodes": outs[2].cpu().tolist()[:4]}
+
+
 def time_lm_head(rows, hidden, vocab, dev, args):
     """clv_lm_head_argmax on `rows` tree nodes: microseconds per launch (CUDA events, launches
     replayed from a CUDA graph over two copies of the weight matrix, 2 x 1.05 GB at vocabulary
@@ -368,8 +399,10 @@ def run_clv(args):
 
     # ---- the step before the argmax: LM head fused with the greedy choice (rank 0 only) ---------
     lm_head = None
+    tree_us = None
     if rank == 0 and not args.no_lm_head:
         lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
+        tree_us = time_token_tree(B, N, dev)
 
     # ---- max over ranks ------------------------------------------------------------------------
     step_ms, e2e_ms, job_bytes = reduce_over_ranks(dist, dev, step_ms, e2e_ms, float(nbytes["total"]))
@@ -400,7 +433,7 @@ def run_clv(args):
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
-        "next_rows": {"lm_head_argmax": lm_head},
+        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us},
         "gpu_launches": 4 * args.steps,
         "clocks": clocks.summary(),
     }
