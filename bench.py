@@ -402,7 +402,7 @@ def run_clv(args):
     tree_us = None
     if rank == 0 and not args.no_lm_head:
         lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
-        tree_us = time_token_tree(B, N, dev)
+        tree_us = time_token_tree(B, 128, dev)
 
     # ---- max over ranks ------------------------------------------------------------------------
     step_ms, e2e_ms, job_bytes = reduce_over_ranks(dist, dev, step_ms, e2e_ms, float(nbytes["total"]))

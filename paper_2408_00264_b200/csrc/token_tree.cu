@@ -30,14 +30,17 @@ struct Params {
 
 __global__ void __launch_bounds__(kThreads) token_tree_kernel(Params p) {
   // rep[d][c]: lowest candidate whose first d+1 tokens equal those of candidate c (-1: c is shorter)
-  __shared__ short s_rep[kMaxLen][kMaxCand];
+  __shared__ int s_rep[kMaxLen][kMaxCand];
   __shared__ short s_node[kMaxLen][kMaxCand];   // node number of (depth d, candidate c) if c is its own rep
+  __shared__ int s_cand[kMaxCand * kMaxLen];     // this sequence's candidates, [c][d]
   __shared__ int s_len[kMaxCand];
   __shared__ int s_total;
   const int b = blockIdx.x, tid = threadIdx.x;
   const int C = p.n_cand, D = p.max_len;
   cudaGridDependencySynchronize();  // programmatic launch: the previous kernel's results are complete
-  const int32_t* cand = p.cand + (int64_t)b * C * D;
+  const int32_t* cand_g = p.cand + (int64_t)b * C * D;
+  for (int w = tid; w < C * D; w += kThreads) s_cand[w] = cand_g[w];
+  const int* cand = s_cand;
   bool bad = false;
   for (int c = tid; c < C; c += kThreads) {
     const int len = p.cand_len[(int64_t)b * C + c];
@@ -48,18 +51,23 @@ __global__ void __launch_bounds__(kThreads) token_tree_kernel(Params p) {
 
   // ---- prefix matching, one depth after the other: candidate c' shares c's prefix of length d+1
   //      iff it shared the prefix of length d and carries the same token at depth d --------------
+  // Every candidate's scan over the earlier ones is shared by `parts` threads (interleaved), which
+  // combine with a shared-memory minimum.
+  const int parts = max(1, kThreads / C);
   for (int d = 0; d < D; ++d) {
-    for (int c = tid; c < C; c += kThreads) {
-      int rep = -1;
-      if (d < s_len[c]) {
-        const int tok = cand[c * D + d];
-        const int up = d == 0 ? 0 : s_rep[d - 1][c];
-        rep = c;
-        for (int o = 0; o < c; ++o) {
-          if (d < s_len[o] && (d == 0 || s_rep[d - 1][o] == up) && cand[o * D + d] == tok) { rep = o; break; }
-        }
+    for (int c = tid; c < C; c += kThreads) s_rep[d][c] = d < s_len[c] ? c : -1;
+    __syncthreads();
+    for (int w = tid; w < C * parts; w += kThreads) {
+      const int c = w / parts, part = w - c * parts;
+      if (d >= s_len[c]) continue;
+      const int tok = cand[c * D + d];
+      const int up = d == 0 ? 0 : s_rep[d - 1][c];
+      int rep = c;
+      for (int o = part; o < c; o += parts) {
+        const bool match = d < s_len[o] && (d == 0 || s_rep[d - 1][o] == up) && cand[o * D + d] == tok;
+        if (match && o < rep) rep = o;
       }
-      s_rep[d][c] = (short)rep;
+      if (rep < c) atomicMin(&s_rep[d][c], rep);
     }
     __syncthreads();
   }
