@@ -63,9 +63,12 @@ __global__ void __launch_bounds__(kThreads) token_tree_kernel(Params p) {
       const int tok = cand[c * D + d];
       const int up = d == 0 ? 0 : s_rep[d - 1][c];
       int rep = c;
+      const int* prev = s_rep[d == 0 ? 0 : d - 1];
+#pragma unroll 4
       for (int o = part; o < c; o += parts) {
-        const bool match = d < s_len[o] && (d == 0 || s_rep[d - 1][o] == up) && cand[o * D + d] == tok;
-        if (match && o < rep) rep = o;
+        // all three loads are issued whatever they return, so that the iterations overlap
+        const bool match = (d < s_len[o]) & ((d == 0) | (prev[o] == up)) & (cand[o * D + d] == tok);
+        rep = (match && o < rep) ? o : rep;
       }
       if (rep < c) atomicMin(&s_rep[d][c], rep);
     }
