@@ -208,7 +208,6 @@ constexpr size_t kStaticTicketBytes = sizeof(unsigned) * (size_t)kStaticMaxRows;
 constexpr size_t kStaticBytes = kStaticTicketBytes + sizeof(unsigned long long) * (size_t)kStaticMaxKeys;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 
-constexpr int kMaxDevices = 64;
 unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device
 }  // namespace
 

@@ -83,4 +83,15 @@ cudaError_t launch_token_tree(int batch, int n_cand, int max_len, int node_cap, 
 
 int sm_count();
 
+// Per-device one-time set-up (function attributes belong to the device that is current when they
+// are set): true the first time it is called with `done` on the current device.
+constexpr int kMaxDevices = 64;
+inline bool first_call_on_device(bool (&done)[kMaxDevices]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return true;
+  if (done[dev]) return false;
+  done[dev] = true;
+  return true;
+}
+
 }  // namespace clv

@@ -281,12 +281,11 @@ bool lm_head_supported(int rows, int hidden, int vocab) {
 cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
                                   int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
                                   unsigned* tickets, cudaStream_t stream) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {};
+  if (first_call_on_device(attr_set)) {
     cudaError_t e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kSmem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   CUtensorMap tm_a, tm_w, tm_w_half;
   if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, BM) ||

@@ -461,12 +461,11 @@ cudaError_t launch_tree_attn(const AttnPlan& plan, const clv_shape& s, const clv
                              const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
                              float* lse, int32_t* status, unsigned* tickets, void* scratch,
                              cudaStream_t stream) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};
+  if (first_call_on_device(attr_done)) {
     cudaError_t e = cudaFuncSetAttribute(tree_attn_mma_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   Params p;
   p.q = static_cast<const uint16_t*>(q);

@@ -836,15 +836,14 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = G * s.n_nodes;
   const int mt = rows > BM ? 2 : 1;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {};
+  if (first_call_on_device(attr_done)) {
     cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)Cfg<1>::kSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tree_attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)Cfg<2>::kSmem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt;
   const uint64_t cache_rows = c.paged ? (uint64_t)c.n_pages * CLV_PAGE_SIZE : (uint64_t)s.batch * c.cap_tokens;
