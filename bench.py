@@ -426,6 +426,7 @@ def run_clv(args):
         "frac_of_hbm_peak": {"of_%s_%.0f_GBps" % (peak_kind, peak): value / world / peak,
                              "of_nominal_8000_GBps": value / world / NOMINAL_HBM_GBS},
         "call_us": call_us, "launch_mode": "per-call" if graphs is None else "cuda-graph replay",
+        "step_schedule": "clv_tree_attn, clv_accept_argmax, clv_accept_walk_commit (walk and commit in one launch) on one stream",
         "algorithmic_bytes": nbytes,
         "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak,
                      "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
@@ -434,7 +435,7 @@ def run_clv(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
         "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us},
-        "gpu_launches": 4 * args.steps,
+        "gpu_launches": 3 * args.steps,   # attention, argmax, walk + commit in one launch
         "clocks": clocks.summary(),
     }
     if not args.no_cpu_baseline and world == 1:

@@ -162,6 +162,21 @@ clv_status clv_accept_argmax_noalloc(const clv_shape* shape,
                                      void* cuda_stream);
 
 /*
+ * clv_accept_walk followed by clv_kv_commit in one launch (Sec. 2.1: the verification keeps the
+ * drafts the target agrees with, and the cache must afterwards equal plain decoding's): a thread
+ * block per sequence walks the tree and then copies the accepted rows.  Arguments, results, error
+ * codes and per-sequence statuses are those of the two calls (walk_status as clv_accept_walk's
+ * status, commit_status as clv_kv_commit's); the result is identical to calling them in turn.
+ */
+clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* cache,
+                                  const int32_t* parent, const int32_t* tokens,
+                                  const int32_t* argmax_ids,
+                                  const void* k_tree, const void* v_tree, const int32_t* ctx_len,
+                                  int32_t* accept_len, int32_t* accept_idx, int32_t* next_token,
+                                  int32_t* ctx_len_out, int32_t* walk_status, int32_t* commit_status,
+                                  void* cuda_stream);
+
+/*
  * LM head fused with the greedy choice (Sec. 3.1: the target's final norm and LM head produce the
  * logits of every tree node; Sec. 4.2: greedy decoding at temperature 0):
  *   argmax_ids[r] = the lowest v that maximises round_bf16(sum_k hidden[r][k] * weight[v][k]),

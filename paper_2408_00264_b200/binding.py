@@ -24,7 +24,7 @@ EXPORTS = (
     "clv_workspace_bytes", "clv_workspace_init", "clv_tree_attn", "clv_accept_argmax",
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
-    "clv_lm_head_argmax", "clv_build_token_tree",
+    "clv_lm_head_argmax", "clv_build_token_tree", "clv_accept_walk_commit",
 )
 
 
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.clv_accept_argmax_noalloc.argtypes = [vp, vp, i64, vp, vp]
         L.clv_lm_head_argmax.restype = i32
         L.clv_lm_head_argmax.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.clv_accept_walk_commit.restype = i32
+        L.clv_accept_walk_commit.argtypes = [vp] * 15
         L.clv_build_token_tree.restype = i32
         L.clv_build_token_tree.argtypes = [i32, i32, i32, i32] + [vp] * 9
         L.clv_accept_walk.restype = i32
@@ -187,6 +189,19 @@ def clv_accept_argmax_noalloc(shape, logits, ld, argmax_ids, stream=None, check=
                                            _stream(stream))
     if check:
         _check(code, "clv_accept_argmax_noalloc")
+    return code
+
+
+def clv_accept_walk_commit(shape, cache, parent, tokens, argmax_ids, k_tree, v_tree, ctx_len, accept_len,
+                           accept_idx, next_token, ctx_len_out, walk_status, commit_status, stream=None,
+                           check=True) -> int:
+    code = lib().clv_accept_walk_commit(_ref(shape), _ref(cache), _ptr(parent), _ptr(tokens),
+                                        _ptr(argmax_ids), _ptr(k_tree), _ptr(v_tree), _ptr(ctx_len),
+                                        _ptr(accept_len), _ptr(accept_idx), _ptr(next_token),
+                                        _ptr(ctx_len_out), _ptr(walk_status), _ptr(commit_status),
+                                        _stream(stream))
+    if check:
+        _check(code, "clv_accept_walk_commit")
     return code
 
 

@@ -150,6 +150,39 @@ clv_status clv_accept_argmax_noalloc(const clv_shape* shape, const void* logits,
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
+static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + nb && y < x + na;
+}
+
+clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* cache,
+                                  const int32_t* parent, const int32_t* tokens, const int32_t* argmax_ids,
+                                  const void* k_tree, const void* v_tree, const int32_t* ctx_len,
+                                  int32_t* accept_len, int32_t* accept_idx, int32_t* next_token,
+                                  int32_t* ctx_len_out, int32_t* walk_status, int32_t* commit_status,
+                                  void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  st = check_cache(cache);
+  if (st != CLV_OK) return st;
+  if (!parent || !tokens || !argmax_ids || !k_tree || !v_tree || !ctx_len || !accept_len || !accept_idx ||
+      !next_token || !ctx_len_out || !walk_status || !commit_status)
+    return CLV_ERR_NULL;
+  if (!aligned16(k_tree) || !aligned16(v_tree)) return CLV_ERR_ALIGN;
+  if (shape->path_cap < 1) return CLV_ERR_SHAPE;
+  const size_t row = (size_t)shape->n_kv_heads * CLV_HEAD_DIM * 2;
+  const size_t tree_bytes = (size_t)shape->batch * shape->n_nodes * row;
+  const size_t cache_bytes = cache->paged ? (size_t)cache->n_pages * CLV_PAGE_SIZE * row
+                                          : (size_t)shape->batch * cache->cap_tokens * row;
+  if (overlaps(k_tree, tree_bytes, cache->k, cache_bytes) || overlaps(k_tree, tree_bytes, cache->v, cache_bytes) ||
+      overlaps(v_tree, tree_bytes, cache->k, cache_bytes) || overlaps(v_tree, tree_bytes, cache->v, cache_bytes))
+    return CLV_ERR_UNSUPPORTED;
+  cudaError_t e = launch_walk_commit(*shape, *cache, parent, tokens, argmax_ids, k_tree, v_tree, ctx_len,
+                                     accept_len, accept_idx, next_token, ctx_len_out, walk_status,
+                                     commit_status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
 clv_status clv_build_token_tree(int32_t batch, int32_t n_cand, int32_t max_len, int32_t node_cap,
                                 const int32_t* root_token, const int32_t* cand, const int32_t* cand_len,
                                 int32_t* tokens, int32_t* parent, int32_t* n_nodes, int32_t* node_of,
@@ -193,11 +226,6 @@ clv_status clv_accept_walk(const clv_shape* shape, const int32_t* parent, const 
   cudaError_t e = launch_walk(*shape, parent, tokens, argmax_ids, accept_len, accept_idx, next_token,
                               status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
-}
-
-static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
-  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
-  return x < y + nb && y < x + na;
 }
 
 clv_status clv_kv_commit(const clv_shape* shape, const clv_kv_cache* cache, const void* k_tree,

@@ -47,6 +47,12 @@ cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void*
                           const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
                           cudaStream_t stream);
 
+cudaError_t launch_walk_commit(const clv_shape& s, const clv_kv_cache& c, const int32_t* parent,
+                               const int32_t* tokens, const int32_t* ids, const void* k_tree,
+                               const void* v_tree, const int32_t* ctx_len, int32_t* accept_len,
+                               int32_t* accept_idx, int32_t* next_token, int32_t* ctx_len_out,
+                               int32_t* walk_status, int32_t* commit_status, cudaStream_t stream);
+
 // ---- tree attention ---------------------------------------------------------------------------
 struct AttnPlan {
   int m_tiles;   // row tiles per (sequence, kv head): ceil(G*N / rows per tile)

@@ -9,18 +9,18 @@ namespace clv {
 namespace {
 
 // ------------------------------------------------------------------------------------ walk
-__global__ void __launch_bounds__(32) walk_kernel(int N, int path_cap, const int32_t* parent,
-                                                  const int32_t* tokens, const int32_t* ids,
-                                                  int32_t* accept_len, int32_t* accept_idx,
-                                                  int32_t* next_token, int32_t* status) {
-  __shared__ int sp[CLV_MAX_NODES], st[CLV_MAX_NODES], si[CLV_MAX_NODES], path[CLV_MAX_NODES];
-  const int b = blockIdx.x, lane = threadIdx.x;
+struct WalkSmem {
+  int sp[CLV_MAX_NODES], st[CLV_MAX_NODES], si[CLV_MAX_NODES], path[CLV_MAX_NODES];
+};
+
+// The walk of sequence b by one warp; returns the accepted length (0 if the tree is malformed).
+// The path is left in sm.path[0 .. len) for the caller (visible after a __syncwarp / barrier).
+__device__ __forceinline__ int walk_sequence(WalkSmem& sm, int b, int lane, int N, int path_cap,
+                                             const int32_t* parent, const int32_t* tokens,
+                                             const int32_t* ids, int32_t* accept_len, int32_t* accept_idx,
+                                             int32_t* next_token, int32_t* status) {
+  int* sp = sm.sp; int* st = sm.st; int* si = sm.si; int* path = sm.path;
   const int64_t o = (int64_t)b * N;
-  // Launched with programmatic stream serialisation: this grid may be set up while the previous
-  // kernel of the stream is still draining, so wait for that kernel's results here, and let the
-  // next kernel (the commit) start its own set-up right away.
-  cudaGridDependencySynchronize();
-  cudaTriggerProgrammaticLaunchCompletion();
   bool bad = false;
   for (int i = lane; i < N; i += 32) {
     const int p = parent[o + i];
@@ -58,6 +58,21 @@ __global__ void __launch_bounds__(32) walk_kernel(int N, int path_cap, const int
     next_token[b] = bad ? -1 : si[cur];
     status[b] = bad ? CLV_ERR_TREE : CLV_OK;
   }
+  return len;
+}
+
+__global__ void __launch_bounds__(32) walk_kernel(int N, int path_cap, const int32_t* parent,
+                                                  const int32_t* tokens, const int32_t* ids,
+                                                  int32_t* accept_len, int32_t* accept_idx,
+                                                  int32_t* next_token, int32_t* status) {
+  __shared__ WalkSmem sm;
+  // Launched with programmatic stream serialisation: this grid may be set up while the previous
+  // kernel of the stream is still draining, so wait for that kernel's results here, and let the
+  // next kernel (the commit) start its own set-up right away.
+  cudaGridDependencySynchronize();
+  cudaTriggerProgrammaticLaunchCompletion();
+  walk_sequence(sm, blockIdx.x, threadIdx.x, N, path_cap, parent, tokens, ids, accept_len, accept_idx,
+                next_token, status);
 }
 
 // ------------------------------------------------------------------------------------ commit
@@ -76,13 +91,17 @@ struct CommitParams {
   int row_vec;  // 16-byte vectors per token row: Hkv * 128 * 2 / 16
 };
 
-__global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
-  __shared__ int s_src[CLV_MAX_NODES];
-  __shared__ long long s_dst[CLV_MAX_NODES];  // destination token row (global row index)
-  __shared__ int s_ok;
-  const int b = blockIdx.x, tid = threadIdx.x;
-  cudaGridDependencySynchronize();  // programmatic launch: the walk's outputs are complete after this
-  cudaTriggerProgrammaticLaunchCompletion();  // a following kernel may set up; it waits for this grid itself
+struct CommitSmem {
+  int src[CLV_MAX_NODES];
+  long long dst[CLV_MAX_NODES];  // destination token row (global row index)
+  int ok;
+};
+
+// The commit of sequence b by one thread block (accept_len / accept_idx are read from memory).
+__device__ __forceinline__ void commit_sequence(CommitSmem& sm, const CommitParams& p, int b, int tid) {
+  int* s_src = sm.src;
+  long long* s_dst = sm.dst;
+  int& s_ok = sm.ok;
   const int L = p.ctx_len[b];
   const int len = p.accept_len[b];
   if (tid == 0) s_ok = (L >= 0 && len >= 0 && len <= p.path_cap && len <= CLV_MAX_NODES) ? 1 : 0;
@@ -123,6 +142,36 @@ __global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
   if (tid == 0) { p.ctx_len_out[b] = L + len; p.status[b] = CLV_OK; }
 }
 
+__global__ void __launch_bounds__(256) commit_kernel(CommitParams p) {
+  __shared__ CommitSmem sm;
+  cudaGridDependencySynchronize();  // programmatic launch: the walk's outputs are complete after this
+  cudaTriggerProgrammaticLaunchCompletion();  // a following kernel may set up; it waits for this grid itself
+  commit_sequence(sm, p, blockIdx.x, threadIdx.x);
+}
+
+// Walk and commit of a sequence in one launch: warp 0 walks, then the whole block copies the rows.
+struct WalkArgs {
+  int N, path_cap;
+  const int32_t* parent;
+  const int32_t* tokens;
+  const int32_t* ids;
+  int32_t* accept_len;
+  int32_t* accept_idx;
+  int32_t* next_token;
+  int32_t* status;
+};
+__global__ void __launch_bounds__(256) walk_commit_kernel(WalkArgs w, CommitParams p) {
+  __shared__ WalkSmem wsm;
+  __shared__ CommitSmem csm;
+  cudaGridDependencySynchronize();
+  cudaTriggerProgrammaticLaunchCompletion();
+  if (threadIdx.x < 32)
+    walk_sequence(wsm, blockIdx.x, threadIdx.x, w.N, w.path_cap, w.parent, w.tokens, w.ids, w.accept_len,
+                  w.accept_idx, w.next_token, w.status);
+  __syncthreads();  // the walk's results, written by this block, are visible to all of it
+  commit_sequence(csm, p, blockIdx.x, threadIdx.x);
+}
+
 }  // namespace
 
 cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
@@ -141,10 +190,10 @@ cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t
                             accept_idx, next_token, status);
 }
 
-cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void* k_tree,
-                          const void* v_tree, const int32_t* accept_idx, const int32_t* accept_len,
-                          const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
-                          cudaStream_t stream) {
+namespace {
+CommitParams commit_params(const clv_shape& s, const clv_kv_cache& c, const void* k_tree, const void* v_tree,
+                           const int32_t* accept_idx, const int32_t* accept_len, const int32_t* ctx_len,
+                           int32_t* ctx_len_out, int32_t* status) {
   CommitParams p;
   p.kc = static_cast<uint4*>(c.k);
   p.vc = static_cast<uint4*>(c.v);
@@ -163,6 +212,15 @@ cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void*
   p.n_pages = c.n_pages;
   p.max_pages = c.max_pages_per_seq;
   p.row_vec = s.n_kv_heads * CLV_HEAD_DIM * 2 / 16;
+  return p;
+}
+}  // namespace
+
+cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void* k_tree,
+                          const void* v_tree, const int32_t* accept_idx, const int32_t* accept_len,
+                          const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
+                          cudaStream_t stream) {
+  const CommitParams p = commit_params(s, c, k_tree, v_tree, accept_idx, accept_len, ctx_len, ctx_len_out, status);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)s.batch, 1, 1);
   cfg.blockDim = dim3(256, 1, 1);
@@ -173,6 +231,35 @@ cudaError_t launch_commit(const clv_shape& s, const clv_kv_cache& c, const void*
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, commit_kernel, p);
+}
+
+cudaError_t launch_walk_commit(const clv_shape& s, const clv_kv_cache& c, const int32_t* parent,
+                               const int32_t* tokens, const int32_t* ids, const void* k_tree,
+                               const void* v_tree, const int32_t* ctx_len, int32_t* accept_len,
+                               int32_t* accept_idx, int32_t* next_token, int32_t* ctx_len_out,
+                               int32_t* walk_status, int32_t* commit_status, cudaStream_t stream) {
+  const CommitParams p =
+      commit_params(s, c, k_tree, v_tree, accept_idx, accept_len, ctx_len, ctx_len_out, commit_status);
+  WalkArgs w;
+  w.N = s.n_nodes;
+  w.path_cap = s.path_cap;
+  w.parent = parent;
+  w.tokens = tokens;
+  w.ids = ids;
+  w.accept_len = accept_len;
+  w.accept_idx = accept_idx;
+  w.next_token = next_token;
+  w.status = walk_status;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)s.batch, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, walk_commit_kernel, w, p);
 }
 
 }  // namespace clv

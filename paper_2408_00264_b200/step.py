@@ -73,9 +73,19 @@ class VerifyStep:
                           self.ctx_len_out if ctx_len_out is None else ctx_len_out,
                           self.status[2], stream)
 
-    def run(self, stream=None):
-        """One whole verify step (four launches, stream-ordered)."""
+    def accept_walk_commit(self, stream=None, ctx_len_out: Optional[torch.Tensor] = None):
+        clv.clv_accept_walk_commit(self.shape, self.cache, self.parent, self.tokens, self.ids, self.k_tree,
+                                   self.v_tree, self.ctx_len, self.accept_len, self.accept_idx,
+                                   self.next_token, self.ctx_len_out if ctx_len_out is None else ctx_len_out,
+                                   self.status[1], self.status[2], stream)
+
+    def run(self, stream=None, fused_tail: bool = True):
+        """One whole verify step, stream-ordered: attention, argmax, then the walk and the commit
+        (in one launch unless ``fused_tail`` is False)."""
         self.tree_attn(stream)
         self.accept_argmax(stream)
-        self.accept_walk(stream)
-        self.kv_commit(stream)
+        if fused_tail:
+            self.accept_walk_commit(stream)
+        else:
+            self.accept_walk(stream)
+            self.kv_commit(stream)

@@ -78,10 +78,12 @@ def full_step(clv, oracle, w, rows=None):
     # a second step on fresh buffers gives bit-identical outputs (no stale workspace state)
     st2 = make_step(w)
     st2.workspace = st.workspace
-    st2.run()
+    st2.run(fused_tail=False)   # the walk and the commit as two launches: same results as the fused one
     torch.cuda.synchronize()
     assert torch.equal(st2.ids, st.ids) and torch.equal(st2.accept_idx, st.accept_idx)
-    assert torch.equal(st2.k_cache, st.k_cache)
+    assert torch.equal(st2.accept_len, st.accept_len) and torch.equal(st2.next_token, st.next_token)
+    assert torch.equal(st2.ctx_len_out, st.ctx_len_out) and torch.equal(st2.status, st.status)
+    assert torch.equal(st2.k_cache, st.k_cache) and torch.equal(st2.v_cache, st.v_cache)
     assert_attn_close(bits(st2.out), W.bf16_bits_to_f64(bits(st.out)), "repeat")
     return alen
 
@@ -359,6 +361,46 @@ def test_commit_edges_alias_and_capacity(clv, oracle, paged):
     assert np.array_equal(st.ctx_len.cpu().numpy(), new_len)
     assert np.array_equal(st.status[2].cpu().numpy(), s2)
     assert np.array_equal(bits(st.k_cache), kc) and np.array_equal(bits(st.v_cache), vc)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_walk_commit_in_one_launch_with_errors(clv, oracle, paged):
+    # malformed trees, a path longer than path_cap and a cache without room: the fused call gives
+    # what the two calls give, sequence by sequence, and what the checker gives
+    cfg = W.small_config(batch=6, n_q_heads=4, n_kv_heads=2, ctx=(10, 200), n_nodes=20, vocab=64,
+                         paged=paged, seed=W.BASE_SEED + 31)
+    w = W.generate(cfg)
+    w.parent[1, 5] = 7            # parent after child
+    w.parent[2, 0] = 0            # root is not a root
+    w.parent[3, 4] = -1           # a second root: the walk refuses, attention would not
+    if paged:
+        w.block_table[4, :] = -1                 # sequence 4 has no page for its accepted rows
+    else:
+        w.ctx_len[4] = w.cap_tokens              # ... or no room left in its cache rows
+    results = []
+    for fused in (True, False):
+        st = make_step(w)
+        st.accept_argmax()
+        if fused:
+            st.accept_walk_commit()
+        else:
+            st.accept_walk()
+            st.kv_commit()
+        torch.cuda.synchronize()
+        results.append(st)
+    a, b = results
+    for name in ("accept_len", "accept_idx", "next_token", "ctx_len_out", "k_cache", "v_cache"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+    assert torch.equal(a.status[1:], b.status[1:])
+    ids = oracle.argmax(w.logits, w.cfg.vocab)
+    alen, aidx, nxt, s1 = oracle.accept_walk(w.parent, w.tokens, ids, w.path_cap)
+    kc, vc, new_len, s2 = oracle.kv_commit(w.k_cache, w.v_cache, w.k_tree, w.v_tree, aidx, alen, w.ctx_len,
+                                           block_table=w.block_table)
+    assert np.array_equal(a.accept_len.cpu().numpy(), alen) and np.array_equal(a.accept_idx.cpu().numpy(), aidx)
+    assert np.array_equal(a.status[1].cpu().numpy(), s1) and np.array_equal(a.status[2].cpu().numpy(), s2)
+    assert np.array_equal(a.ctx_len_out.cpu().numpy(), new_len)
+    assert np.array_equal(bits(a.k_cache), kc) and np.array_equal(bits(a.v_cache), vc)
+    assert s1.tolist()[1:4] == [7, 7, 7] and s2.tolist()[4] == 7 and s2.tolist()[0] == 0
 
 
 def test_guard_bands_untouched(clv, oracle):
