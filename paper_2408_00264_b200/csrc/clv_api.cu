@@ -324,14 +324,11 @@ clv_status clv_verify_step_host(const clv_shape* shape, const clv_kv_cache* cach
   st = clv_accept_argmax(shape, d + L.logits, in->ld, reinterpret_cast<int32_t*>(d + L.ids),
                          workspace, workspace_bytes, cuda_stream);
   if (st != CLV_OK) return st;
-  st = clv_accept_walk(shape, reinterpret_cast<int32_t*>(d + L.parent),
-                       reinterpret_cast<int32_t*>(d + L.tokens), reinterpret_cast<int32_t*>(d + L.ids),
-                       reinterpret_cast<int32_t*>(d + L.alen), reinterpret_cast<int32_t*>(d + L.aidx),
-                       reinterpret_cast<int32_t*>(d + L.next), dstat + B, cuda_stream);
-  if (st != CLV_OK) return st;
-  st = clv_kv_commit(shape, cache, d + L.k_tree, d + L.v_tree, reinterpret_cast<int32_t*>(d + L.aidx),
-                     reinterpret_cast<int32_t*>(d + L.alen), ctx_len, ctx_len, dstat + 2 * B,
-                     cuda_stream);
+  st = clv_accept_walk_commit(shape, cache, reinterpret_cast<int32_t*>(d + L.parent),
+                              reinterpret_cast<int32_t*>(d + L.tokens), reinterpret_cast<int32_t*>(d + L.ids),
+                              d + L.k_tree, d + L.v_tree, ctx_len, reinterpret_cast<int32_t*>(d + L.alen),
+                              reinterpret_cast<int32_t*>(d + L.aidx), reinterpret_cast<int32_t*>(d + L.next),
+                              ctx_len, dstat + B, dstat + 2 * B, cuda_stream);
   if (st != CLV_OK) return st;
   CLV_COPY(out->out, d + L.out, qb, cudaMemcpyDeviceToHost);
   CLV_COPY(out->argmax_ids, d + L.ids, B * N * 4, cudaMemcpyDeviceToHost);
