@@ -115,7 +115,7 @@ __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t u) {
 // normalised weights divided by the rows' scales.
 template <int NSRC, int MT>
 __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
-                                           int rot, int warp, int lane, int tile_base, int rows_total, int G,
+                                           int rot, int warp, int lane, int tile_base, int RT, int rows_total, int G,
                                            int64_t seq_row0, int Hq, int head0, uint16_t* out) {
   constexpr int RB = 32 / NSRC;
   for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
@@ -137,8 +137,8 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
       if (k0 + u >= per_rank) continue;
       const int k = k0 + u;
       const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const int rg = (tile_base + tile) * BM + trow;
-      if (rg >= rows_total) continue;
+      const int rg = (tile_base + tile) * RT + trow;
+      if (trow >= RT || rg >= rows_total) continue;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
@@ -181,6 +181,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   int b = unit / p.Hkv;
   const int kvh = unit - b * p.Hkv;
   const int N = p.N, G = p.G, rows_total = G * N;
+  // A row tile holds whole nodes: BM / G of them, i.e. RT = (BM / G) * G of its 128 rows (all 128
+  // when G divides 128); the remaining rows of the tile are idle.
+  const int RT = (BM / G) * G;
   // ---- set-up that reads no global memory: barriers, tensor memory, descriptor prefetch.  The
   //      kernel is launched with programmatic stream serialisation, so this part may run while the
   //      previous kernel of the stream drains; everything after the grid dependency wait sees that
@@ -295,8 +298,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int quarter = warp & 3;                  // TMEM lanes this warp may touch
   const int row = quarter * 32 + lane;           // row inside the 128-row tile
   const int my_rounds = slot == 0 ? rounds0 : rounds1;
-  const int r_glob = (row_cta * MT + ((MT == 2) ? slot : 0)) * BM + row;
-  const bool row_valid = r_glob < rows_total;
+  const int r_glob = (row_cta * MT + ((MT == 2) ? slot : 0)) * RT + row;
+  const bool row_valid = row < RT && r_glob < rows_total;
   const int node = row_valid ? r_glob / G : 0;
   const int gq = row_valid ? r_glob - node * G : 0;
   const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
@@ -432,7 +435,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     bool ok = true;
     if (warp == 2 && n_tiles > 0) {  // the Q tile(s): issued here so that the producer starts with K/V
       if (lane == 0) {
-        mbar_expect_tx(bar_q, MT * kQTile);
+        mbar_expect_tx(bar_q, (uint32_t)(MT * RT * HD * 2));   // the boxes hold RT rows of a tile
         const int nodes_per_tile = BM / G;
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
@@ -758,8 +761,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       float lsum = wgt * ml.y;
       for (int o = 1; o < n_src; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
       s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
-      const int rg = (row_cta * MT + tile) * BM + trow;
-      if (q == 0 && p.lse != nullptr && rg < rows_total) {
+      const int rg = (row_cta * MT + tile) * RT + trow;
+      if (q == 0 && p.lse != nullptr && trow < RT && rg < rows_total) {
         const int onode = rg / G, ogq = rg - onode * G;
         p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
       }
@@ -771,10 +774,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint16_t* outp = p.out;
     const int64_t seq_row0 = (int64_t)b * N;
     switch (n_src) {
-      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
@@ -799,7 +802,7 @@ bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t heads, 
 
 bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
   const int G = s.n_q_heads / s.n_kv_heads;
-  if (G > BM || (BM % G) != 0) return false;           // a row tile must hold whole nodes
+  if (G > BM) return false;                            // a row tile must hold at least one whole node
   const int64_t cache_rows = c.paged ? (int64_t)c.n_pages * CLV_PAGE_SIZE : (int64_t)s.batch * c.cap_tokens;
   if (cache_rows >= (1ll << 31) || (int64_t)s.batch * s.n_nodes >= (1ll << 31)) return false;
   return encode_fn() != nullptr;
@@ -808,9 +811,9 @@ bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
 AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
   AttnPlan pl;
   const int G = s.n_q_heads / s.n_kv_heads;
-  const int rows = G * s.n_nodes;
-  const int mt = rows > BM ? 2 : 1;
-  const int row_ctas = (rows + mt * BM - 1) / (mt * BM);
+  const int tiles = (s.n_nodes + BM / G - 1) / (BM / G);   // row tiles of BM / G whole nodes
+  const int mt = tiles > 1 ? 2 : 1;
+  const int row_ctas = (tiles + mt - 1) / mt;
   pl.m_tiles = row_ctas;
   const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * row_ctas;
   const int BN = mt == 2 ? Cfg<2>::BN : Cfg<1>::BN;
@@ -834,8 +837,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 cudaStream_t stream) {
   (void)tickets; (void)scratch;
   const int G = s.n_q_heads / s.n_kv_heads;
-  const int rows = G * s.n_nodes;
-  const int mt = rows > BM ? 2 : 1;
+  const int mt = (s.n_nodes + BM / G - 1) / (BM / G) > 1 ? 2 : 1;   // as in tc_attn_plan
   static bool attr_done[kMaxDevices] = {};
   if (first_call_on_device(attr_done)) {
     cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,

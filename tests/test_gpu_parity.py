@@ -132,10 +132,11 @@ def test_attention_special_trees_and_paging(clv, oracle, tree, paged):
     check_attention(oracle, w, st)
 
 
-@pytest.mark.parametrize("hq,hkv", [(6, 2), (12, 2), (5, 1)])
-def test_attention_group_sizes_that_do_not_divide_128(clv, oracle, hq, hkv):
-    # these shapes are served by the warp-level MMA kernel (a 128-row tile must hold whole nodes)
-    cfg = W.small_config(batch=2, n_q_heads=hq, n_kv_heads=hkv, ctx=(30, 500), n_nodes=37, vocab=64,
+@pytest.mark.parametrize("hq,hkv,n_nodes", [(6, 2, 37), (12, 2, 37), (5, 1, 37), (28, 4, 64), (24, 2, 128),
+                                             (7, 1, 18), (7, 1, 19)])
+def test_attention_group_sizes_that_do_not_divide_128(clv, oracle, hq, hkv, n_nodes):
+    # a 128-row tile holds whole nodes only, so with such group sizes some of its rows stay idle
+    cfg = W.small_config(batch=2, n_q_heads=hq, n_kv_heads=hkv, ctx=(30, 500), n_nodes=n_nodes, vocab=64,
                          seed=W.BASE_SEED + hq)
     w = W.generate(cfg)
     st = make_step(w)
