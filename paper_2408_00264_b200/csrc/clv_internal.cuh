@@ -67,7 +67,7 @@ cudaError_t launch_tree_attn(const AttnPlan& plan, const clv_shape& s, const clv
                              float* lse, int32_t* status, unsigned* tickets, void* scratch,
                              cudaStream_t stream);
 
-// tcgen05 / TMA path (row tiles must hold whole nodes: G divides 128)
+// tcgen05 / TMA path (a row tile holds whole nodes: any group size G up to 128)
 bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c);
 AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len);
 cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,

@@ -4,13 +4,14 @@
 // One thread block owns up to 256 query rows of one (sequence, kv head) - a row is a
 // (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes reuse every
 // K/V byte - and a contiguous range of key tiles (cache tiles first, then the tree's own keys).
-// A key tile is 128 keys when the block has two row tiles (an MMA costs about the same for 64 as
-// for 128 columns, so wide S tiles halve the tensor time) and 64 keys otherwise; tiles are loaded
-// as 64-key pieces, which is also the page size of a paged cache.  K and V travel through separate
+// A row tile of 128 rows holds whole nodes: 128 / G of them (rounded down; its other rows idle).
+// A key tile is 128 keys (an MMA costs about the same for 64 as for 128 columns, so wide S tiles
+// halve the tensor time); tiles are loaded as 64-key pieces, which is also the page size of a
+// paged cache.  K and V travel through separate
 // rings so that a K buffer is refilled as soon as its Q K^T is done.
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation), warps 2-5 and
 // 6-9 = two softmax groups of 128 threads, one thread per query row ("slot" 0 and 1).
-//   MT = 2 (more than 128 rows): slot s works on row tile s; both slots consume every K/V tile.
+//   MT = 2 (more than one row tile): slot s works on row tile s; both slots consume every K/V tile.
 //   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
 //           accumulators are merged like split-KV partials.
 // Split-KV: the blocks that share a row tile form a thread-block cluster; each stages its
