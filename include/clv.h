@@ -109,9 +109,14 @@ clv_status clv_workspace_init(void* workspace, size_t workspace_bytes, void* cud
  * q/k are taken as given (rotary positions L_b + depth(i) are the caller's business).
  * Several roots (extra -1 parents) are accepted here.  L_b = 0 is allowed.
  * status[b] = CLV_ERR_TREE if parent[b] is malformed, L_b < 0, L_b exceeds the cache capacity or
- * a needed block-table entry is outside [0, n_pages); that sequence's outputs are unspecified.
+ * a needed block-table entry is outside [0, n_pages); CLV_ERR_TIMEOUT if a bounded on-chip wait of
+ * one of the sequence's thread blocks ran out (about a second; never seen on a healthy device);
+ * CLV_OK otherwise.  With a non-zero status that sequence's outputs are unspecified; the word is
+ * written once per call, by the last thread block of the sequence to finish.
  * max_ctx_len (host): an upper bound of ctx_len[], used only to choose the split count; the
  * result does not depend on it.
+ * workspace: required (CLV_ERR_WORKSPACE), at least clv_workspace_bytes(); batch <= 32768.
+ * Group sizes G above 128 are refused with CLV_ERR_UNSUPPORTED.
  */
 clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache,
                          const void* q,        /* bf16 [B, N, Hq, 128]            */
@@ -145,9 +150,11 @@ clv_status clv_accept_argmax(const clv_shape* shape,
  * not acceptable.  For them the arrival counters and per-chunk partial results live in a fixed
  * array inside the library's device image instead of a workspace.
  *   - Same inputs, outputs and result as clv_accept_argmax (bit-identical ids).
- *   - Limit: B * N <= 4096 rows and rows * (thread blocks per row) <= 131072; anything larger is
- *     refused with CLV_ERR_TOO_LARGE and nothing is enqueued.  The array is about 1.04 MB and
- *     stays resident on every GPU that loads the library until the process exits.
+ *   - Limit: B * N <= 4096 rows and rows * (thread blocks per row) <= 131072, where a row is cut
+ *     into at most ceil(vocab / 2048) thread blocks: B * N * ceil(vocab / 2048) <= 131072 always
+ *     fits.  Anything larger is refused with CLV_ERR_TOO_LARGE and nothing is enqueued.  The
+ *     array is about 1.04 MB and stays resident on every GPU that loads the library until the
+ *     process exits.
  *   - The call allocates and frees nothing (no cudaMalloc / cudaFree, no allocating library
  *     routine).  The first call on a device looks up the array's device address (with that device
  *     current) and remembers it; make that first call outside of any stream capture.
@@ -289,6 +296,16 @@ clv_status clv_verify_step_host(const clv_shape* shape, const clv_kv_cache* cach
                                 int32_t max_ctx_len, float softmax_scale,
                                 void* staging, size_t staging_bytes, /* device */
                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * For tests only (the paper has no counterpart): the number of SM clock cycles after which a
+ * bounded on-chip wait of clv_tree_attn / clv_lm_head_argmax gives up and the call reports
+ * CLV_ERR_TIMEOUT in its device status.  The default is about a second; a test passes a few dozen
+ * cycles to make a wait for the first tile run out, which exercises the abort path without any
+ * fault (copies and tensor-core work in flight are still waited for with the long bound).
+ * sm_cycles <= 0 restores the default.  Process-wide; applies to launches made afterwards.
+ */
+void clv_test_set_wait_limit(int64_t sm_cycles);
 
 const char* clv_status_string(clv_status s);
 int clv_last_cuda_error(void); /* cudaError_t of the most recent CLV_ERR_CUDA on this thread */

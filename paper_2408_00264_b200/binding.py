@@ -25,6 +25,7 @@ EXPORTS = (
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
     "clv_lm_head_argmax", "clv_build_token_tree", "clv_accept_walk_commit",
+    "clv_test_set_wait_limit",
 )
 
 
@@ -105,6 +106,8 @@ def lib() -> ctypes.CDLL:
         L.clv_status_string.argtypes = [i32]
         L.clv_last_cuda_error.restype = ctypes.c_int
         L.clv_version.restype = ctypes.c_int
+        L.clv_test_set_wait_limit.restype = None
+        L.clv_test_set_wait_limit.argtypes = [i64]
         _lib = L
     return _lib
 
@@ -277,3 +280,8 @@ def clv_version() -> int:
 
 def clv_status_string(code: int) -> str:
     return lib().clv_status_string(int(code)).decode()
+
+
+def clv_test_set_wait_limit(sm_cycles: int) -> None:
+    """Tests only: SM cycles after which a bounded on-chip wait gives up (<= 0: the default)."""
+    lib().clv_test_set_wait_limit(int(sm_cycles))

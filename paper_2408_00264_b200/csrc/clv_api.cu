@@ -4,6 +4,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "clv_internal.cuh"
 
 namespace clv {
@@ -11,18 +14,25 @@ namespace clv {
 static thread_local int g_last_cuda_error = 0;
 
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      n = v;
-    else
-      n = 148;  // B200; used for sizing only when no device can be queried
+  static std::mutex mu;
+  static int cached[kMaxDevices] = {};
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
     (void)cudaGetLastError();
+    return 148;  // B200; used for sizing only when no device can be queried
   }
-  return n;
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[dev] == 0) {
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      cached[dev] = v;
+    else
+      return 148;
+  }
+  return cached[dev];
 }
+
+static std::atomic<long long> g_wait_limit{2000000000ll};  // SM cycles: about a second
+long long wait_limit_cycles() { return g_wait_limit.load(std::memory_order_relaxed); }
 
 static clv_status cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;
@@ -53,14 +63,6 @@ static clv_status check_cache(const clv_kv_cache* c) {
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Which attention kernel serves a call: the tcgen05 kernel whenever the shape allows it.
-// CLV_ATTN_PATH=mma (environment, read at each call) forces the warp-level path, for comparisons.
-static bool use_tc_path(const clv_shape& s, const clv_kv_cache& c) {
-  const char* e = getenv("CLV_ATTN_PATH");
-  if (e && strcmp(e, "mma") == 0) return false;
-  return tc_attn_supported(s, c);
-}
-
 }  // namespace clv
 
 using namespace clv;
@@ -71,9 +73,7 @@ size_t clv_workspace_bytes(const clv_shape* shape, const clv_kv_cache* cache, in
   (void)cache;
   if (check_shape(shape) != CLV_OK) return 0;
   if (max_ctx_len < 0) max_ctx_len = 0;
-  const AttnPlan ap = attn_plan(*shape, max_ctx_len);
-  const AttnPlan tp = tc_attn_plan(*shape, max_ctx_len);   // either kernel may serve the call
-  size_t scratch = ap.scratch_bytes > tp.scratch_bytes ? ap.scratch_bytes : tp.scratch_bytes;
+  size_t scratch = tc_attn_plan(*shape, max_ctx_len).scratch_bytes;
   if (shape->vocab > 0) {
     const ArgmaxPlan gp = argmax_plan(shape->batch * shape->n_nodes, shape->vocab);
     if (gp.scratch_bytes > scratch) scratch = gp.scratch_bytes;
@@ -89,11 +89,12 @@ clv_status clv_workspace_init(void* workspace, size_t workspace_bytes, void* cud
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
-clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, const void* q,
-                         const void* k_tree, const void* v_tree, const int32_t* parent,
-                         const int32_t* ctx_len, int32_t max_ctx_len, float softmax_scale,
-                         void* out, float* lse, int32_t* status, void* workspace,
-                         size_t workspace_bytes, void* cuda_stream) {
+// Argument checks of clv_tree_attn (nothing is enqueued); fills the plan on success.
+static clv_status validate_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, const void* q,
+                                     const void* k_tree, const void* v_tree, const int32_t* parent,
+                                     const int32_t* ctx_len, int32_t max_ctx_len, const void* out,
+                                     const int32_t* status, const void* workspace, size_t workspace_bytes,
+                                     AttnPlan* plan) {
   clv_status st = check_shape(shape);
   if (st != CLV_OK) return st;
   st = check_cache(cache);
@@ -101,22 +102,33 @@ clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, cons
   if (!q || !k_tree || !v_tree || !parent || !ctx_len || !out || !status) return CLV_ERR_NULL;
   if (!aligned16(q) || !aligned16(k_tree) || !aligned16(v_tree) || !aligned16(out)) return CLV_ERR_ALIGN;
   if (max_ctx_len < 0) return CLV_ERR_SHAPE;
-  const bool tc = use_tc_path(*shape, *cache);
-  const AttnPlan plan = tc ? tc_attn_plan(*shape, max_ctx_len) : attn_plan(*shape, max_ctx_len);
-  if (plan.scratch_bytes > 0) {
-    if (!workspace || workspace_bytes < kWsFixedBytes + plan.scratch_bytes) return CLV_ERR_WORKSPACE;
-    if (!aligned16(workspace)) return CLV_ERR_ALIGN;
-  }
-  cudaError_t e = (tc ? launch_tree_attn_tc : launch_tree_attn)(
-      plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len, softmax_scale, out, lse, status,
-      workspace ? ws_tickets(workspace) : nullptr, workspace ? ws_scratch(workspace) : nullptr,
-      static_cast<cudaStream_t>(cuda_stream));
+  if (shape->n_q_heads / shape->n_kv_heads > 128) return CLV_ERR_UNSUPPORTED;
+  if (shape->batch > kTickets / 2) return CLV_ERR_UNSUPPORTED;   // two counters per sequence
+  *plan = tc_attn_plan(*shape, max_ctx_len);
+  if (!workspace || workspace_bytes < kWsFixedBytes + plan->scratch_bytes) return CLV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  if (!tc_attn_supported(*shape, *cache)) return CLV_ERR_UNSUPPORTED;   // asks the driver: last
+  return CLV_OK;
+}
+
+clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, const void* q,
+                         const void* k_tree, const void* v_tree, const int32_t* parent,
+                         const int32_t* ctx_len, int32_t max_ctx_len, float softmax_scale,
+                         void* out, float* lse, int32_t* status, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  AttnPlan plan;
+  const clv_status st = validate_tree_attn(shape, cache, q, k_tree, v_tree, parent, ctx_len, max_ctx_len,
+                                           out, status, workspace, workspace_bytes, &plan);
+  if (st != CLV_OK) return st;
+  cudaError_t e = launch_tree_attn_tc(plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len,
+                                      softmax_scale, out, lse, status, ws_tickets(workspace),
+                                      ws_scratch(workspace), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
-clv_status clv_accept_argmax(const clv_shape* shape, const void* logits, int64_t ld,
-                             int32_t* argmax_ids, void* workspace, size_t workspace_bytes,
-                             void* cuda_stream) {
+static clv_status validate_accept_argmax(const clv_shape* shape, const void* logits, int64_t ld,
+                                         const int32_t* argmax_ids, const void* workspace,
+                                         size_t workspace_bytes, ArgmaxPlan* plan) {
   clv_status st = check_shape(shape);
   if (st != CLV_OK) return st;
   if (!logits || !argmax_ids) return CLV_ERR_NULL;
@@ -124,11 +136,20 @@ clv_status clv_accept_argmax(const clv_shape* shape, const void* logits, int64_t
   if (!aligned16(logits) || (ld % 8) != 0) return CLV_ERR_ALIGN;
   const int64_t rows = (int64_t)shape->batch * shape->n_nodes;
   if (rows > kTickets) return CLV_ERR_UNSUPPORTED;
-  const ArgmaxPlan plan = argmax_plan((int)rows, shape->vocab);
-  if (plan.chunks > 1) {
-    if (!workspace || workspace_bytes < kWsFixedBytes + plan.scratch_bytes) return CLV_ERR_WORKSPACE;
+  *plan = argmax_plan((int)rows, shape->vocab);
+  if (plan->chunks > 1) {
+    if (!workspace || workspace_bytes < kWsFixedBytes + plan->scratch_bytes) return CLV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return CLV_ERR_ALIGN;
   }
+  return CLV_OK;
+}
+
+clv_status clv_accept_argmax(const clv_shape* shape, const void* logits, int64_t ld,
+                             int32_t* argmax_ids, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+  ArgmaxPlan plan;
+  const clv_status st = validate_accept_argmax(shape, logits, ld, argmax_ids, workspace, workspace_bytes, &plan);
+  if (st != CLV_OK) return st;
   cudaError_t e = launch_argmax(plan, logits, ld, shape->vocab, argmax_ids,
                                 workspace ? ws_tickets(workspace) : nullptr,
                                 workspace ? ws_scratch(workspace) : nullptr,
@@ -155,12 +176,12 @@ static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
   return x < y + nb && y < x + na;
 }
 
-clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* cache,
-                                  const int32_t* parent, const int32_t* tokens, const int32_t* argmax_ids,
-                                  const void* k_tree, const void* v_tree, const int32_t* ctx_len,
-                                  int32_t* accept_len, int32_t* accept_idx, int32_t* next_token,
-                                  int32_t* ctx_len_out, int32_t* walk_status, int32_t* commit_status,
-                                  void* cuda_stream) {
+static clv_status validate_walk_commit(const clv_shape* shape, const clv_kv_cache* cache,
+                                       const int32_t* parent, const int32_t* tokens, const int32_t* argmax_ids,
+                                       const void* k_tree, const void* v_tree, const int32_t* ctx_len,
+                                       const int32_t* accept_len, const int32_t* accept_idx,
+                                       const int32_t* next_token, const int32_t* ctx_len_out,
+                                       const int32_t* walk_status, const int32_t* commit_status) {
   clv_status st = check_shape(shape);
   if (st != CLV_OK) return st;
   st = check_cache(cache);
@@ -177,6 +198,19 @@ clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* ca
   if (overlaps(k_tree, tree_bytes, cache->k, cache_bytes) || overlaps(k_tree, tree_bytes, cache->v, cache_bytes) ||
       overlaps(v_tree, tree_bytes, cache->k, cache_bytes) || overlaps(v_tree, tree_bytes, cache->v, cache_bytes))
     return CLV_ERR_UNSUPPORTED;
+  return CLV_OK;
+}
+
+clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* cache,
+                                  const int32_t* parent, const int32_t* tokens, const int32_t* argmax_ids,
+                                  const void* k_tree, const void* v_tree, const int32_t* ctx_len,
+                                  int32_t* accept_len, int32_t* accept_idx, int32_t* next_token,
+                                  int32_t* ctx_len_out, int32_t* walk_status, int32_t* commit_status,
+                                  void* cuda_stream) {
+  const clv_status st = validate_walk_commit(shape, cache, parent, tokens, argmax_ids, k_tree, v_tree, ctx_len,
+                                             accept_len, accept_idx, next_token, ctx_len_out, walk_status,
+                                             commit_status);
+  if (st != CLV_OK) return st;
   cudaError_t e = launch_walk_commit(*shape, *cache, parent, tokens, argmax_ids, k_tree, v_tree, ctx_len,
                                      accept_len, accept_idx, next_token, ctx_len_out, walk_status,
                                      commit_status, static_cast<cudaStream_t>(cuda_stream));
@@ -307,6 +341,23 @@ clv_status clv_verify_step_host(const clv_shape* shape, const clv_kv_cache* cach
   const size_t B = shape->batch, N = shape->n_nodes;
   const size_t qb = B * N * shape->n_q_heads * CLV_HEAD_DIM * 2;
   const size_t tb = B * N * shape->n_kv_heads * CLV_HEAD_DIM * 2;
+  int32_t* const dstat = reinterpret_cast<int32_t*>(d + L.status);
+  // every check of the three calls first: a mistake the host can see must leave the stream empty
+  AttnPlan attn_plan_unused;
+  ArgmaxPlan argmax_plan_unused;
+  st = validate_tree_attn(shape, cache, d + L.q, d + L.k_tree, d + L.v_tree,
+                          reinterpret_cast<int32_t*>(d + L.parent), ctx_len, max_ctx_len, d + L.out, dstat,
+                          workspace, workspace_bytes, &attn_plan_unused);
+  if (st != CLV_OK) return st;
+  st = validate_accept_argmax(shape, d + L.logits, in->ld, reinterpret_cast<int32_t*>(d + L.ids), workspace,
+                              workspace_bytes, &argmax_plan_unused);
+  if (st != CLV_OK) return st;
+  st = validate_walk_commit(shape, cache, reinterpret_cast<int32_t*>(d + L.parent),
+                            reinterpret_cast<int32_t*>(d + L.tokens), reinterpret_cast<int32_t*>(d + L.ids),
+                            d + L.k_tree, d + L.v_tree, ctx_len, reinterpret_cast<int32_t*>(d + L.alen),
+                            reinterpret_cast<int32_t*>(d + L.aidx), reinterpret_cast<int32_t*>(d + L.next),
+                            ctx_len, dstat + B, dstat + 2 * B);
+  if (st != CLV_OK) return st;
   cudaError_t e;
 #define CLV_COPY(dst, src, n, kind) \
   if ((e = cudaMemcpyAsync(dst, src, n, kind, s)) != cudaSuccess) return cuda_fail(e)
@@ -316,7 +367,6 @@ clv_status clv_verify_step_host(const clv_shape* shape, const clv_kv_cache* cach
   CLV_COPY(d + L.parent, in->parent, B * N * 4, cudaMemcpyHostToDevice);
   CLV_COPY(d + L.tokens, in->tokens, B * N * 4, cudaMemcpyHostToDevice);
   CLV_COPY(d + L.logits, in->logits, B * N * (size_t)in->ld * 2, cudaMemcpyHostToDevice);
-  int32_t* dstat = reinterpret_cast<int32_t*>(d + L.status);
   st = clv_tree_attn(shape, cache, d + L.q, d + L.k_tree, d + L.v_tree,
                      reinterpret_cast<int32_t*>(d + L.parent), ctx_len, max_ctx_len, softmax_scale,
                      d + L.out, nullptr, dstat, workspace, workspace_bytes, cuda_stream);
@@ -357,6 +407,10 @@ const char* clv_status_string(clv_status s) {
 }
 
 int clv_last_cuda_error(void) { return g_last_cuda_error; }
+
+void clv_test_set_wait_limit(int64_t sm_cycles) {
+  g_wait_limit.store(sm_cycles > 0 ? (long long)sm_cycles : 2000000000ll, std::memory_order_relaxed);
+}
 int clv_version(void) { return 100; }
 
 }  // extern "C"

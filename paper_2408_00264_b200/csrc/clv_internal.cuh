@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "clv.h"
 
 namespace clv {
@@ -53,21 +55,13 @@ cudaError_t launch_walk_commit(const clv_shape& s, const clv_kv_cache& c, const 
                                int32_t* accept_idx, int32_t* next_token, int32_t* ctx_len_out,
                                int32_t* walk_status, int32_t* commit_status, cudaStream_t stream);
 
-// ---- tree attention ---------------------------------------------------------------------------
+// ---- tree attention (tcgen05 / TMA; a row tile holds whole nodes: any group size G up to 128) -------
 struct AttnPlan {
-  int m_tiles;   // row tiles per (sequence, kv head): ceil(G*N / rows per tile)
+  int m_tiles;   // row tiles per (sequence, kv head)
   int splits;    // thread blocks along the key axis per row tile
   size_t scratch_bytes;
   int tickets;   // counters used
 };
-AttnPlan attn_plan(const clv_shape& s, int max_ctx_len);
-cudaError_t launch_tree_attn(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,
-                             const void* q, const void* k_tree, const void* v_tree,
-                             const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
-                             float* lse, int32_t* status, unsigned* tickets, void* scratch,
-                             cudaStream_t stream);
-
-// tcgen05 / TMA path (a row tile holds whole nodes: any group size G up to 128)
 bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c);
 AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len);
 cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,
@@ -87,17 +81,32 @@ cudaError_t launch_token_tree(int batch, int n_cand, int max_len, int node_cap, 
                               const int32_t* cand, const int32_t* cand_len, int32_t* tokens, int32_t* parent,
                               int32_t* n_nodes, int32_t* node_of, int32_t* status, cudaStream_t stream);
 
-int sm_count();
+int sm_count();   // of the current device
+
+// SM cycles a bounded on-chip wait may last before the block gives up (default: about a second;
+// clv_test_set_wait_limit shortens it for the tests of the time-out path).
+long long wait_limit_cycles();
 
 // Per-device one-time set-up (function attributes belong to the device that is current when they
-// are set): true the first time it is called with `done` on the current device.
+// are set).  run_once_per_device(state, fn) runs fn() with the current device until it has
+// succeeded once on that device; concurrent first calls from several host threads are serialised,
+// and a failed set-up is retried by the next call.
 constexpr int kMaxDevices = 64;
-inline bool first_call_on_device(bool (&done)[kMaxDevices]) {
+struct OncePerDevice {
+  std::mutex mu;
+  bool done[kMaxDevices] = {};
+};
+template <class Fn>
+inline cudaError_t run_once_per_device(OncePerDevice& st, Fn fn) {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return true;
-  if (done[dev]) return false;
-  done[dev] = true;
-  return true;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return fn();   // not remembered: set up at every call
+  std::lock_guard<std::mutex> lock(st.mu);
+  if (st.done[dev]) return cudaSuccess;
+  e = fn();
+  if (e == cudaSuccess) st.done[dev] = true;
+  return e;
 }
 
 }  // namespace clv

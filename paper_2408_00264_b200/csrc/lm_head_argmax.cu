@@ -44,6 +44,7 @@ struct Params {
   unsigned* counter;          // zero between calls
   unsigned* aborts;           // blocks that gave up a wait; zero between calls
   int32_t* status;            // one word: CLV_OK or CLV_ERR_TIMEOUT
+  long long wait_limit;       // SM cycles a bounded wait may last
 };
 
 __device__ __forceinline__ unsigned long long pack_key(float v, int i) {
@@ -111,6 +112,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abort_flag = &s_abort;
+  const long long wlim = p.wait_limit;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   auto sA = [&](int s, int mt) { return smem_base + (uint32_t)s * kStageBytes + (uint32_t)mt * kATile; };
@@ -133,7 +135,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         const uint32_t w_bytes = (uint32_t)wi.cols * BK * 2;
         for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
           const int s = it % kStages;
-          if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag);
+          if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag, wlim);
           if (!ok) break;
           mbar_expect_tx(bar_full(s), w_bytes + (uint32_t)m_tiles * kATile);
           tma_load_2d(sW(s), wi.cols == BN ? &tm_w : &tm_w_half, kc * BK, wi.col0, bar_full(s));
@@ -153,13 +155,13 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         const int m_tiles = (p.M - wi.mb * MB) > BM ? 2 : 1;
         const uint32_t idesc = wi.cols == BN ? kIdesc : kIdescHalf;
         if (tile > 0) {  // the epilogue has taken the previous tile out of tensor memory
-          ok = mbar_wait(bar_acc_empty, (tile - 1) & 1, abort_flag);
+          ok = mbar_wait(bar_acc_empty, (tile - 1) & 1, abort_flag, wlim);
           if (!ok) break;
           tc_fence_after();
         }
         for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
           const int s = it % kStages;
-          ok = mbar_wait(bar_full(s), (it / kStages) & 1, abort_flag);
+          ok = mbar_wait(bar_full(s), (it / kStages) & 1, abort_flag, wlim);
           if (!ok) break;
           tc_fence_after();
           const uint64_t wd = smem_desc(sW(s), 16, 1024);
@@ -188,7 +190,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       const int mb = wi.mb;
       const int row = mb * MB + mt * BM + row_in_tile;
       const bool row_valid = row < p.M;
-      ok = mbar_wait(bar_acc_full, tile & 1, abort_flag);
+      ok = mbar_wait(bar_acc_full, tile & 1, abort_flag, wlim);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -281,12 +283,11 @@ bool lm_head_supported(int rows, int hidden, int vocab) {
 cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
                                   int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
                                   unsigned* tickets, cudaStream_t stream) {
-  static bool attr_set[kMaxDevices] = {};
-  if (first_call_on_device(attr_set)) {
-    cudaError_t e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmem);
-    if (e != cudaSuccess) return e;
-  }
+  static OncePerDevice once;
+  cudaError_t e0 = run_once_per_device(once, [] {
+    return cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
+  });
+  if (e0 != cudaSuccess) return e0;
   CUtensorMap tm_a, tm_w, tm_w_half;
   if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, BM) ||
       !make_map_2d(&tm_w, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN) ||
@@ -303,6 +304,7 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
   p.aborts = tickets + 1;
   p.keys = reinterpret_cast<unsigned long long*>(tickets + 2);
   p.status = status;
+  p.wait_limit = wait_limit_cycles();
   const int tiles = p.n_tiles * p.m_blocks;
   const int grid = tiles < sm_count() ? tiles : sm_count();
   const int rem = tiles % grid;   // tiles of the last, incomplete round

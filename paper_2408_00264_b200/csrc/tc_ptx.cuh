@@ -45,25 +45,35 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // n
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
-// try_wait itself suspends the thread for a hardware-bounded time, so the first polls need no
-// clock; after that the SM clock (cheap to read, unlike the global timer) bounds the wait.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait of at most `limit` SM cycles (the library's default is kWaitLimitCycles; tests may
+// shorten it).  Returns false when the block is aborting (this wait or another one ran out).
+// try_wait itself suspends the thread for a hardware-bounded time, so with the default limit the
+// first polls need no clock; after that the SM clock (cheap to read, unlike the global timer)
+// bounds the wait.  A short limit (below kSuspendFreeLimit) is polled with test_wait only, which
+// never suspends, so that the limit is what ends the wait.
+constexpr long long kSuspendFreeLimit = 1000000ll;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit) {
   if (mbar_test(bar, parity)) return true;  // the common case in steady state: already complete
+  const bool may_suspend = limit >= kSuspendFreeLimit;
+  if (may_suspend) {
 #pragma unroll 1
-  for (int spin = 0; spin < 32; ++spin)
-    if (mbar_try(bar, parity)) return true;
+    for (int spin = 0; spin < 32; ++spin)
+      if (mbar_try(bar, parity)) return true;
+  }
   const long long t0 = clock64();
   for (;;) {
-    if (mbar_try(bar, parity)) return true;
+    if (may_suspend ? mbar_try(bar, parity) : mbar_test(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       return false;
     }
   }
 }
-__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {  // teardown only
+// Teardown only: waits for work that is already in flight (a TMA copy, issued MMAs) and therefore
+// always keeps the long bound, whatever limit the block's other waits had.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
   const long long t0 = clock64();
   while (!mbar_try(bar, parity) && clock64() - t0 < kWaitLimitCycles) {}
 }

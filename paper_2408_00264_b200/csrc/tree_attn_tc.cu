@@ -70,6 +70,9 @@ struct Params {
   int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
   int splits;      // thread blocks along the key axis = cluster size (1, 2, 4 or 8)
   float scale_log2;
+  long long wait_limit;   // SM cycles a bounded wait may last
+  unsigned* tickets;      // per sequence: [2b] blocks that have finished, [2b+1] error bits; zero between calls
+  int blocks_per_seq;
 };
 
 constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
@@ -249,9 +252,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   const bool reporter = (row_cta == 0 && split == 0 && kvh == 0);
+  // status[b] is written once, by whichever block of the sequence finishes last: every block adds
+  // its error bits (1 malformed input, 2 a wait ran out) to the sequence's word in the workspace
+  // and then takes a ticket; the holder of the last ticket turns the bits into the status code and
+  // leaves both words zero for the next call.  So no verdict can be overwritten by a later "fine".
+  auto report = [&](unsigned bits) -> unsigned {   // one thread per block; returns the ticket
+    if (bits) atomicOr(p.tickets + 2 * b + 1, bits);
+    __threadfence();
+    return atomicInc(p.tickets + 2 * b, (unsigned)p.blocks_per_seq - 1);  // wraps to 0
+  };
+  auto publish = [&](unsigned ticket) {
+    if (ticket != (unsigned)p.blocks_per_seq - 1) return;
+    __threadfence();
+    const unsigned bits = atomicExch(p.tickets + 2 * b + 1, 0u);
+    p.status[b] = (bits & 1u) ? CLV_ERR_TREE : (bits & 2u) ? CLV_ERR_TIMEOUT : CLV_OK;
+  };
   if (seq_bad) {  // the whole cluster leaves together; nothing has been issued yet
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-    if (reporter && tid == 0) p.status[b] = CLV_ERR_TREE;
+    if (tid == 0) publish(report(1u));
     return;
   }
 
@@ -285,6 +303,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t bar_drain = bar0 + 8u * (NRING + 7);
 
   volatile int* abort_flag = &s_abort;
+  const long long wlim = p.wait_limit;
   // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
   // the scores have been read); O of slot s at 2 BN + 128 s
   auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
@@ -344,7 +363,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
           const uint32_t bytes = (uint32_t)n_pieces * 2u * kPiece;  // both halves of the head dim
-          if (i >= KST) ok = mbar_wait(bar_k_empty(ks), ((i / KST) - 1) & 1, abort_flag);
+          if (i >= KST) ok = mbar_wait(bar_k_empty(ks), ((i / KST) - 1) & 1, abort_flag, wlim);
           if (ok) {
             mbar_expect_tx(bar_k_full(ks), bytes);
 #pragma unroll
@@ -355,7 +374,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               tma_load_3d(sK + ks * kTile + kHalf + j * kPiece, mk, 64, kvh, row0[j], bar_k_full(ks));
             }
             issued_k = i + 1;
-            if (i >= VST) ok = mbar_wait(bar_v_empty(vs), ((i / VST) - 1) & 1, abort_flag);
+            if (i >= VST) ok = mbar_wait(bar_v_empty(vs), ((i / VST) - 1) & 1, abort_flag, wlim);
           }
           if (ok) {
             s_tile_ok[vs] = tile_ok;  // read by the softmax threads after this V barrier completes
@@ -376,7 +395,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   } else if (warp == 1) {
     // =========================== MMA issuer ===================================================
     if (lane == 0 && n_tiles > 0) {
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      bool ok = mbar_wait(bar_q, 0, abort_flag, wlim);
       tc_fence_after();
       auto local_tile = [&](int s, int r) { return (MT == 2) ? r : 2 * r + s; };
       // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
@@ -388,7 +407,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int i = local_tile(s, r), st = i % KST;
         // with two row tiles, slot 1 uses the K tile that slot 0 has just waited for
         if (MT == 1 || s == 0) {
-          if (!mbar_wait(bar_k_full(st), (i / KST) & 1, abort_flag)) return false;
+          if (!mbar_wait(bar_k_full(st), (i / KST) & 1, abort_flag, wlim)) return false;
           tc_fence_after();
         }
         const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
@@ -409,11 +428,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int r = 0; r < rounds0 && ok; ++r) {
         for (int s = 0; s < 2 && ok; ++s) {
           if (r >= rounds[s]) continue;
-          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag);
+          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag, wlim);
           if (!ok) break;
           const int i = local_tile(s, r), st = i % VST;
           if (MT == 1 || s == 0) {  // likewise the V tile
-            ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
+            ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag, wlim);
             if (!ok) break;
           }
           tc_fence_after();
@@ -466,7 +485,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
       pbad = __any_sync(0xFFFFFFFFu, pbad);
-      if (lane == 0) p.status[b] = pbad ? CLV_ERR_TREE : CLV_OK;
+      if (lane == 0 && pbad) atomicOr(p.tickets + 2 * b + 1, 1u);  // before this block's ticket
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
 
@@ -496,14 +515,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         short_tile |= valid[j] < PG;
       }
-      ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag);
+      ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag, wlim);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
       if (p.paged && cache_tile) {
         // the producer's verdict on this tile's pages, written before it armed the V barrier (the
         // V stage is not reused before this tile's P V, so the flag is stable)
-        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
+        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag, wlim);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         if (!*(volatile int*)&s_tile_ok[st]) {  // sequence is flagged; hide the whole tile
@@ -576,7 +595,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const float mx = suspect ? row_max() : m_ref;
         const bool need = mx > m_ref;
         if (r > 0) {  // O must be at rest: the previous P V has completed
-          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag);
+          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag, wlim);
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -609,7 +628,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (short_tile) {
         // Rows of a V piece beyond its real keys hold whatever lies behind them in memory (or were
         // never loaded); their probabilities are exactly 0, but 0 * NaN would poison O: clear them.
-        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag);
+        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag, wlim);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         uint8_t* vt = sV_gen + st * kTile;
@@ -630,7 +649,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 
     if (ok && rounds > 0) {  // the last P V of this slot has landed in O
-      ok = mbar_wait(bar_pv_done(slot), (rounds - 1) & 1, abort_flag);
+      ok = mbar_wait(bar_pv_done(slot), (rounds - 1) & 1, abort_flag, wlim);
       ok = __all_sync(0xFFFFFFFFu, ok);
     }
   }
@@ -653,6 +672,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   tc_fence_after();
   const bool aborted = *abort_flag != 0;
+  // the ticket is taken here and looked at when the block leaves, so that its round trip is hidden
+  // behind the epilogue (no wait can run out after this point)
+  unsigned my_ticket = 0;
+  if (tid == 0) my_ticket = report(aborted ? 2u : 0u);
   const int n_src = p.splits * (MT == 1 ? 2 : 1);  // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
   // staging area for the merge: O of both slots as fp16 [slot][128 rows][128], every row scaled by
@@ -736,8 +759,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-  if (aborted && tid == 0) atomicMax(p.status + b, CLV_ERR_TIMEOUT);
-  if (n_src == 1) return;  // such a block is its own cluster
+  if (n_src == 1) {  // such a block is its own cluster
+    if (tid == 0) publish(my_ticket);
+    return;
+  }
 
   // ---- merge across the cluster (the split-KV blocks of one row tile) through distributed
   //      shared memory: rank j finalises rows [j, j+1) * rows/splits of the tile(s) ------------
@@ -782,6 +807,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
+  if (tid == 0) publish(my_ticket);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -836,18 +862,18 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
                                 cudaStream_t stream) {
-  (void)tickets; (void)scratch;
+  (void)scratch;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int mt = (s.n_nodes + BM / G - 1) / (BM / G) > 1 ? 2 : 1;   // as in tc_attn_plan
-  static bool attr_done[kMaxDevices] = {};
-  if (first_call_on_device(attr_done)) {
+  static OncePerDevice once;
+  cudaError_t e0 = run_once_per_device(once, [] {
     cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)Cfg<1>::kSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(tree_attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)Cfg<2>::kSmem);
-    if (e != cudaSuccess) return e;
-  }
+    return cudaFuncSetAttribute(tree_attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)Cfg<2>::kSmem);
+  });
+  if (e0 != cudaSuccess) return e0;
   alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt;
   const uint64_t cache_rows = c.paged ? (uint64_t)c.n_pages * CLV_PAGE_SIZE : (uint64_t)s.batch * c.cap_tokens;
   const uint64_t tree_rows = (uint64_t)s.batch * s.n_nodes;
@@ -872,6 +898,9 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.splits = plan.splits;
   p.longest_first = (ctas > sm_count() && s.batch > 1 && s.batch <= 256) ? 1 : 0;
   p.scale_log2 = scale * 1.4426950408889634f;
+  p.wait_limit = wait_limit_cycles();
+  p.tickets = tickets;
+  p.blocks_per_seq = s.n_kv_heads * plan.m_tiles * plan.splits;
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)ctas, (unsigned)plan.splits, 1);

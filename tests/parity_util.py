@@ -27,13 +27,13 @@ def assert_attn_close(got_bits, ref, what=""):
     assert a <= ATTN_MAX_ABS and r <= ATTN_MAX_REL, "%s max-abs %.3e max-rel %.3e" % (what, a, r)
 
 
-def sample_rows(w, n, seed=0):
-    """n random (b, i, h) triples, always including first/last node and head of each sequence."""
-    c = w.cfg
-    rng = np.random.default_rng(seed)
-    rows = [(b, i, h) for b in (0, c.batch - 1) for i in (0, c.n_nodes - 1)
-            for h in (0, c.n_q_heads - 1)]
-    while len(rows) < n:
-        rows.append((int(rng.integers(c.batch)), int(rng.integers(c.n_nodes)),
-                     int(rng.integers(c.n_q_heads))))
-    return np.array(sorted(set(rows)), dtype=np.int32)
+def log_parity(workload, **figures):
+    """Appends one line of observed parity figures to the file named by CLV_PARITY_LOG (if set)."""
+    import json
+    import os
+    path = os.environ.get("CLV_PARITY_LOG")
+    if not path:
+        return
+    os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+    with open(path, "a") as f:
+        f.write(json.dumps(dict(workload=workload, **figures)) + "\n")

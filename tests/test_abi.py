@@ -74,3 +74,28 @@ def test_workspace_size_is_monotone_and_covers_fixed_part(clv):
     big = clv.clv_workspace_bytes(s, None, 4096)
     assert small >= 256 + 4 * 65536 and big >= small
     assert clv.clv_staging_bytes(s, 128256) > 4 * 64 * 128256 * 2
+
+
+def test_host_step_checks_everything_before_it_enqueues_anything(clv):
+    # clv_verify_step_host runs the argument checks of all three calls before its first copy, so
+    # a mistake the host can see returns its code with nothing on the stream.  No device is needed
+    # to see the codes: the pointers below are never dereferenced.
+    L = clv.lib()
+    s = clv.make_shape(2, 8, 4, 2, 1000, 5)
+    cache = clv.ClvKvCache(0x1000_0000, 0x2000_0000, 0, 256, 64, 0, 0, None)
+    host = ctypes.c_void_p(0x5000_0000)
+    hin = clv.ClvHostInputs(*([0x5000_0000] * 6), 1000)
+    hout = clv.ClvHostOutputs(*([0x6000_0000] * 6))
+    staging = ctypes.c_void_p(0x7000_0000)
+    need = clv.clv_staging_bytes(s, 1000)
+    ws = ctypes.c_void_p(0x7800_0000)
+    ws_need = clv.clv_workspace_bytes(s, None, 200)
+
+    def call(hin=hin, staging_bytes=need, ws=ws, ws_bytes=ws_need):
+        return L.clv_verify_step_host(clv._ref(s), clv._ref(cache), clv._ref(hin), clv._ref(hout), host, 200,
+                                      1.0, staging, staging_bytes, ws, ws_bytes, None)
+    bad_ld = clv.ClvHostInputs(*([0x5000_0000] * 6), 999)              # row stride below the vocabulary
+    assert call(hin=bad_ld) == clv.CLV_ERR_SHAPE
+    assert call(staging_bytes=need - 1) == clv.CLV_ERR_WORKSPACE
+    assert call(ws=None, ws_bytes=0) == clv.CLV_ERR_WORKSPACE           # the attention's check
+    assert call(ws_bytes=1024) == clv.CLV_ERR_WORKSPACE

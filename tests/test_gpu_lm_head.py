@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def clv():
     if not torch.cuda.is_available():
-        pytest.skip("needs a GPU")
+        pytest.fail("these tests need a CUDA device")
     from paper_2408_00264_b200 import binding
     binding.lib()
     return binding
@@ -89,6 +89,68 @@ def test_ties_and_special_values(clv, oracle):
     got = run_gpu(clv, hb, wb)
     assert np.array_equal(got, oracle.lm_head_argmax(hb, wb))
     assert got[1] == 0
+
+
+def test_best_two_logits_one_bf16_step_apart(clv, oracle):
+    # Built, not drawn: every product and sum below is exact in fp32, so the GPU must pick the
+    # checker's index although the two best logits are neighbouring bf16 numbers (1.75 and
+    # 1.75 + 2^-7): this is the near-tie branch of check_rows, entered on purpose, in both orders
+    # of the two candidates and with the candidates in different 256-entry tiles.
+    K, V = 64, 700
+    hid = np.zeros((4, K), dtype=np.float32)
+    hid[:, :3] = 1.0
+    w = np.zeros((V, K), dtype=np.float32)
+    w[:, 0] = 1.0                                    # every other logit is 1.0
+    lo = np.array([1.0, 0.5, 0.25], dtype=np.float32)            # sums to 1.75
+    hi = np.array([1.0, 0.5, 0.25 + 2.0 ** -7], dtype=np.float32)  # one bf16 step above
+    cases = [(100, 300), (300, 100), (5, 6), (699, 0)]           # (index of hi, index of lo)
+    got_all, ref_all = [], []
+    for i_hi, i_lo in cases:
+        wc = w.copy()
+        wc[i_hi, :3] = hi
+        wc[i_lo, :3] = lo
+        hb, wb = W.f32_to_bf16_bits(hid), W.f32_to_bf16_bits(wc)
+        got = run_gpu(clv, hb, wb)
+        ref, z = oracle.lm_head_argmax(hb, wb, want_logits=True)
+        assert z[0, i_hi] - z[0, i_lo] == 2.0 ** -7
+        assert check_rows(oracle, hb, wb, got) == 0      # no row has a clear winner ...
+        assert np.array_equal(got, ref) and (got == i_hi).all()   # ... and yet the choice is exact
+        got_all.append(got)
+        ref_all.append(ref)
+
+
+def test_unplanted_rows_agree_with_the_checker_almost_everywhere(clv, oracle):
+    # drawn logits, no planted winner: the exact index wherever the lead is clear, a logit within
+    # reach of the maximum elsewhere, and the two sides may differ only on such near ties
+    h, w, _ = W.make_lm_head(300, 256, 6000, seed=78, planted=0.0)
+    got = run_gpu(clv, h, w)
+    n_exact = check_rows(oracle, h, w, got)
+    ref = oracle.lm_head_argmax(h, w)
+    assert n_exact >= 150
+    assert (got == ref).mean() >= 0.9
+
+
+def test_wait_that_runs_out_is_reported_and_leaves_the_library_usable(clv, oracle):
+    # the kernel's waits are bounded; with the bound cut to a few dozen SM cycles the wait for the
+    # first weight tile runs out: the call succeeds, status says CLV_ERR_TIMEOUT, nothing faults,
+    # and the same workspace serves an ordinary call right afterwards
+    h, w, win = W.make_lm_head(40, 128, 3000, seed=41)
+    hid, wgt = W.as_torch_bf16(h).cuda(), W.as_torch_bf16(w).cuda()
+    ids = torch.full((40,), -7, dtype=torch.int32, device="cuda")
+    status = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+    ws = clv.new_workspace(clv.make_shape(1, 1, 1, 1, vocab=8), None, 0)
+    try:
+        clv.clv_test_set_wait_limit(32)
+        clv.clv_lm_head_argmax(hid, wgt, ids, status, ws)
+        torch.cuda.synchronize()
+    finally:
+        clv.clv_test_set_wait_limit(0)
+    assert int(status.item()) == clv.CLV_ERR_TIMEOUT
+    clv.clv_lm_head_argmax(hid, wgt, ids, status, ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(ids.cpu().numpy(), win)
+    assert np.array_equal(ids.cpu().numpy(), oracle.lm_head_argmax(h, w))
 
 
 def test_full_size_sampled_rows(clv, oracle):

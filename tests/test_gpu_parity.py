@@ -8,7 +8,7 @@ import pytest
 import torch
 
 from paper_2408_00264_b200 import workloads as W
-from parity_util import assert_attn_close, sample_rows
+from parity_util import assert_attn_close, attn_errors, log_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -49,6 +49,10 @@ def check_attention(oracle, w, st, rows=None):
     assert np.array_equal(st.status[0].cpu().numpy(), status)
     assert_attn_close(got, ref, w.cfg.name)
     assert np.abs(got_lse - lse).max() < 2e-3
+    if w.cfg.name in W.CONFIGS:
+        a, r = attn_errors(got, ref)
+        log_parity(w.cfg.name, rows=int(np.prod(got.shape[:-1])), max_abs=a, max_row_rel=r,
+                   max_lse_abs=float(np.abs(got_lse - lse).max()))
     return ref
 
 
@@ -89,19 +93,13 @@ def full_step(clv, oracle, w, rows=None):
 
 
 # ------------------------------------------------------------------ the five stated workloads
-@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5"])
 def test_config_full_compare(clv, oracle, name):
+    # every attention row, every id, the accepted paths and the whole committed cache, at the
+    # stated sizes (the checker needs a few seconds for C4 and some tens of seconds for C5)
     w = W.generate(W.CONFIGS[name])
     alen = full_step(clv, oracle, w)
     assert (alen >= 1).all()
-
-
-@pytest.mark.parametrize("name", ["C4", "C5"])
-def test_config_sampled_attention(clv, oracle, name):
-    # the checker evaluates sampled (b, node, head) rows one by one; integer outputs and the
-    # committed cache are compared in full
-    w = W.generate(W.CONFIGS[name])
-    full_step(clv, oracle, w, rows=sample_rows(w, 48, seed=11))
 
 
 # ------------------------------------------------------------------ shapes around tile edges
@@ -143,24 +141,6 @@ def test_attention_group_sizes_that_do_not_divide_128(clv, oracle, hq, hkv, n_no
     st.tree_attn()
     torch.cuda.synchronize()
     check_attention(oracle, w, st)
-
-
-@pytest.mark.parametrize("paged", [False, True])
-def test_attention_both_kernels_agree_with_the_checker(clv, oracle, paged, monkeypatch):
-    # CLV_ATTN_PATH=mma forces the warp-level kernel on a shape the tcgen05 kernel normally serves
-    cfg = W.small_config(batch=3, n_q_heads=8, n_kv_heads=2, ctx=(100, 900), n_nodes=64, vocab=64,
-                         paged=paged, seed=W.BASE_SEED + 21)
-    w = W.generate(cfg)
-    outs = []
-    for path in ("tc", "mma"):
-        monkeypatch.setenv("CLV_ATTN_PATH", path)
-        st = make_step(w)
-        st.tree_attn()
-        torch.cuda.synchronize()
-        check_attention(oracle, w, st)
-        outs.append(W.bf16_bits_to_f64(bits(st.out)))
-    monkeypatch.delenv("CLV_ATTN_PATH")
-    assert np.abs(outs[0] - outs[1]).max() < 1e-2
 
 
 def test_attention_many_splits_and_ragged(clv, oracle):
@@ -252,6 +232,29 @@ def test_attention_flags_bad_sequences(clv, oracle):
     ref = oracle.tree_attn(w.q, w.k_cache, w.v_cache, w.k_tree, w.v_tree, w.parent, w.ctx_len,
                            w.scale)[0]
     assert_attn_close(bits(st.out)[0], ref[0], "valid sequence beside bad ones")
+
+
+def test_attention_wait_that_runs_out_is_reported_and_leaves_the_library_usable(clv, oracle):
+    # Every on-chip wait of the attention kernel is bounded.  With the bound cut to a few dozen SM
+    # cycles the ordinary wait for the first tile (a load from device memory takes far longer)
+    # runs out: the blocks must leave in order - copies and tensor-core work in flight waited for,
+    # tensor memory released - the call itself succeeds, and status[] says CLV_ERR_TIMEOUT.
+    # Nothing faults; the next call, on the same workspace, is an ordinary one.
+    cfg = W.small_config(batch=2, n_q_heads=8, n_kv_heads=2, ctx=(300, 700), n_nodes=24, vocab=64,
+                         seed=W.BASE_SEED + 404)
+    w = W.generate(cfg)
+    st = make_step(w)
+    try:
+        clv.clv_test_set_wait_limit(32)
+        st.tree_attn()
+        torch.cuda.synchronize()
+    finally:
+        clv.clv_test_set_wait_limit(0)
+    assert st.status[0].cpu().tolist() == [clv.CLV_ERR_TIMEOUT] * 2
+    st.status.zero_()
+    st.tree_attn()
+    torch.cuda.synchronize()
+    check_attention(oracle, w, st)
 
 
 # ------------------------------------------------------------------ argmax
@@ -468,3 +471,25 @@ def test_verify_step_from_host_buffers(clv, oracle):
                                           w.ctx_len)
     assert np.array_equal(st.ctx_len.cpu().numpy(), new_len)
     assert np.array_equal(bits(st.k_cache), kc) and np.array_equal(bits(st.v_cache), vc)
+
+
+def test_host_step_with_a_bad_argument_leaves_the_stream_empty(clv, oracle):
+    # a stride the argmax refuses: the call must fail before its first copy, so neither the
+    # staging area nor the device-side context lengths change
+    cfg = W.small_config(batch=2, n_q_heads=4, n_kv_heads=2, ctx=(20, 100), n_nodes=10, vocab=1000)
+    w = W.generate(cfg, ld_pad=4)                       # ld = 1004, not a multiple of 8
+    st = make_step(w, logits=False)
+    pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+    host = [pin(x) for x in (w.q, w.k_tree, w.v_tree, w.parent, w.tokens, w.logits)]
+    hin = clv.ClvHostInputs(*[t.data_ptr() for t in host], w.logits.shape[-1])
+    outs = [torch.zeros(4096, dtype=torch.int32).pin_memory() for _ in range(6)]
+    hout = clv.ClvHostOutputs(*[t.data_ptr() for t in outs])
+    staging = torch.full((clv.clv_staging_bytes(st.shape, w.logits.shape[-1]),), 0x5A, dtype=torch.uint8,
+                         device="cuda")
+    ctx_before = st.ctx_len.clone()
+    code = clv.clv_verify_step_host(st.shape, st.cache, hin, hout, st.ctx_len, st.max_ctx_len, st.scale,
+                                    staging, st.workspace, check=False)
+    torch.cuda.synchronize()
+    assert code == clv.CLV_ERR_ALIGN
+    assert bool((staging == 0x5A).all()) and torch.equal(st.ctx_len, ctx_before)
+    assert all(int(t.abs().sum()) == 0 for t in outs)

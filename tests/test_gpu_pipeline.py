@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("paged", [False, True])
 def test_draft_to_commit(oracle, paged):
     if not torch.cuda.is_available():
-        pytest.skip("needs a GPU")
+        pytest.fail("these tests need a CUDA device")
     from paper_2408_00264_b200 import binding as clv
     from paper_2408_00264_b200.step import VerifyStep, bits_of
     B, N, V, K = 3, 64, 3000, 128

@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def clv():
     if not torch.cuda.is_available():
-        pytest.skip("needs a GPU")
+        pytest.fail("these tests need a CUDA device")
     from paper_2408_00264_b200 import binding
     binding.lib()
     return binding

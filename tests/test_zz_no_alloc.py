@@ -37,7 +37,7 @@ def _logits(rows, vocab, seed):
 
 
 @pytest.mark.parametrize("batch,nodes,vocab", [(2, 5, 2049), (4, 64, 128256), (1, 16, 32000)])
-def test_noalloc_matches_workspace_entry_point_twice(clv, batch, nodes, vocab):
+def test_noalloc_matches_workspace_entry_point_twice(clv, oracle, batch, nodes, vocab):
     shape = clv.make_shape(batch, nodes, 1, 1, vocab, 1)
     ws = clv.new_workspace(shape, None, 0)
     ids_ref = torch.empty(batch, nodes, dtype=torch.int32, device="cuda")
@@ -53,6 +53,8 @@ def test_noalloc_matches_workspace_entry_point_twice(clv, batch, nodes, vocab):
         torch.cuda.synchronize()
         assert torch.equal(ids_new, ids_ref)    # integer output: exact
         assert int(ids_new.min()) >= 0 and int(ids_new.max()) < vocab
+        # and both are what the CPU checker finds, so this file stands on its own
+        assert np.array_equal(ids_new.cpu().numpy().reshape(-1), oracle.argmax(lg, vocab))
 
 
 def test_noalloc_rejects_sizes_beyond_its_fixed_scratch(clv):
@@ -64,3 +66,25 @@ def test_noalloc_rejects_sizes_beyond_its_fixed_scratch(clv):
     assert "scratch" in clv.clv_status_string(code)
     with pytest.raises(clv.ClvError):
         clv.clv_accept_argmax_noalloc(too_many_rows, d, 32000, ids)
+    # as many rows as allowed, but a vocabulary so wide that rows x (thread blocks per row)
+    # exceeds the array: 4096 rows x 33 pieces of 32768 logits
+    too_many_pieces = clv.make_shape(32, 128, 1, 1, 33 * 32768, 1)
+    code = clv.clv_accept_argmax_noalloc(too_many_pieces, d, 33 * 32768, ids, check=False)
+    assert code == clv.CLV_ERR_TOO_LARGE
+
+
+def test_noalloc_allocates_nothing(clv):
+    # the point of the entry point: the free device memory is the same before and after a call
+    # (the first call on the device has already been made by the tests above or is made here)
+    vocab, rows = 32000, 16
+    lg, ld = _logits(rows, vocab, seed=5)
+    d = torch.from_numpy(lg.view(np.int16)).cuda()
+    shape = clv.make_shape(1, rows, 1, 1, vocab, 1)
+    ids = torch.empty(1, rows, dtype=torch.int32, device="cuda")
+    clv.clv_accept_argmax_noalloc(shape, d, ld, ids)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    clv.clv_accept_argmax_noalloc(shape, d, ld, ids)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
