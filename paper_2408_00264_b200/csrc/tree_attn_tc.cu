@@ -1,29 +1,34 @@
 // Tree attention (Sec. 2.1) on the 5th-generation tensor cores: tcgen05.mma with accumulators in
 // tensor memory, K/V/Q tiles staged by TMA into 128-byte-swizzled shared memory.
 //
-// One thread block owns up to 256 query rows of one (sequence, kv head) - a row is a
-// (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes reuse every
-// K/V byte - and a contiguous range of key tiles (cache tiles first, then the tree's own keys).
-// A row tile of 128 rows holds whole nodes: 128 / G of them (rounded down; its other rows idle).
-// A key tile is 128 keys (an MMA costs about the same for 64 as for 128 columns, so wide S tiles
-// halve the tensor time); tiles are loaded as 64-key pieces, which is also the page size of a
-// paged cache.  K and V travel through separate
-// rings so that a K buffer is refilled as soon as its Q K^T is done.
-// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation), warps 2-5 and
-// 6-9 = two softmax groups of 128 threads, one thread per query row ("slot" 0 and 1).
-//   MT = 2 (more than one row tile): slot s works on row tile s; both slots consume every K/V tile.
-//   MT = 1: both slots work on the same 128 rows; slot s takes every second key tile and the two
-//           accumulators are merged like split-KV partials.
-// Split-KV: the blocks that share a row tile form a thread-block cluster; each stages its
-// accumulators in its own shared memory and every block finalises a share of the rows by reading
-// its peers' staging areas (distributed shared memory), so no partial result touches global memory.
-// Per slot and key tile:  S = Q K^T (tcgen05.mma -> TMEM)  ->  softmax thread reads its row of S,
-// masks, exponentiates against a lazily updated reference maximum, writes P (bf16) back to tensor
-// memory  ->  O += P V (tcgen05.mma with A from TMEM, accumulator stays in TMEM).  While one slot is in its softmax
-// the tensor core works for the other.  The tree columns are masked with per-node ancestor
-// bitsets derived from parent[] on chip; masked scores are replaced, not added to, so they
-// contribute exactly zero.  Every mbarrier wait is bounded: on expiry the block raises a flag,
-// all roles leave their loops, in-flight copies and MMAs are drained, TMEM is released and
+// Query row = (tree node, head-in-group) pair, so all G heads of a GQA group and all tree nodes
+// reuse every K/V byte.  A row tile of 128 rows holds whole nodes: 128 / G of them (rounded down;
+// its other rows idle).  One thread block owns ONE row tile of one (sequence, kv head) and a
+// contiguous range of the key axis (cache keys first, then the tree's own), walked in tiles of
+// 128 keys that are loaded as 64-key pieces (also the page size of a paged cache).
+//   CG = 1: the block works alone (the unit has a single row tile).
+//   CG = 2: two blocks on neighbouring SMs share every MMA (cta_group::2, M = 256): each holds its
+//           own row tile, and each stages only HALF of every K and V tile - K: one 64-key piece,
+//           V: one 64-wide half of the head dimension - so a unit of two row tiles costs each SM
+//           half the shared-memory fill.  Every block's TMA copies signal its own barriers (so it
+//           can wait for, patch and drain its own tiles); a relay thread of the odd block forwards
+//           the completions to the even block, whose single thread issues the pair's MMAs.
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (even block) or relay (odd block), owner of
+// the tensor-memory allocation; warps 2-9 = softmax, two threads per query row: thread `ch` of a
+// row takes the 64 columns of piece `ch` of every key tile.
+// Tensor memory: three score buffers of 128 columns and one output accumulator of 128.  The
+// issuer runs Q K^T up to three tiles ahead, so the softmax threads find the next scores ready
+// when they finish a tile, and P V of a tile runs beside the softmax of the next one.
+// Per tile: S = Q K^T -> the row's two threads read their halves, mask, exponentiate against a
+// lazily updated reference maximum and add up the row -> P (bf16) overwrites consumed score
+// columns -> O += P V (A operand from tensor memory).  The tree columns are masked with per-node
+// ancestor bitsets derived from parent[] on chip; masked scores are replaced, not added to, so
+// they contribute exactly zero.
+// Split-KV: the blocks (pairs) that share a row tile form one thread-block cluster; each stages
+// its accumulator in its own shared memory and every block finalises a share of the rows by
+// reading its peers' staging areas (distributed shared memory): no partial result touches global
+// memory.  Every wait is bounded: on expiry the block raises a flag, all roles leave their loops,
+// in-flight copies and MMAs are drained, the cluster meets, tensor memory is released and
 // CLV_ERR_TIMEOUT is reported for the sequence.
 #include <cooperative_groups.h>
 #include <cuda.h>
@@ -41,20 +46,23 @@ namespace {
 
 constexpr int PG = CLV_PAGE_SIZE;      // 64: keys per TMA piece (= page size)
 constexpr int HD = CLV_HEAD_DIM;       // 128
-constexpr int BM = 128;                // rows per MMA / per slot
+constexpr int BM = 128;                // rows per block
+constexpr int BN = 128;                // keys per tile
+constexpr int PPT = BN / PG;           // pieces per tile
+constexpr int NSB = 3;                 // score buffers (= depth of the K ring)
 constexpr int kThreads = 320;
+constexpr int kSoftmaxThreads = 256;
 constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
 constexpr uint32_t kTmemCols = 512;
-constexpr float kRowSumLimit = 256.0f;        // a row of P may sum to 2^8 before the reference is replaced
+constexpr float kRowSumLimit = 256.0f;        // a thread's part of a row of P may sum to 2^8 before the reference is replaced
 
-template <int MT>
+template <int CG>
 struct Cfg {
-  static constexpr int BN = 128;                         // keys per tile
-  static constexpr int kStagesK = (MT == 1) ? 3 : 2;     // depth of the K ring
-  static constexpr int kStagesV = 2;                     // depth of the V ring
-  static constexpr uint32_t kTile = BN * HD * 2;         // bytes of one K (or V) tile
-  static constexpr uint32_t kSmem = MT * kQTile + (kStagesK + kStagesV) * kTile + 1024;
+  static constexpr int KST = NSB;                        // a K buffer and a score buffer free together
+  static constexpr int VST = (CG == 2) ? NSB : 2;        // depth of the V ring
+  static constexpr uint32_t kStage = BN * HD * 2 / CG;   // bytes of this block's share of a K (or V) tile
+  static constexpr uint32_t kSmem = kQTile + (KST + VST) * kStage + 1024;
 };
 
 struct Params {
@@ -67,24 +75,17 @@ struct Params {
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
   int longest_first;  // hand out sequences in order of decreasing context length
-  int row_ctas;    // thread blocks along the row axis per (sequence, kv head)
-  int splits;      // thread blocks along the key axis = cluster size (1, 2, 4 or 8)
+  int row_groups;  // clusters along the row axis per (sequence, kv head); each covers CG row tiles
+  int tiles;       // row tiles per (sequence, kv head)
+  int splits;      // blocks (pairs) along the key axis; cluster size = CG * splits
   float scale_log2;
   long long wait_limit;   // SM cycles a bounded wait may last
   unsigned* tickets;      // per sequence: [2b] blocks that have finished, [2b+1] error bits; zero between calls
   int blocks_per_seq;
 };
 
-constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 x 128] += P[128 x 16k] V[16k x 128]
-
-// Distributed shared memory: address of the same variable in block `rank` of the cluster, and a
-// 16-byte load from it.  The loads are volatile asm so that a batch of them is issued back to back
-// (all in flight together) before the first result is used.
-__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-  return r;
-}
+// Distributed shared memory: 8- and 16-byte loads from a peer's shared memory.  Volatile asm, so
+// that a batch of them is issued back to back (all in flight) before the first result is used.
 __device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
@@ -92,7 +93,11 @@ __device__ __forceinline__ float4 dsmem_ld16(uint32_t addr) {
                : "r"(addr));
   return v;
 }
-
+__device__ __forceinline__ uint2 dsmem_ld8u(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared::cluster.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -102,46 +107,60 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-
-__device__ __forceinline__ uint2 dsmem_ld8u(uint32_t addr) {
-  uint2 v;
-  asm volatile("ld.shared::cluster.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-  return v;
-}
 __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t u) {
   return __half22float2(*reinterpret_cast<const __half2*>(&u));
 }
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 
-// Final combination of NSRC accumulators per output row, for the rows [k_begin, k_end) that this
-// block finalises.  The staged accumulators are fp16 (each row scaled by a power of two of its
-// own, which the weight undoes), 256 bytes per row.  One warp takes 32 / NSRC rows at a time (32
-// remote 8-byte loads in flight per lane); lane j owns output columns 4j .. 4j+3.  w[] holds the
-// normalised weights divided by the rows' scales.
-template <int NSRC, int MT>
-__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank,
-                                           int rot, int warp, int lane, int tile_base, int RT, int rows_total, int G,
-                                           int64_t seq_row0, int Hq, int head0, uint16_t* out) {
-  constexpr int RB = 32 / NSRC;
+template <int CG>
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  if (CG == 2) umma_bf16_pair(d, a, b, idesc, acc);
+  else umma_bf16(d, a, b, idesc, acc);
+}
+template <int CG>
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  if (CG == 2) umma_bf16_ts_pair(d, a, b, idesc, acc);
+  else umma_bf16_ts(d, a, b, idesc, acc);
+}
+// one arrival, once the MMAs issued so far are complete, at barrier `bar` of every block of the pair
+template <int CG>
+__device__ __forceinline__ void commit_all(uint32_t bar, uint16_t pair_mask) {
+  if (CG == 2) umma_commit_pair_both(bar, pair_mask);
+  else umma_commit(bar);
+}
+
+// Final combination of NSRC accumulators per output row, for the rows [first_row, first_row +
+// per_rank) of the tile that this block finalises.  The staged accumulators are fp16 (each row
+// scaled by a power of two of its own, which the weight undoes), 256 bytes per row.  One warp takes
+// 16 / NSRC rows at a time (16 remote 8-byte loads in flight per lane); lane j owns output
+// columns 4j .. 4j+3.  w[] holds the normalised weights divided by the rows' scales; source q of
+// a row lives in cluster rank q * rank_stride + rank_base.
+template <int NSRC>
+__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank, int rot,
+                                           int rank_stride, int rank_base, int warp, int lane, int tile_row0,
+                                           int RT, int rows_total, int G, int64_t seq_row0, int Hq, int head0,
+                                           uint16_t* out) {
+  constexpr int RB = 16 / NSRC;
   for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
     uint2 x[RB * NSRC];
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
-      const int k = min(k0 + u, per_rank - 1);
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
+      const int trow = first_row + min(k0 + u, per_rank - 1);
       const uint32_t off = (uint32_t)(trow * (HD * 2) + (((lane >> 1) ^ (trow & 15)) << 4) + ((lane & 1) << 3));
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
         const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
-        const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-        x[u * NSRC + j] = dsmem_ld8u(dsmem_addr(sO_addr + (uint32_t)(qs * BM * HD * 2) + off, qc));
+        x[u * NSRC + j] = dsmem_ld8u(cluster_map(sO_addr + off, (uint32_t)(q * rank_stride + rank_base)));
       }
     }
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
       if (k0 + u >= per_rank) continue;
       const int k = k0 + u;
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const int rg = (tile_base + tile) * RT + trow;
+      const int trow = first_row + k;
+      const int rg = tile_row0 + trow;
       if (trow >= RT || rg >= rows_total) continue;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -158,68 +177,93 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
 }
 
 // ------------------------------------------------------------------------------------ kernel
-template <int MT>
+template <int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                     const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
                     const __grid_constant__ CUtensorMap tm_vt, const Params p) {
-  constexpr int BN = Cfg<MT>::BN;          // keys per tile
-  constexpr int PPT = BN / PG;             // 64-key pieces per tile
-  constexpr int KST = Cfg<MT>::kStagesK, VST = Cfg<MT>::kStagesV;
-  constexpr uint32_t kTile = Cfg<MT>::kTile;
-  constexpr uint32_t kHalf = kTile / 2;    // one 64-wide half of the head dimension: [BN keys][64 d]
-  constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 x BN] = Q[128 x 16k] K[BN x 16k]^T
+  constexpr int KST = Cfg<CG>::KST, VST = Cfg<CG>::VST;
+  constexpr uint32_t kStage = Cfg<CG>::kStage;
+  constexpr uint32_t kKHalf = kStage / 2;   // K stage: [64-wide half of d][keys of this block][64 d]
+  constexpr bool kVOwnRing = (VST != NSB);  // V buffers then have hand-back barriers of their own
+  constexpr uint32_t kIdescQK = make_idesc(BM * CG, BN, false);  // S[rows x 128 keys] = Q K^T
+  constexpr uint32_t kIdescPV = make_idesc(BM * CG, HD, true);   // O[rows x 128 d] += P V
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
-  __shared__ __align__(8) unsigned long long s_bar[2 * KST + 2 * VST + 8];
+  // barriers: K full [KST] | V full [VST] | S full [NSB] | P full [NSB] | P V done [NSB] | V empty [VST] | Q |
+  //           drain | the peer's K [KST], V [VST] and Q have landed (arrivals of the relay; even block only)
+  constexpr int B_KF = 0, B_VF = B_KF + KST, B_SF = B_VF + VST, B_PF = B_SF + NSB, B_PV = B_PF + NSB,
+                B_VE = B_PV + NSB, B_Q = B_VE + VST, B_DR = B_Q + 1, B_KP = B_DR + 1, B_VP = B_KP + KST,
+                B_QP = B_VP + VST, NBAR = B_QP + 1;
+  __shared__ __align__(8) unsigned long long s_bar[NBAR];
   __shared__ int s_tile_ok[VST];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ float4 s_ml[2][BM];   // (reference maximum, row sum, 1 / staging scale, -) of both slots, for the merge
-  __shared__ float s_w[2 * BM];    // merge: normalised weight of every (row of this rank, source)
+  __shared__ int s_redo[8];        // per softmax warp: the last tile in which one of its row sums was suspect
+  __shared__ int s_fail[8];        // per softmax warp: one of its waits has run out
+  __shared__ float s_xch[2][BM];   // values exchanged between the two threads of a row
+  __shared__ float s_xch2[2][BM];
+  __shared__ float4 s_ml[BM];      // (reference maximum, row sum, 1 / staging scale, -) for the merge
+  __shared__ float s_w[BM];        // merge: normalised weight of every (row of this rank, source)
+  __shared__ int s_seq;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int unit = blockIdx.x / p.row_ctas, row_cta = blockIdx.x - unit * p.row_ctas;
-  const int split = blockIdx.y;
+  const int CS = CG * p.splits;                       // cluster size
+  const int crank = (int)(blockIdx.x % (unsigned)CS); // rank in the cluster (clusters are laid along x)
+  const int c = (CG == 2) ? (crank & 1) : 0;          // block of the pair
+  const int split = crank / CG;
+  const int cluster_id = (int)(blockIdx.x / (unsigned)CS);
+  const int unit = cluster_id / p.row_groups, rgrp = cluster_id - unit * p.row_groups;
   int b = unit / p.Hkv;
   const int kvh = unit - b * p.Hkv;
   const int N = p.N, G = p.G, rows_total = G * N;
-  // A row tile holds whole nodes: BM / G of them, i.e. RT = (BM / G) * G of its 128 rows (all 128
-  // when G divides 128); the remaining rows of the tile are idle.
-  const int RT = (BM / G) * G;
+  const int RT = (BM / G) * G;                        // rows of a tile that hold whole nodes
+  const int tile_idx = rgrp * CG + c;                 // this block's row tile of the unit
+  const bool has_rows = tile_idx < p.tiles;
+  const bool leader = (c == 0);
+  const uint32_t leader_rank = (uint32_t)(crank & ~(CG - 1));
+  const uint16_t pair_mask = (uint16_t)((CG == 2 ? 3u : 1u) << leader_rank);
+
   // ---- set-up that reads no global memory: barriers, tensor memory, descriptor prefetch.  The
   //      kernel is launched with programmatic stream serialisation, so this part may run while the
-  //      previous kernel of the stream drains; everything after the grid dependency wait sees that
-  //      kernel's results.
-  constexpr int NRING = 2 * KST + 2 * VST;
+  //      previous kernel of the stream drains.
   const uint32_t bar0 = smem_u32(&s_bar[0]);
+  auto bar = [&](int idx) { return bar0 + 8u * (uint32_t)idx; };
   if (tid == 0) {
-    for (int i = 0; i < NRING; ++i) mbar_init(bar0 + 8u * i, 1);                 // K/V rings
-    mbar_init(bar0 + 8u * (NRING), 1);                                           // Q
-    for (int s2 = 0; s2 < 2; ++s2) {
-      mbar_init(bar0 + 8u * (NRING + 1 + s2), 1);                                // S ready
-      mbar_init(bar0 + 8u * (NRING + 3 + s2), BM);                               // P ready
-      mbar_init(bar0 + 8u * (NRING + 5 + s2), 1);                                // P V done
+    for (int i = 0; i < KST; ++i) { mbar_init(bar(B_KF + i), 1); mbar_init(bar(B_KP + i), 1); }
+    for (int i = 0; i < VST; ++i) {
+      mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1); mbar_init(bar(B_VP + i), 1);
     }
-    mbar_init(bar0 + 8u * (NRING + 7), 1);                                       // drain
+    for (int i = 0; i < NSB; ++i) {
+      mbar_init(bar(B_SF + i), 1);
+      mbar_init(bar(B_PF + i), 8u * CG);   // one arrival per softmax warp of the pair
+      mbar_init(bar(B_PV + i), 1);
+    }
+    mbar_init(bar(B_Q), 1);
+    mbar_init(bar(B_QP), 1);
+    mbar_init(bar(B_DR), 1);
     s_abort = 0;
+    for (int i = 0; i < 8; ++i) { s_redo[i] = -1; s_fail[i] = 0; }
     fence_barrier_init();
     fence_async_smem();
   }
-  if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+  if (warp == 1) {
+    if (CG == 2) tmem_alloc_pair(smem_u32(&s_tmem), kTmemCols);
+    else tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+  }
   if (tid == 64) {
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
     tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
   }
+  __syncthreads();                     // this block's barriers exist ...
+  if (CG == 2) cluster_arrive();       // ... and the peer learns of it at the matching wait below
   cudaGridDependencySynchronize();
 
   if (p.longest_first) {
     // More blocks than SMs and contexts of different lengths (ragged batch): hand the sequences
     // out longest first, so that the block scheduler packs the short ones into the gaps.  Block
-    // group `b` takes the sequence whose length has rank b (ties by index); every thread ranks
-    // at most one sequence.
-    __shared__ int s_seq;
+    // group `b` takes the sequence whose length has rank b (ties by index).
     const int want = b;
     for (int i = tid; i < p.B; i += kThreads) {
       const int Li = p.ctx_len[i];
@@ -234,8 +278,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     b = s_seq;
   }
 
-  // ---- per-sequence checks: everybody reads parent[] and the context length; the one block-wide
-  //      synchronisation below publishes them together with the set-up above --------------------
+  // ---- per-sequence checks ------------------------------------------------------------------
   const int L = p.ctx_len[b];
   bool bad = false;
   for (int i = tid; i < N; i += kThreads) {
@@ -250,12 +293,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_before();
   const int seq_bad = __syncthreads_or(bad ? 1 : 0);  // same verdict in every block of the sequence
   tc_fence_after();
+  if (CG == 2) cluster_wait();         // the peer's barriers exist: remote arrivals may begin
   const uint32_t tmem = s_tmem;
-  const bool reporter = (row_cta == 0 && split == 0 && kvh == 0);
+  const bool reporter = (rgrp == 0 && crank == 0 && kvh == 0);
   // status[b] is written once, by whichever block of the sequence finishes last: every block adds
   // its error bits (1 malformed input, 2 a wait ran out) to the sequence's word in the workspace
   // and then takes a ticket; the holder of the last ticket turns the bits into the status code and
-  // leaves both words zero for the next call.  So no verdict can be overwritten by a later "fine".
+  // leaves both words zero for the next call.
   auto report = [&](unsigned bits) -> unsigned {   // one thread per block; returns the ticket
     if (bits) atomicOr(p.tickets + 2 * b + 1, bits);
     __threadfence();
@@ -267,207 +311,261 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const unsigned bits = atomicExch(p.tickets + 2 * b + 1, 0u);
     p.status[b] = (bits & 1u) ? CLV_ERR_TREE : (bits & 2u) ? CLV_ERR_TIMEOUT : CLV_OK;
   };
+  auto release_tmem = [&]() {   // warp 1 of every block of the pair
+    if (CG == 2) tmem_dealloc_pair(tmem, kTmemCols);
+    else tmem_dealloc(tmem, kTmemCols);
+  };
   if (seq_bad) {  // the whole cluster leaves together; nothing has been issued yet
-    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 1) release_tmem();
     if (tid == 0) publish(report(1u));
     return;
   }
 
-  // ---- tile range and per-slot rounds -------------------------------------------------------
+  // ---- this block's range of the key axis -----------------------------------------------------
   // The key axis is cut in 64-key pieces: p_cache pieces of context, then the tree's own pieces.
-  // A block takes a contiguous range of pieces (so the split balances to one piece) and walks it
-  // in tiles of PPT pieces; a tile may end early or mix context and tree pieces.
+  // A split takes a contiguous range of pieces and walks it in tiles of two pieces; the last tile
+  // of a range may hold one piece only.
   const int p_total = p_cache + (N + PG - 1) / PG;
   const int pc_begin = (int)((int64_t)split * p_total / p.splits);
   const int pc_end = (int)((int64_t)(split + 1) * p_total / p.splits);
-  const int n_tiles = (pc_end - pc_begin + PPT - 1) / PPT;
-  // local tile index of round r of slot s: MT == 2: r;  MT == 1: 2 r + s
-  const int rounds0 = (MT == 2) ? n_tiles : (n_tiles + 1) / 2;
-  const int rounds1 = (MT == 2) ? n_tiles : n_tiles / 2;
+  const int T = (pc_end - pc_begin + PPT - 1) / PPT;   // tiles of this block
 
   // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem_base;
-  const uint32_t sK = sQ + MT * kQTile;      // ring of KST K tiles
-  const uint32_t sV = sK + KST * kTile;      // ring of VST V tiles
+  const uint32_t sK = sQ + kQTile;           // ring of KST K stages
+  const uint32_t sV = sK + KST * kStage;     // ring of VST V stages
   uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
-
-  auto bar_k_full = [&](int st) { return bar0 + 8u * st; };
-  auto bar_k_empty = [&](int st) { return bar0 + 8u * (KST + st); };
-  auto bar_v_full = [&](int st) { return bar0 + 8u * (2 * KST + st); };
-  auto bar_v_empty = [&](int st) { return bar0 + 8u * (2 * KST + VST + st); };
-  const uint32_t bar_q = bar0 + 8u * NRING;
-  auto bar_s_full = [&](int s) { return bar0 + 8u * (NRING + 1 + s); };
-  auto bar_p_full = [&](int s) { return bar0 + 8u * (NRING + 3 + s); };
-  auto bar_pv_done = [&](int s) { return bar0 + 8u * (NRING + 5 + s); };
-  const uint32_t bar_drain = bar0 + 8u * (NRING + 7);
 
   volatile int* abort_flag = &s_abort;
   const long long wlim = p.wait_limit;
-  // columns: S of slot s at BN s (P, two bf16 per column, overwrites its first BN/2 columns once
-  // the scores have been read); O of slot s at 2 BN + 128 s
-  auto tmem_S = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_P = [&](int s) { return tmem + (uint32_t)(s * BN); };
-  auto tmem_O = [&](int s) { return tmem + (uint32_t)(2 * BN + s * HD); };
+  auto tmem_S = [&](int buf) { return tmem + (uint32_t)(buf * BN); };   // P overwrites its first 64 columns
+  const uint32_t tmem_O = tmem + (uint32_t)(NSB * BN);
 
   int issued_k = 0, issued_v = 0;  // producer bookkeeping for the drain
 
-  // per-thread state of the softmax groups (warps 2..9); declared here because the epilogue runs
+  // per-thread state of the softmax threads (warps 2..9); declared here because the epilogue runs
   // after block-wide synchronisation points that all roles must reach together
-  const int slot = warp >= 2 ? (warp - 2) >> 2 : 0;
+  const int sw = warp >= 2 ? warp - 2 : 0;
+  const int ch = sw >> 2;                        // which 64-key piece of every tile (= column half)
   const int quarter = warp & 3;                  // TMEM lanes this warp may touch
   const int row = quarter * 32 + lane;           // row inside the 128-row tile
-  const int my_rounds = slot == 0 ? rounds0 : rounds1;
-  const int r_glob = (row_cta * MT + ((MT == 2) ? slot : 0)) * RT + row;
-  const bool row_valid = row < RT && r_glob < rows_total;
+  const int r_glob = tile_idx * RT + row;
+  const bool row_valid = has_rows && row < RT && r_glob < rows_total;
   const int node = row_valid ? r_glob / G : 0;
   const int gq = row_valid ? r_glob - node * G : 0;
   const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+  const int pair_bar = 2 + quarter;              // named barrier of the two warps that share rows
   float m_ref = -INFINITY, l_run = 0.f;
 
   if (warp == 0) {
     // =========================== TMA producer ===============================================
-    if (n_tiles > 0) {
-      int page_cache = 0;   // lane j: pool page of context piece (page_base + j)
-      int page_base = -64;
-      bool ok = true;
-      for (int i = 0; i < n_tiles && ok; ++i) {
-        const int ks = i % KST, vs = i % VST;
-        const int g0 = pc_begin + i * PPT;  // first piece of this tile
-        if (p.paged && g0 < p_cache && g0 + PPT > page_base + 32) {  // warp-uniform refill
-          page_base = g0;
-          const int pc = g0 + lane;
-          page_cache = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
-        }
-        int row0[PPT];          // first source row of each piece, -1: piece not present
-        bool is_tree[PPT];
-        int tile_ok = 1;
-#pragma unroll
-        for (int j = 0; j < PPT; ++j) {
-          const int g = g0 + j;
-          int pg = __shfl_sync(0xFFFFFFFFu, page_cache, (g - page_base) & 31);
-          is_tree[j] = g >= p_cache;
-          if (g >= pc_end) {
-            row0[j] = -1;
-          } else if (is_tree[j]) {
-            row0[j] = b * N + (g - p_cache) * PG;
-          } else if (p.paged) {
-            if (pg < 0 || pg >= p.n_pages) { tile_ok = 0; pg = 0; }  // flagged by the reporter; masked
-            row0[j] = pg * PG;
-          } else {
-            row0[j] = b * p.cap_tokens + g * PG;
+    // K and V advance independently: whichever ring has a free buffer gets its next tile.  Lane j
+    // caches the pool page of context piece (base + j) for each ring (paged cache).
+    int kt = 0, vt = 0;
+    int pk_page = 0, pk_base = -64, pv_page = 0, pv_base = -64;
+    long long t_idle = clock64();
+    bool ok = true;
+    while (ok && (kt < T || vt < T)) {
+      bool progress = false;
+      // ---- K of tile kt: this block's piece(s)
+      if (kt < T) {
+        const int st = kt % KST;
+        int ready = 1;
+        if (kt >= KST && lane == 0) ready = mbar_test(bar(B_SF + st), ((kt / KST) - 1) & 1) ? 1 : 0;
+        ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
+        if (ready) {
+          const int g0 = pc_begin + kt * PPT;
+          if (p.paged && g0 < p_cache && g0 + PPT > pk_base + 32) {
+            pk_base = g0;
+            const int pc = g0 + lane;
+            pk_page = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
           }
-        }
-        if (lane == 0) {
-          int n_pieces = 0;
+          int row0[PPT];
+          bool is_tree[PPT];
 #pragma unroll
-          for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
-          const uint32_t bytes = (uint32_t)n_pieces * 2u * kPiece;  // both halves of the head dim
-          if (i >= KST) ok = mbar_wait(bar_k_empty(ks), ((i / KST) - 1) & 1, abort_flag, wlim);
-          if (ok) {
-            mbar_expect_tx(bar_k_full(ks), bytes);
+          for (int j = 0; j < PPT; ++j) {
+            const int g = g0 + j;
+            int pg = __shfl_sync(0xFFFFFFFFu, pk_page, (g - pk_base) & 31);
+            is_tree[j] = g >= p_cache;
+            if (g >= pc_end || (CG == 2 && j != c)) row0[j] = -1;     // absent, or the peer's piece
+            else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
+            else if (p.paged) { if (pg < 0 || pg >= p.n_pages) pg = 0; row0[j] = pg * PG; }
+            else row0[j] = b * p.cap_tokens + g * PG;
+          }
+          if (lane == 0) {
+            int n_pieces = 0;
+#pragma unroll
+            for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
+            mbar_expect_tx(bar(B_KF + st), (uint32_t)n_pieces * 2u * kPiece);  // 0 bytes: a plain arrival
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
               const CUtensorMap* mk = is_tree[j] ? &tm_kt : &tm_kc;
-              tma_load_3d(sK + ks * kTile + j * kPiece, mk, 0, kvh, row0[j], bar_k_full(ks));
-              tma_load_3d(sK + ks * kTile + kHalf + j * kPiece, mk, 64, kvh, row0[j], bar_k_full(ks));
+              const uint32_t dst = sK + st * kStage + (CG == 2 ? 0u : (uint32_t)j * kPiece);
+              tma_load_3d(dst, mk, 0, kvh, row0[j], bar(B_KF + st));
+              tma_load_3d(dst + kKHalf, mk, 64, kvh, row0[j], bar(B_KF + st));
             }
-            issued_k = i + 1;
-            if (i >= VST) ok = mbar_wait(bar_v_empty(vs), ((i / VST) - 1) & 1, abort_flag, wlim);
           }
-          if (ok) {
-            s_tile_ok[vs] = tile_ok;  // read by the softmax threads after this V barrier completes
-            mbar_expect_tx(bar_v_full(vs), bytes);
+          ++kt;
+          issued_k = kt;
+          progress = true;
+        }
+      }
+      // ---- V of tile vt: CG = 1: both pieces, both halves of d;  CG = 2: both pieces, half c of d
+      if (vt < T) {
+        const int st = vt % VST;
+        int ready = 1;
+        if (vt >= VST && lane == 0)
+          ready = mbar_test(bar((kVOwnRing ? B_VE : B_PV) + st), ((vt / VST) - 1) & 1) ? 1 : 0;
+        ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
+        if (ready) {
+          const int g0 = pc_begin + vt * PPT;
+          if (p.paged && g0 < p_cache && g0 + PPT > pv_base + 32) {
+            pv_base = g0;
+            const int pc = g0 + lane;
+            pv_page = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
+          }
+          int row0[PPT];
+          bool is_tree[PPT];
+          int tile_ok = 1;
+#pragma unroll
+          for (int j = 0; j < PPT; ++j) {
+            const int g = g0 + j;
+            int pg = __shfl_sync(0xFFFFFFFFu, pv_page, (g - pv_base) & 31);
+            is_tree[j] = g >= p_cache;
+            if (g >= pc_end) row0[j] = -1;
+            else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
+            else if (p.paged) {
+              if (pg < 0 || pg >= p.n_pages) { tile_ok = 0; pg = 0; }  // flagged by the reporter; masked
+              row0[j] = pg * PG;
+            } else row0[j] = b * p.cap_tokens + g * PG;
+          }
+          if (lane == 0) {
+            int n_pieces = 0;
+#pragma unroll
+            for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
+            s_tile_ok[st] = tile_ok;  // read by the softmax threads after this V barrier completes
+            mbar_expect_tx(bar(B_VF + st), (uint32_t)n_pieces * (CG == 2 ? 1u : 2u) * kPiece);
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
               const CUtensorMap* mv = is_tree[j] ? &tm_vt : &tm_vc;
-              tma_load_3d(sV + vs * kTile + j * kPiece, mv, 0, kvh, row0[j], bar_v_full(vs));
-              tma_load_3d(sV + vs * kTile + kHalf + j * kPiece, mv, 64, kvh, row0[j], bar_v_full(vs));
+              const uint32_t dst = sV + st * kStage + (uint32_t)j * kPiece;
+              if (CG == 2) {
+                tma_load_3d(dst, mv, 64 * c, kvh, row0[j], bar(B_VF + st));
+              } else {
+                tma_load_3d(dst, mv, 0, kvh, row0[j], bar(B_VF + st));
+                tma_load_3d(dst + kStage / 2, mv, 64, kvh, row0[j], bar(B_VF + st));
+              }
             }
-            issued_v = i + 1;
           }
+          ++vt;
+          issued_v = vt;
+          progress = true;
         }
-        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+      }
+      if (progress) {
+        t_idle = clock64();
+      } else {
+        int stop = 0;
+        if (lane == 0) {
+          if (*abort_flag) stop = 1;
+          else if (clock64() - t_idle > wlim) { *abort_flag = 1; stop = 1; }
+        }
+        if (__shfl_sync(0xFFFFFFFFu, stop, 0)) ok = false;
       }
     }
   } else if (warp == 1) {
-    // =========================== MMA issuer ===================================================
-    if (lane == 0 && n_tiles > 0) {
-      bool ok = mbar_wait(bar_q, 0, abort_flag, wlim);
-      tc_fence_after();
-      auto local_tile = [&](int s, int r) { return (MT == 2) ? r : 2 * r + s; };
-      // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
-      // constant (the address field counts 16-byte units and never carries out of its 14 bits).
-      const uint64_t q_desc = smem_desc(sQ, 16, 1024);
-      const uint64_t k_desc = smem_desc(sK, 16, 1024);
-      const uint64_t v_desc = smem_desc(sV, kHalf, 1024);
-      auto issue_qk = [&](int s, int r) -> bool {
-        const int i = local_tile(s, r), st = i % KST;
-        // with two row tiles, slot 1 uses the K tile that slot 0 has just waited for
-        if (MT == 1 || s == 0) {
-          if (!mbar_wait(bar_k_full(st), (i / KST) & 1, abort_flag, wlim)) return false;
+    if (leader) {
+      // =========================== MMA issuer ===================================================
+      if (lane == 0 && T > 0) {
+        // a tile is ready when this block's copies have landed and, in a pair, the relay has
+        // reported the peer's
+        auto wait_both = [&](int own, int peer, uint32_t parity) -> bool {
+          if (!mbar_wait(bar(own), parity, abort_flag, wlim)) return false;
+          return CG == 1 || mbar_wait_cluster(bar(peer), parity, abort_flag, wlim);
+        };
+        bool ok = wait_both(B_Q, B_QP, 0);
+        tc_fence_after();
+        // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
+        // constant (the address field counts 16-byte units and never carries out of its 14 bits).
+        const uint64_t q_desc = smem_desc(sQ, 16, 1024);
+        const uint64_t k_desc = smem_desc(sK, 16, 1024);
+        const uint64_t v_desc = smem_desc(sV, kStage / 2, 1024);   // lbo: the other half of d (CG = 1)
+        auto issue_qk = [&](int t) -> bool {
+          const int st = t % KST;
+          if (!wait_both(B_KF + st, B_KP + st, (t / KST) & 1)) return false;
           tc_fence_after();
-        }
-        const uint64_t qd = q_desc + (uint64_t)((((MT == 2) ? s : 0) * kQTile) >> 4);
-        const uint64_t kd = k_desc + (uint64_t)((st * kTile) >> 4);
+          const uint64_t kd = k_desc + (uint64_t)((st * kStage) >> 4);
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ++ks) {
-          const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
-          const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
-          umma_bf16(tmem_S(s), qd + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
-        }
-        umma_commit(bar_s_full(s));
-        if (MT == 1 || s == 1) umma_commit(bar_k_empty(st));  // last reader of this K buffer
-        return true;
-      };
-      const int rounds[2] = {rounds0, rounds1};
-      for (int s = 0; s < 2 && ok; ++s)
-        if (rounds[s] > 0) ok = issue_qk(s, 0);
-      for (int r = 0; r < rounds0 && ok; ++r) {
-        for (int s = 0; s < 2 && ok; ++s) {
-          if (r >= rounds[s]) continue;
-          ok = mbar_wait(bar_p_full(s), r & 1, abort_flag, wlim);
+          for (int ks = 0; ks < HD / 16; ++ks) {
+            const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
+            const uint32_t ko = (ks >> 2) * kKHalf + (ks & 3) * 32;
+            mma_ss<CG>(tmem_S(t % NSB), q_desc + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
+          }
+          commit_all<CG>(bar(B_SF + t % NSB), pair_mask);   // scores ready; this K buffer is free
+          return true;
+        };
+        for (int t = 0; t < NSB && t < T && ok; ++t) ok = issue_qk(t);
+        for (int t = 0; t < T && ok; ++t) {
+          const int buf = t % NSB, st = t % VST;
+          ok = mbar_wait_cluster(bar(B_PF + buf), (t / NSB) & 1, abort_flag, wlim);
           if (!ok) break;
-          const int i = local_tile(s, r), st = i % VST;
-          if (MT == 1 || s == 0) {  // likewise the V tile
-            ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag, wlim);
-            if (!ok) break;
-          }
+          ok = wait_both(B_VF + st, B_VP + st, (t / VST) & 1);
+          if (!ok) break;
           tc_fence_after();
-          const uint64_t vd = v_desc + (uint64_t)((st * kTile) >> 4);
-#pragma unroll
-          for (int kk = 0; kk < BN / 16; ++kk) {
-            umma_bf16_ts(tmem_O(s), tmem_P(s) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
-                         (r > 0 || kk > 0) ? 1u : 0u);
+          const int n_kk = min(PPT, pc_end - (pc_begin + t * PPT)) * (PG / 16);   // a missing piece is skipped
+          const uint64_t vd = v_desc + (uint64_t)((st * kStage) >> 4);
+          for (int kk = 0; kk < n_kk; ++kk)
+            mma_ts<CG>(tmem_O, tmem_S(buf) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                       (t > 0 || kk > 0) ? 1u : 0u);
+          commit_all<CG>(bar(B_PV + buf), pair_mask);   // O holds tile t; P buffer (and with it the V buffer) free
+          if (kVOwnRing) commit_all<CG>(bar(B_VE + st), pair_mask);
+          if (t + NSB < T) ok = issue_qk(t + NSB);
+        }
+      }
+    } else {
+      // =========================== relay (odd block of a pair) ==================================
+      // forwards "my share of this tile has landed" to the barriers of the block that issues
+      if (lane == 0 && T > 0) {
+        bool ok = mbar_wait(bar(B_Q), 0, abort_flag, wlim);
+        if (ok) mbar_arrive_cluster(cluster_map(bar(B_QP), leader_rank));
+        int kt = 0, vt = 0;
+        long long t_idle = clock64();
+        while (ok && (kt < T || vt < T)) {
+          bool progress = false;
+          if (kt < T && mbar_test(bar(B_KF + kt % KST), (kt / KST) & 1)) {
+            mbar_arrive_cluster(cluster_map(bar(B_KP + kt % KST), leader_rank));
+            ++kt;
+            progress = true;
           }
-          umma_commit(bar_pv_done(s));
-          if (MT == 1 || s == 1) umma_commit(bar_v_empty(st));  // last reader of this V buffer
-          if (r + 1 < rounds[s]) ok = issue_qk(s, r + 1);
+          if (vt < T && mbar_test(bar(B_VF + vt % VST), (vt / VST) & 1)) {
+            mbar_arrive_cluster(cluster_map(bar(B_VP + vt % VST), leader_rank));
+            ++vt;
+            progress = true;
+          }
+          if (progress) t_idle = clock64();
+          else if (*abort_flag) ok = false;
+          else if (clock64() - t_idle > wlim) { *abort_flag = 1; ok = false; }
         }
       }
     }
   } else {
-    // =========================== softmax groups ===============================================
-    constexpr int NH = BN / 64;   // the row of S is taken in 64-column halves (register budget)
-    const int rounds = my_rounds;
-    bool ok = true;
-    if (warp == 2 && n_tiles > 0) {  // the Q tile(s): issued here so that the producer starts with K/V
-      if (lane == 0) {
-        mbar_expect_tx(bar_q, (uint32_t)(MT * RT * HD * 2));   // the boxes hold RT rows of a tile
-        const int nodes_per_tile = BM / G;
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-          const int node0 = b * N + (row_cta * MT + m) * nodes_per_tile;
-          tma_load_3d(sQ + m * kQTile, &tm_q, 0, kvh * G, node0, bar_q);
-          tma_load_3d(sQ + m * kQTile + kQTile / 2, &tm_q, 64, kvh * G, node0, bar_q);
-        }
+    // =========================== softmax threads ==============================================
+    if (warp == 2 && T > 0 && lane == 0) {  // the Q tile: issued here so that the producer starts with K/V
+      if (has_rows) {
+        mbar_expect_tx(bar(B_Q), (uint32_t)(RT * HD * 2));   // the boxes hold RT rows
+        const int node0 = b * N + tile_idx * (BM / G);
+        tma_load_3d(sQ, &tm_q, 0, kvh * G, node0, bar(B_Q));
+        tma_load_3d(sQ + kQTile / 2, &tm_q, 64, kvh * G, node0, bar(B_Q));
+      } else {
+        mbar_arrive(bar(B_Q));   // a block without rows (odd number of row tiles) loads no Q
       }
     }
-    // ancestor bitsets (row i of the tree's topology matrix), built by the softmax warps while
-    // the first tiles are on their way; the 256 threads meet at a named barrier of their own
-    for (int i = tid - 64; i < N; i += 2 * BM) {
+    // ancestor bitsets (row i of the tree's topology matrix), built while the first tiles are on
+    // their way; the 256 threads meet at a named barrier of their own
+    for (int i = tid - 64; i < N; i += kSoftmaxThreads) {
       uint32_t w[4] = {0, 0, 0, 0};
       int j = i;
       for (int hop = 0; hop < N && j >= 0; ++hop) {
@@ -487,170 +585,175 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       pbad = __any_sync(0xFFFFFFFFu, pbad);
       if (lane == 0 && pbad) atomicOr(p.tickets + 2 * b + 1, 1u);  // before this block's ticket
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
+    named_barrier(1, kSoftmaxThreads);
+    const uint32_t pf_leader0 = cluster_map(bar(B_PF), leader_rank);
 
-    for (int r = 0; r < rounds && ok; ++r) {
-      const int i = (MT == 2) ? r : 2 * r + slot;
-      const int st = i % VST;   // these threads only touch the V ring
-      // allowed columns of this row in this tile (64 per piece), and how many rows of each V
-      // piece are real keys
-      uint32_t allow[BN / 32];
+    // A wait that runs out raises the block's abort flag and sets `fail`; the thread then skips
+    // the work but keeps walking through the named barriers it shares with its partner warp, and
+    // both leave the loop together at the next exchange (a warp must never be left alone at a
+    // named barrier, which has no time limit).
+    bool fail = false;
+    for (int t = 0; t < T; ++t) {
+      const int buf = t % NSB, vst = t % VST;
+      const int g0 = pc_begin + t * PPT;
+      // real keys in each piece of the tile, and the allowed columns of this thread's piece
       int valid[PPT];
       bool cache_tile = false, short_tile = false;
 #pragma unroll
       for (int j = 0; j < PPT; ++j) {
-        const int g = pc_begin + i * PPT + j;
-        if (g >= pc_end) {                 // the range ended inside this tile
-          valid[j] = 0;
-          allow[2 * j] = allow[2 * j + 1] = 0;
-        } else if (g < p_cache) {          // context piece: everything up to the context length
-          cache_tile = true;
-          valid[j] = min(PG, L - g * PG);
-          const uint64_t bits = valid[j] >= 64 ? ~0ull : ((1ull << valid[j]) - 1ull);
-          allow[2 * j] = (uint32_t)bits; allow[2 * j + 1] = (uint32_t)(bits >> 32);
-        } else {                           // tree piece: the node's ancestors (itself included)
-          const int tp = g - p_cache;
-          valid[j] = min(PG, N - tp * PG);
-          allow[2 * j] = s_anc[node][2 * tp]; allow[2 * j + 1] = s_anc[node][2 * tp + 1];
-        }
-        short_tile |= valid[j] < PG;
+        const int g = g0 + j;
+        if (g >= pc_end) valid[j] = -1;                       // no such piece: P V skips it
+        else if (g < p_cache) { valid[j] = min(PG, L - g * PG); cache_tile = true; }
+        else valid[j] = min(PG, N - (g - p_cache) * PG);
+        short_tile |= (valid[j] >= 0 && valid[j] < PG);
       }
-      ok = mbar_wait(bar_s_full(slot), r & 1, abort_flag, wlim);
-      ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) break;
+      const int g = g0 + ch;
+      const bool present = g < pc_end;
+      uint32_t allow0 = 0, allow1 = 0;
+      if (present && row_valid) {
+        if (g < p_cache) {
+          const uint64_t bits = valid[ch] >= 64 ? ~0ull : ((1ull << valid[ch]) - 1ull);
+          allow0 = (uint32_t)bits; allow1 = (uint32_t)(bits >> 32);
+        } else {
+          const int tp = g - p_cache;
+          allow0 = s_anc[node][2 * tp]; allow1 = s_anc[node][2 * tp + 1];
+        }
+      }
+      auto wait_all = [&](uint32_t barrier, uint32_t parity) {   // warp-uniform verdict
+        if (fail) return;
+        const bool w_ok = mbar_wait(barrier, parity, abort_flag, wlim);
+        fail = !__all_sync(0xFFFFFFFFu, w_ok);
+      };
+      wait_all(bar(B_SF + buf), (t / NSB) & 1);
       tc_fence_after();
       if (p.paged && cache_tile) {
-        // the producer's verdict on this tile's pages, written before it armed the V barrier (the
-        // V stage is not reused before this tile's P V, so the flag is stable)
-        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag, wlim);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        if (!*(volatile int*)&s_tile_ok[st]) {  // sequence is flagged; hide the whole tile
+        // the producer's verdict on this tile's pages, written before it armed the V barrier
+        wait_all(bar(B_VF + vst), (t / VST) & 1);
+        if (!fail && !*(volatile int*)&s_tile_ok[vst]) {  // sequence is flagged; hide the whole tile
           short_tile = true;
 #pragma unroll
-          for (int j = 0; j < PPT; ++j) valid[j] = 0;
-#pragma unroll
-          for (int w = 0; w < BN / 32; ++w) allow[w] = 0;
+          for (int j = 0; j < PPT; ++j) if (valid[j] > 0) valid[j] = 0;
+          allow0 = allow1 = 0;
         }
       }
-
-      bool full = row_valid;
-#pragma unroll
-      for (int w = 0; w < BN / 32; ++w) {
-        if (!row_valid) allow[w] = 0;
-        full = full && (allow[w] == 0xFFFFFFFFu);
-      }
-      const bool all_full = __all_sync(0xFFFFFFFFu, full);
+      const bool all_full = __all_sync(0xFFFFFFFFu, (allow0 & allow1) == 0xFFFFFFFFu);
 
       uint32_t sv[64];
-      // loads half h of the row and replaces the scores of columns that are not allowed by -inf
-      auto load_half = [&](int h) {
-        tmem_ld_x64(tmem_S(slot) + lane_addr + h * 64, sv);
+      // this thread's 64 scores; columns that are not allowed become -inf
+      auto load_scores = [&]() {
+        tmem_ld_x64(tmem_S(buf) + lane_addr + ch * 64, sv);
         tmem_wait_ld();
         if (!all_full) {
 #pragma unroll
           for (int j = 0; j < 64; ++j) {
-            const uint32_t wbits = allow[2 * h + (j >> 5)];
+            const uint32_t wbits = (j < 32) ? allow0 : allow1;
             if (!((wbits >> (j & 31)) & 1u)) sv[j] = 0xFF800000u;  // -inf
           }
         }
       };
       // One pass with the reference maximum as it stands: exponentiate, pack P (kept in registers)
-      // and add up the row.  No per-element maximum is tracked (the softmax threads are bound by
-      // instruction issue): a row sum of at most 2^8 proves that no probability exceeded 2^8,
-      // i.e. that the reference is still good.  Otherwise (rare after the first tile; inf or NaN
-      // from an overflow also lands here) the true maximum is taken from the scores - still
-      // intact, because P is stored last - the reference replaced, O rescaled and the tile redone.
-      uint32_t pk[NH * 32];
-      auto row_max = [&]() {
-        float m0 = -INFINITY;
-#pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          load_half(h);
-#pragma unroll
-          for (int j = 0; j < 64; ++j) m0 = fmaxf(m0, __uint_as_float(sv[j]));
-        }
-        return m0 * p.scale_log2;  // scale > 0; -inf (no allowed key) stays -inf
-      };
-      if (r == 0) m_ref = row_max();  // no reference yet: a cheap extra pass instead of a redo
+      // and add up.  No per-element maximum is tracked: a sum of at most 2^8 proves that no
+      // probability exceeded 2^8, i.e. that the reference is still good.  Otherwise (rare after
+      // the first tile; inf or NaN from an overflow also lands here) the true maximum of the row is
+      // taken from the scores - still intact, because P is stored last - the reference replaced,
+      // O rescaled and the tile redone.  The two threads of a row decide together.
+      uint32_t pk[32];
       float sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       auto exp_pass = [&]() {
         sum = 0.f;
+        if (!present || fail) return;
+        load_scores();
 #pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          load_half(h);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-            sum += p0 + p1;
-            pk[h * 32 + j] = pack_bf16(p0, p1);
-          }
+        for (int j = 0; j < 32; ++j) {
+          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
+          sum += p0 + p1;
+          pk[j] = pack_bf16(p0, p1);
         }
       };
-      exp_pass();
-      const bool suspect = !(sum <= kRowSumLimit);  // also catches inf and NaN
-      if (__any_sync(0xFFFFFFFFu, suspect)) {
-        const float mx = suspect ? row_max() : m_ref;
+      if (t > 0) {
+        exp_pass();
+        // a row without a reference yet must take one as soon as it sees a score
+        const bool suspect = !(sum <= kRowSumLimit) || (m_ref == -INFINITY && sum != 0.f);
+        if (__any_sync(0xFFFFFFFFu, suspect) && lane == 0) *(volatile int*)&s_redo[sw] = t;
+      }
+      if (fail && lane == 0) *(volatile int*)&s_fail[sw] = 1;
+      named_barrier(pair_bar, 64);
+      if (*(volatile int*)&s_fail[sw] | *(volatile int*)&s_fail[sw ^ 4]) break;   // both warps see the same
+      const bool redo = (t == 0) ||   // no reference yet
+                        (*(volatile int*)&s_redo[sw] == t) || (*(volatile int*)&s_redo[sw ^ 4] == t);
+      if (redo) {
+        float mx = -INFINITY;
+        if (present) {
+          load_scores();
+#pragma unroll
+          for (int j = 0; j < 64; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
+          mx *= p.scale_log2;   // scale > 0; -inf (no allowed key) stays -inf
+        }
+        s_xch[ch][row] = mx;
+        named_barrier(pair_bar, 64);
+        mx = fmaxf(mx, s_xch[ch ^ 1][row]);
         const bool need = mx > m_ref;
-        if (r > 0) {  // O must be at rest: the previous P V has completed
-          ok = mbar_wait(bar_pv_done(slot), (r - 1) & 1, abort_flag, wlim);
-          ok = __all_sync(0xFFFFFFFFu, ok);
-          if (!ok) break;
+        if (t > 0) {  // O must be at rest: P V of the previous tile has completed
+          wait_all(bar(B_PV + (t - 1) % NSB), ((t - 1) / NSB) & 1);
           tc_fence_after();
         }
         const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
         if (need) { m_ref = mx; l_run *= alpha; }
-        if (r > 0) {
+        if (t > 0 && !fail) {
 #pragma unroll 1
-          for (int c = 0; c < HD; c += 32) {
+          for (int cc = 0; cc < 64; cc += 32) {
             uint32_t ov[32];
-            tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+            tmem_ld_x32(tmem_O + lane_addr + ch * 64 + cc, ov);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-            tmem_st_x32(tmem_O(slot) + lane_addr + c, ov);
+            tmem_st_x32(tmem_O + lane_addr + ch * 64 + cc, ov);
           }
           tmem_wait_st();
         }
         neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
         exp_pass();
+        named_barrier(pair_bar, 64);   // the partner has read its scores: P may overwrite them
       }
-      // P (the A operand of P V) takes the place of score columns that have been consumed.  The
-      // previous P V read these columns before this tile's Q K^T, issued after it, wrote them.
-#pragma unroll
-      for (int h = 0; h < NH; ++h)
-        tmem_st_x32(tmem_P(slot) + lane_addr + h * 32, *reinterpret_cast<const uint32_t(*)[32]>(&pk[h * 32]));
-      tmem_wait_st();
+      // P (the A operand of P V) takes the place of score columns that have been consumed: keys
+      // 64 ch .. 64 ch + 63 of the tile are columns 32 ch .. 32 ch + 31 (two bf16 per column).
+      if (present && !fail) {
+        tmem_st_x32(tmem_S(buf) + lane_addr + ch * 32, pk);
+        tmem_wait_st();
+      }
       l_run += sum;
 
       if (short_tile) {
-        // Rows of a V piece beyond its real keys hold whatever lies behind them in memory (or were
-        // never loaded); their probabilities are exactly 0, but 0 * NaN would poison O: clear them.
-        ok = mbar_wait(bar_v_full(st), (i / VST) & 1, abort_flag, wlim);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        uint8_t* vt = sV_gen + st * kTile;
-        const int me = (warp - 2 - slot * 4) * 32 + lane;   // 0 .. 127 within the softmax group
+        // Rows of a V piece beyond its real keys hold whatever lies behind them in memory; their
+        // probabilities are exactly 0, but 0 * NaN would poison O: clear them.
+        wait_all(bar(B_VF + vst), (t / VST) & 1);
+        if (!fail) {
+          uint8_t* vt = sV_gen + vst * kStage;
+          const int me = tid - 64;   // 0 .. 255 among the softmax threads
+          constexpr int kHalves = (CG == 2) ? 1 : 2;   // halves of the head dimension held here
 #pragma unroll
-        for (int j = 0; j < PPT; ++j) {
-          const int per_half = (PG - valid[j]) * 8;  // 16-byte chunks per half of the head dimension
-          for (int c = me; c < 2 * per_half; c += BM) {
-            const int half = c / per_half, rem = c - half * per_half;
-            const int vr = j * PG + valid[j] + (rem >> 3), ch = rem & 7;
-            *reinterpret_cast<uint4*>(vt + half * kHalf + vr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+          for (int j = 0; j < PPT; ++j) {
+            if (valid[j] < 0) continue;
+            const int per_half = (PG - valid[j]) * 8;  // 16-byte chunks per half of the head dimension
+            for (int cidx = me; cidx < kHalves * per_half; cidx += kSoftmaxThreads) {
+              const int half = cidx / per_half, rem = cidx - half * per_half;
+              const int vr = j * PG + valid[j] + (rem >> 3), chk = rem & 7;
+              *reinterpret_cast<uint4*>(vt + half * (kStage / 2) + vr * 128 + chk * 16) = make_uint4(0, 0, 0, 0);
+            }
           }
+          fence_async_smem();   // cleared V rows visible to the tensor core's reads
         }
-        fence_async_smem();   // cleared V rows visible to the tensor core's reads
       }
       tc_fence_before();
-      mbar_arrive(bar_p_full(slot));
+      __syncwarp();
+      if (lane == 0 && !fail) mbar_arrive_cluster(pf_leader0 + 8u * (uint32_t)buf);
     }
 
-    if (ok && rounds > 0) {  // the last P V of this slot has landed in O
-      ok = mbar_wait(bar_pv_done(slot), (rounds - 1) & 1, abort_flag, wlim);
-      ok = __all_sync(0xFFFFFFFFu, ok);
+    if (!fail && !*abort_flag && T > 0) {  // the last P V has landed in O
+      const bool w_ok = mbar_wait(bar(B_PV + (T - 1) % NSB), ((T - 1) / NSB) & 1, abort_flag, wlim);
+      (void)__all_sync(0xFFFFFFFFu, w_ok);
     }
   }
 
@@ -659,13 +762,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (*abort_flag) {
     if (warp == 0 && lane == 0) {
       // TMA copies that were issued land on their own; wait for the newest phase of each stage
-      for (int i = max(0, issued_k - KST); i < issued_k; ++i) mbar_drain(bar_k_full(i % KST), (i / KST) & 1);
-      for (int i = max(0, issued_v - VST); i < issued_v; ++i) mbar_drain(bar_v_full(i % VST), (i / VST) & 1);
-      if (n_tiles > 0) mbar_drain(bar_q, 0);
+      for (int i = max(0, issued_k - KST); i < issued_k; ++i) mbar_drain(bar(B_KF + i % KST), (i / KST) & 1);
+      for (int i = max(0, issued_v - VST); i < issued_v; ++i) mbar_drain(bar(B_VF + i % VST), (i / VST) & 1);
     }
-    if (warp == 1 && lane == 0) {
-      umma_commit(bar_drain);  // completes when every MMA issued so far has finished
-      mbar_drain(bar_drain, 0);
+    if (warp == 2 && lane == 0 && T > 0 && has_rows) mbar_drain(bar(B_Q), 0);
+    if (warp == 1 && lane == 0 && leader) {
+      if (CG == 2) umma_commit_pair(bar(B_DR)); else umma_commit(bar(B_DR));
+      mbar_drain(bar(B_DR), 0);  // completes when every MMA issued so far has finished
     }
   }
   tc_fence_before();
@@ -676,25 +779,42 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // behind the epilogue (no wait can run out after this point)
   unsigned my_ticket = 0;
   if (tid == 0) my_ticket = report(aborted ? 2u : 0u);
-  const int n_src = p.splits * (MT == 1 ? 2 : 1);  // accumulators that cover one output row
+  const int n_src = p.splits;   // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
-  // staging area for the merge: O of both slots as fp16 [slot][128 rows][128], every row scaled by
-  // a power of two that puts its largest magnitude in [2^13, 2^14) (half the bytes of fp32 through
-  // distributed shared memory, at a relative rounding error of 2^-11, far below that of the bf16
-  // output; the scale travels with the row's maximum and sum).  The 16-byte chunk c of row r is
-  // stored at chunk (c ^ (r & 15)) so that row-per-thread writes and row-per-warp reads are both
-  // conflict free.  The area reuses the tile memory, which nothing reads any more.
+  // staging area for the merge: O as fp16 [128 rows][128], every row scaled by a power of two that
+  // puts its largest magnitude in [2^13, 2^14) (half the bytes of fp32 through distributed shared
+  // memory, at a relative rounding error of 2^-11, far below that of the bf16 output; the scale
+  // travels with the row's maximum and sum).  The 16-byte chunk c of row r is stored at chunk
+  // (c ^ (r & 15)) so that row-per-thread writes and row-per-warp reads are both conflict free.
+  // The area reuses the tile memory, which nothing reads any more.
   uint8_t* const sO = smem_raw + (sQ - smem_u32(smem_raw));
 
   if (!aborted && warp >= 2) {
-    if (n_src == 1) {
-      // only accumulator of these rows: normalise and store
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD;
+    // the row's two threads add up their sums (and, for staging, agree on the row's scale)
+    float amax = 0.f;
+    if (n_src > 1 && T > 0) {
 #pragma unroll 1
-      for (int c = 0; c < HD; c += 32) {
+      for (int cc = 0; cc < 64; cc += 32) {
         uint32_t ov[32];
-        tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+        tmem_ld_x32(tmem_O + lane_addr + ch * 64 + cc, ov);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(__uint_as_float(ov[j])));
+      }
+    }
+    s_xch[ch][row] = l_run;
+    s_xch2[ch][row] = amax;
+    named_barrier(1, kSoftmaxThreads);
+    const float l_tot = l_run + s_xch[ch ^ 1][row];
+    amax = fmaxf(amax, s_xch2[ch ^ 1][row]);
+    if (n_src == 1) {
+      // only accumulator of these rows: normalise and store this thread's 64 columns
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      uint16_t* dst = p.out + (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD + ch * 64;
+#pragma unroll 1
+      for (int cc = 0; cc < 64; cc += 32) {
+        uint32_t ov[32];
+        tmem_ld_x32(tmem_O + lane_addr + ch * 64 + cc, ov);
         tmem_wait_ld();
         if (row_valid) {
 #pragma unroll
@@ -704,26 +824,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             v.y = pack_bf16(__uint_as_float(ov[q4 * 8 + 2]) * inv, __uint_as_float(ov[q4 * 8 + 3]) * inv);
             v.z = pack_bf16(__uint_as_float(ov[q4 * 8 + 4]) * inv, __uint_as_float(ov[q4 * 8 + 5]) * inv);
             v.w = pack_bf16(__uint_as_float(ov[q4 * 8 + 6]) * inv, __uint_as_float(ov[q4 * 8 + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + c + q4 * 8) = v;
+            *reinterpret_cast<uint4*>(dst + cc + q4 * 8) = v;
           }
         }
       }
-      if (p.lse != nullptr && row_valid)
-        p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_run)) * kLn2;
+      if (p.lse != nullptr && row_valid && ch == 0)
+        p.lse[((int64_t)b * N + node) * p.Hq + kvh * G + gq] = (m_ref + log2f(l_tot)) * kLn2;
     } else {
-      uint8_t* orow = sO + ((size_t)slot * BM + row) * (HD * 2);
-      // first pass: the row's largest magnitude, which fixes its scale
-      float amax = 0.f;
-      if (my_rounds > 0) {
-#pragma unroll 1
-        for (int c = 0; c < HD; c += 32) {
-          uint32_t ov[32];
-          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(__uint_as_float(ov[j])));
-        }
-      }
+      uint8_t* orow = sO + (size_t)row * (HD * 2);
       // scale 2^lc with amax * 2^lc in [2^13, 2^14); lc is clamped so that the scale and its
       // inverse are normal numbers (a zero row keeps zeros, inf or NaN stay what they are)
       const int biased = (int)((__float_as_uint(amax) >> 23) & 255u);
@@ -731,12 +839,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const float cscale = __uint_as_float((uint32_t)(127 + lc) << 23);
       const float cinv = __uint_as_float((uint32_t)(127 - lc) << 23);
 #pragma unroll 1
-      for (int c = 0; c < HD; c += 32) {
+      for (int cc = 0; cc < 64; cc += 32) {
         uint32_t ov[32];
-        if (my_rounds > 0) {
-          tmem_ld_x32(tmem_O(slot) + lane_addr + c, ov);
+        if (T > 0) {
+          tmem_ld_x32(tmem_O + lane_addr + ch * 64 + cc, ov);
           tmem_wait_ld();
-        } else {  // a slot without tiles contributes zeros with weight zero
+        } else {  // a block without tiles contributes zeros with weight zero
 #pragma unroll
           for (int j = 0; j < 32; ++j) ov[j] = 0u;
         }
@@ -749,37 +857,34 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                                 __uint_as_float(ov[q4 * 8 + 2 * e + 1]) * cscale);
             h[e] = *reinterpret_cast<const uint32_t*>(&v);
           }
-          const int chunk = (c >> 3) + q4;
+          const int chunk = ((ch * 64 + cc) >> 3) + q4;
           *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 15)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
         }
       }
-      s_ml[slot][row] = make_float4(my_rounds > 0 ? m_ref : -INFINITY, my_rounds > 0 ? l_run : 0.f, cinv, 0.f);
+      if (ch == 0) s_ml[row] = make_float4(T > 0 ? m_ref : -INFINITY, T > 0 ? l_tot : 0.f, cinv, 0.f);
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-  if (n_src == 1) {  // such a block is its own cluster
+  if (CS == 1) {  // a block that is its own cluster
+    if (warp == 1) release_tmem();
     if (tid == 0) publish(my_ticket);
     return;
   }
 
-  // ---- merge across the cluster (the split-KV blocks of one row tile) through distributed
-  //      shared memory: rank j finalises rows [j, j+1) * rows/splits of the tile(s) ------------
   cg::cluster_group cluster = cg::this_cluster();
-  cluster.sync();  // every block's staging area is complete (also reached by an aborted block)
-  if (!aborted) {
-    // Every rank finalises per_rank rows; per_rank * n_src is 256 whatever the split count.
-    const int per_rank = MT * BM / p.splits;
+  cluster.sync();  // every block's staging area is complete and its MMAs are done (also reached by an aborted block)
+  if (n_src > 1 && !aborted) {
+    // ---- merge across the key splits through distributed shared memory: split j finalises rows
+    //      [j, j+1) * 128 / splits of the tile; source q of a row lives in cluster rank q CG + c ----
+    const int per_rank = BM / p.splits;
     const int first_row = split * per_rank;
-    // (a) thread (k, q) fetches the (maximum, sum) pair of source q of row k; the n_src lanes of a
-    //     row sit side by side in one warp, so the normalised weights come from shuffles.
-    //     Source q is (block q, slot `tile`) when MT == 2 and (block q / 2, slot q % 2) when MT == 1.
-    if (tid < 2 * BM) {
+    // (a) thread (k, q) fetches the (maximum, sum, scale) of source q of row k; the n_src lanes of
+    //     a row sit side by side in one warp, so the normalised weights come from shuffles.
+    if (tid < BM) {
       const int k = tid / n_src, q = tid - k * n_src;
-      const int rr = first_row + k, tile = rr / BM, trow = rr % BM;
-      const int qc = (MT == 2) ? q : q >> 1, qs = (MT == 2) ? tile : q & 1;
-      const float4 ml = dsmem_ld16(dsmem_addr(smem_u32(&s_ml[qs][trow]), qc));
+      const int trow = first_row + k;
+      const float4 ml = dsmem_ld16(cluster_map(smem_u32(&s_ml[trow]), (uint32_t)(q * CG + c)));
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
@@ -787,26 +892,27 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       float lsum = wgt * ml.y;
       for (int o = 1; o < n_src; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
       s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
-      const int rg = (row_cta * MT + tile) * RT + trow;
-      if (q == 0 && p.lse != nullptr && trow < RT && rg < rows_total) {
+      const int rg = tile_idx * RT + trow;
+      if (q == 0 && p.lse != nullptr && has_rows && trow < RT && rg < rows_total) {
         const int onode = rg / G, ogq = rg - onode * G;
         p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
       }
     }
     __syncthreads();
     // (b) weighted sums, rows spread over the warps
-    const uint32_t sO_addr = smem_u32(sO);
-    const int rot = (split + 1) * (MT == 1 ? 2 : 1);  // first source read: the next block's
-    uint16_t* outp = p.out;
-    const int64_t seq_row0 = (int64_t)b * N;
-    switch (n_src) {
-      case 2: merge_rows<2, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 4: merge_rows<4, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      case 8: merge_rows<8, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
-      default: merge_rows<16, MT>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, row_cta * MT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, outp); break;
+    if (has_rows) {
+      const uint32_t sO_addr = smem_u32(sO);
+      const int rot = split + 1;  // first source read: the next split's
+      const int64_t seq_row0 = (int64_t)b * N;
+      switch (n_src) {
+        case 2: merge_rows<2>(sO_addr, s_w, first_row, per_rank, rot, CG, c, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+        case 4: merge_rows<4>(sO_addr, s_w, first_row, per_rank, rot, CG, c, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+        default: merge_rows<8>(sO_addr, s_w, first_row, per_rank, rot, CG, c, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+      }
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
+  if (warp == 1) release_tmem();
   if (tid == 0) publish(my_ticket);
 }
 
@@ -825,6 +931,11 @@ bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t heads, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int row_tiles(const clv_shape& s) {
+  const int G = s.n_q_heads / s.n_kv_heads;
+  return (s.n_nodes + BM / G - 1) / (BM / G);   // row tiles of BM / G whole nodes
+}
+
 }  // namespace
 
 bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
@@ -837,19 +948,16 @@ bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
 
 AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
   AttnPlan pl;
-  const int G = s.n_q_heads / s.n_kv_heads;
-  const int tiles = (s.n_nodes + BM / G - 1) / (BM / G);   // row tiles of BM / G whole nodes
-  const int mt = tiles > 1 ? 2 : 1;
-  const int row_ctas = (tiles + mt - 1) / mt;
-  pl.m_tiles = row_ctas;
-  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * row_ctas;
-  const int BN = mt == 2 ? Cfg<2>::BN : Cfg<1>::BN;
+  const int tiles = row_tiles(s);
+  const int cgrp = tiles > 1 ? 2 : 1;                  // units of several row tiles are worked by pairs
+  pl.m_tiles = (tiles + cgrp - 1) / cgrp;
+  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * pl.m_tiles * cgrp;
   const int key_tiles = (max_ctx_len > 0 ? (max_ctx_len + BN - 1) / BN : 0) + (s.n_nodes + BN - 1) / BN;
-  // The key axis is split over a thread-block cluster (merged through distributed shared memory),
-  // so the split count is a power of two up to the portable cluster size; one block per SM.
-  const int per_cta_min = mt == 1 ? 2 : 1;  // MT == 1 blocks eat two tiles per round
+  // The key axis is split over a thread-block cluster (merged through distributed shared memory):
+  // a power of two that keeps the cluster within the portable size of 8 and the grid within one
+  // block per SM, and leaves every block at least two key tiles.
   int splits = 1;
-  while (splits < 8 && ctas * (splits * 2) <= sm_count() && key_tiles / (splits * 2) >= per_cta_min)
+  while (cgrp * splits * 2 <= 8 && ctas * (splits * 2) <= sm_count() && key_tiles / (splits * 2) >= 2)
     splits *= 2;
   pl.splits = splits;
   pl.tickets = 0;
@@ -864,7 +972,8 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 cudaStream_t stream) {
   (void)scratch;
   const int G = s.n_q_heads / s.n_kv_heads;
-  const int mt = (s.n_nodes + BM / G - 1) / (BM / G) > 1 ? 2 : 1;   // as in tc_attn_plan
+  const int tiles = row_tiles(s);
+  const int cgrp = tiles > 1 ? 2 : 1;   // as in tc_attn_plan
   static OncePerDevice once;
   cudaError_t e0 = run_once_per_device(once, [] {
     cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -891,32 +1000,34 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.status = status;
-  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
+  const int cs = cgrp * plan.splits;
+  const int64_t clusters = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
   p.B = s.batch; p.N = s.n_nodes; p.Hq = s.n_q_heads; p.Hkv = s.n_kv_heads; p.G = G;
   p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
-  p.row_ctas = plan.m_tiles;
+  p.row_groups = plan.m_tiles;
+  p.tiles = tiles;
   p.splits = plan.splits;
-  p.longest_first = (ctas > sm_count() && s.batch > 1 && s.batch <= 256) ? 1 : 0;
+  p.longest_first = (clusters * cs > sm_count() && s.batch > 1 && s.batch <= 256) ? 1 : 0;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.wait_limit = wait_limit_cycles();
   p.tickets = tickets;
-  p.blocks_per_seq = s.n_kv_heads * plan.m_tiles * plan.splits;
+  p.blocks_per_seq = s.n_kv_heads * plan.m_tiles * cs;
 
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)ctas, (unsigned)plan.splits, 1);
+  cfg.gridDim = dim3((unsigned)(clusters * cs), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = mt == 1 ? Cfg<1>::kSmem : Cfg<2>::kSmem;
+  cfg.dynamicSmemBytes = cgrp == 1 ? Cfg<1>::kSmem : Cfg<2>::kSmem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;  // the blocks that split one row tile's keys
-  attr[0].val.clusterDim.x = 1;
-  attr[0].val.clusterDim.y = (unsigned)plan.splits;
+  attr[0].id = cudaLaunchAttributeClusterDimension;  // the blocks that share one row group's keys
+  attr[0].val.clusterDim.x = (unsigned)cs;
+  attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up overlaps the previous kernel's tail
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if (mt == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  if (cgrp == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
   return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<2>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
 }
 
