@@ -197,7 +197,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 B_VE = B_PV + NSB, B_Q = B_VE + VST, B_DR = B_Q + 1, B_KP = B_DR + 1, B_VP = B_KP + KST,
                 B_QP = B_VP + VST, NBAR = B_QP + 1;
   __shared__ __align__(8) unsigned long long s_bar[NBAR];
-  __shared__ int s_tile_ok[VST];  // paged cache: every page of the tile in this V stage is valid
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ int s_redo[8];        // per softmax warp: the last tile in which one of its row sums was suspect
@@ -339,7 +338,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   volatile int* abort_flag = &s_abort;
   const long long wlim = p.wait_limit;
-  auto tmem_S = [&](int buf) { return tmem + (uint32_t)(buf * BN); };   // P overwrites its first 64 columns
+  auto tmem_S = [&](int buf) { return tmem + (uint32_t)(buf * BN); };   // P overwrites columns 0-31 and 64-95
   const uint32_t tmem_O = tmem + (uint32_t)(NSB * BN);
 
   int issued_k = 0, issued_v = 0;  // producer bookkeeping for the drain
@@ -428,7 +427,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
           int row0[PPT];
           bool is_tree[PPT];
-          int tile_ok = 1;
 #pragma unroll
           for (int j = 0; j < PPT; ++j) {
             const int g = g0 + j;
@@ -437,7 +435,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (g >= pc_end) row0[j] = -1;
             else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
             else if (p.paged) {
-              if (pg < 0 || pg >= p.n_pages) { tile_ok = 0; pg = 0; }  // flagged by the reporter; masked
+              if (pg < 0 || pg >= p.n_pages) pg = 0;   // the reporter flags the sequence; any page will do
               row0[j] = pg * PG;
             } else row0[j] = b * p.cap_tokens + g * PG;
           }
@@ -445,7 +443,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int n_pieces = 0;
 #pragma unroll
             for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
-            s_tile_ok[st] = tile_ok;  // read by the softmax threads after this V barrier completes
             mbar_expect_tx(bar(B_VF + st), (uint32_t)n_pieces * (CG == 2 ? 1u : 2u) * kPiece);
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
@@ -517,9 +514,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tc_fence_after();
           const int n_kk = min(PPT, pc_end - (pc_begin + t * PPT)) * (PG / 16);   // a missing piece is skipped
           const uint64_t vd = v_desc + (uint64_t)((st * kStage) >> 4);
+          // P of piece j of the tile sits in the first 32 columns of that piece's 64 score columns
           for (int kk = 0; kk < n_kk; ++kk)
-            mma_ts<CG>(tmem_O, tmem_S(buf) + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), kIdescPV,
-                       (t > 0 || kk > 0) ? 1u : 0u);
+            mma_ts<CG>(tmem_O, tmem_S(buf) + (kk >> 2) * 64 + (kk & 3) * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                       kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
           commit_all<CG>(bar(B_PV + buf), pair_mask);   // O holds tile t; P buffer (and with it the V buffer) free
           if (kVOwnRing) commit_all<CG>(bar(B_VE + st), pair_mask);
           if (t + NSB < T) ok = issue_qk(t + NSB);
@@ -593,83 +591,91 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // both leave the loop together at the next exchange (a warp must never be left alone at a
     // named barrier, which has no time limit).
     bool fail = false;
+    auto wait_all = [&](uint32_t barrier, uint32_t parity) {   // warp-uniform verdict
+      if (fail) return;
+      const bool w_ok = mbar_wait(barrier, parity, abort_flag, wlim);
+      fail = !__all_sync(0xFFFFFFFFu, w_ok);
+    };
+    const bool warp_rows_valid = __all_sync(0xFFFFFFFFu, row_valid);
+    // tiles [0, t_plain) of this block consist of two complete pieces of context: nothing to mask
+    const int t_plain = max(0, (min(pc_end, L / PG) - pc_begin) / PPT);
+    // The scores of a tile (this thread's 64) are fetched into registers while the previous tile's
+    // P is on its way to tensor memory; they stay there until the tile is done, so a tile can be
+    // redone against a new reference without another read.
+    uint32_t sv[64];
+    auto fetch_scores = [&](int t, int sbuf) {
+      if (pc_begin + t * PPT + ch < pc_end && !fail) tmem_ld_x64(tmem_S(sbuf) + lane_addr + ch * 64, sv);
+    };
+    int buf = 0;
+    uint32_t ph = 0;   // score buffer of tile t and the parity of its phase
+    if (T > 0) {
+      wait_all(bar(B_SF), 0);
+      tc_fence_after();
+      fetch_scores(0, 0);
+    }
     for (int t = 0; t < T; ++t) {
-      const int buf = t % NSB, vst = t % VST;
       const int g0 = pc_begin + t * PPT;
-      // real keys in each piece of the tile, and the allowed columns of this thread's piece
-      int valid[PPT];
-      bool cache_tile = false, short_tile = false;
-#pragma unroll
-      for (int j = 0; j < PPT; ++j) {
-        const int g = g0 + j;
-        if (g >= pc_end) valid[j] = -1;                       // no such piece: P V skips it
-        else if (g < p_cache) { valid[j] = min(PG, L - g * PG); cache_tile = true; }
-        else valid[j] = min(PG, N - (g - p_cache) * PG);
-        short_tile |= (valid[j] >= 0 && valid[j] < PG);
-      }
       const int g = g0 + ch;
       const bool present = g < pc_end;
-      uint32_t allow0 = 0, allow1 = 0;
-      if (present && row_valid) {
-        if (g < p_cache) {
-          const uint64_t bits = valid[ch] >= 64 ? ~0ull : ((1ull << valid[ch]) - 1ull);
-          allow0 = (uint32_t)bits; allow1 = (uint32_t)(bits >> 32);
-        } else {
-          const int tp = g - p_cache;
-          allow0 = s_anc[node][2 * tp]; allow1 = s_anc[node][2 * tp + 1];
-        }
-      }
-      auto wait_all = [&](uint32_t barrier, uint32_t parity) {   // warp-uniform verdict
-        if (fail) return;
-        const bool w_ok = mbar_wait(barrier, parity, abort_flag, wlim);
-        fail = !__all_sync(0xFFFFFFFFu, w_ok);
-      };
-      wait_all(bar(B_SF + buf), (t / NSB) & 1);
-      tc_fence_after();
-      if (p.paged && cache_tile) {
-        // the producer's verdict on this tile's pages, written before it armed the V barrier
-        wait_all(bar(B_VF + vst), (t / VST) & 1);
-        if (!fail && !*(volatile int*)&s_tile_ok[vst]) {  // sequence is flagged; hide the whole tile
-          short_tile = true;
+      // real keys in each piece of the tile, and the allowed columns of this thread's piece
+      int valid[PPT] = {PG, PG};
+      bool short_tile = false, need_mask = !warp_rows_valid;
+      uint32_t allow0 = row_valid ? 0xFFFFFFFFu : 0u, allow1 = allow0;
+      if (t >= t_plain) {
 #pragma unroll
-          for (int j = 0; j < PPT; ++j) if (valid[j] > 0) valid[j] = 0;
-          allow0 = allow1 = 0;
+        for (int j = 0; j < PPT; ++j) {
+          const int gj = g0 + j;
+          if (gj >= pc_end) valid[j] = -1;                       // no such piece: P V skips it
+          else if (gj < p_cache) valid[j] = min(PG, L - gj * PG);
+          else valid[j] = min(PG, N - (gj - p_cache) * PG);
+          short_tile |= (valid[j] >= 0 && valid[j] < PG);
+        }
+        need_mask = true;
+        allow0 = allow1 = 0;
+        if (present && row_valid) {
+          if (g < p_cache) {
+            const uint64_t bits = valid[ch] >= 64 ? ~0ull : ((1ull << valid[ch]) - 1ull);
+            allow0 = (uint32_t)bits; allow1 = (uint32_t)(bits >> 32);
+          } else {
+            const int tp = g - p_cache;
+            allow0 = s_anc[node][2 * tp]; allow1 = s_anc[node][2 * tp + 1];
+          }
         }
       }
-      const bool all_full = __all_sync(0xFFFFFFFFu, (allow0 & allow1) == 0xFFFFFFFFu);
-
-      uint32_t sv[64];
-      // this thread's 64 scores; columns that are not allowed become -inf
-      auto load_scores = [&]() {
-        tmem_ld_x64(tmem_S(buf) + lane_addr + ch * 64, sv);
-        tmem_wait_ld();
-        if (!all_full) {
+      if (present && !fail) {
+        tmem_wait_ld();   // the scores of this tile
+        if (need_mask) {  // columns that are not allowed become -inf
 #pragma unroll
           for (int j = 0; j < 64; ++j) {
             const uint32_t wbits = (j < 32) ? allow0 : allow1;
-            if (!((wbits >> (j & 31)) & 1u)) sv[j] = 0xFF800000u;  // -inf
+            if (!((wbits >> (j & 31)) & 1u)) sv[j] = 0xFF800000u;
           }
         }
-      };
-      // One pass with the reference maximum as it stands: exponentiate, pack P (kept in registers)
-      // and add up.  No per-element maximum is tracked: a sum of at most 2^8 proves that no
-      // probability exceeded 2^8, i.e. that the reference is still good.  Otherwise (rare after
-      // the first tile; inf or NaN from an overflow also lands here) the true maximum of the row is
-      // taken from the scores - still intact, because P is stored last - the reference replaced,
-      // O rescaled and the tile redone.  The two threads of a row decide together.
-      uint32_t pk[32];
+      }
+      // One pass with the reference maximum as it stands: exponentiate, pack P and add up.  P goes
+      // to tensor memory as soon as 32 keys are done: keys 64 ch + 32 h .. + 31 of the tile land in
+      // columns 64 ch + 16 h .. + 15 of the score buffer (two bf16 per column), i.e. on top of
+      // scores that this very thread has already taken.  No per-element maximum is tracked: a sum
+      // of at most 2^8 proves that no probability exceeded 2^8, i.e. that the reference is still
+      // good.  Otherwise (rare after the first tile; inf or NaN from an overflow also lands here)
+      // the true maximum of the row is taken from the scores, the reference replaced, O rescaled
+      // and the tile redone from the registers.  The two threads of a row decide together.
       float sum = 0.f;
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       auto exp_pass = [&]() {
         sum = 0.f;
         if (!present || fail) return;
-        load_scores();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), p.scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), p.scale_log2, neg_m));
-          sum += p0 + p1;
-          pk[j] = pack_bf16(p0, p1);
+        for (int h = 0; h < 2; ++h) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[32 * h + 2 * j]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[32 * h + 2 * j + 1]), p.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[j] = pack_bf16(p0, p1);
+          }
+          tmem_st_x16(tmem_S(buf) + lane_addr + ch * 64 + h * 16, pk);
         }
       };
       if (t > 0) {
@@ -685,8 +691,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         (*(volatile int*)&s_redo[sw] == t) || (*(volatile int*)&s_redo[sw ^ 4] == t);
       if (redo) {
         float mx = -INFINITY;
-        if (present) {
-          load_scores();
+        if (present && !fail) {
 #pragma unroll
           for (int j = 0; j < 64; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
           mx *= p.scale_log2;   // scale > 0; -inf (no allowed key) stays -inf
@@ -702,6 +707,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const float alpha = need ? ex2(m_ref - mx) : 1.0f;  // ex2(-inf) = 0
         if (need) { m_ref = mx; l_run *= alpha; }
         if (t > 0 && !fail) {
+          if (present) tmem_wait_st();   // this thread's stores of the first pass, before it touches O
 #pragma unroll 1
           for (int cc = 0; cc < 64; cc += 32) {
             uint32_t ov[32];
@@ -715,19 +721,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
         exp_pass();
-        named_barrier(pair_bar, 64);   // the partner has read its scores: P may overwrite them
-      }
-      // P (the A operand of P V) takes the place of score columns that have been consumed: keys
-      // 64 ch .. 64 ch + 63 of the tile are columns 32 ch .. 32 ch + 31 (two bf16 per column).
-      if (present && !fail) {
-        tmem_st_x32(tmem_S(buf) + lane_addr + ch * 32, pk);
-        tmem_wait_st();
       }
       l_run += sum;
+      // the next tile's scores travel to the registers while this tile's P travels the other way
+      const int nbuf = (buf == NSB - 1) ? 0 : buf + 1;
+      const uint32_t nph = (buf == NSB - 1) ? ph ^ 1u : ph;
+      if (t + 1 < T) {
+        wait_all(bar(B_SF + nbuf), nph);
+        tc_fence_after();
+        fetch_scores(t + 1, nbuf);
+      }
+      if (present && !fail) tmem_wait_st();
 
       if (short_tile) {
         // Rows of a V piece beyond its real keys hold whatever lies behind them in memory; their
         // probabilities are exactly 0, but 0 * NaN would poison O: clear them.
+        const int vst = t % VST;
         wait_all(bar(B_VF + vst), (t / VST) & 1);
         if (!fail) {
           uint8_t* vt = sV_gen + vst * kStage;
@@ -749,6 +758,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0 && !fail) mbar_arrive_cluster(pf_leader0 + 8u * (uint32_t)buf);
+      buf = nbuf;
+      ph = nph;
     }
 
     if (!fail && !*abort_flag && T > 0) {  // the last P V has landed in O
