@@ -6,15 +6,8 @@
 // its other rows idle).  One thread block owns ONE row tile of one (sequence, kv head) and a
 // contiguous range of the key axis (cache keys first, then the tree's own), walked in tiles of
 // 128 keys that are loaded as 64-key pieces (also the page size of a paged cache).
-//   CG = 1: the block works alone (the unit has a single row tile).
-//   CG = 2: two blocks on neighbouring SMs share every MMA (cta_group::2, M = 256): each holds its
-//           own row tile, and each stages only HALF of every K and V tile - K: one 64-key piece,
-//           V: one 64-wide half of the head dimension - so a unit of two row tiles costs each SM
-//           half the shared-memory fill.  Every block's TMA copies signal its own barriers (so it
-//           can wait for, patch and drain its own tiles); a relay thread of the odd block forwards
-//           the completions to the even block, whose single thread issues the pair's MMAs.
-// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (even block) or relay (odd block), owner of
-// the tensor-memory allocation; warps 2-9 = softmax, two threads per query row: thread `ch` of a
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer and owner of the tensor-memory allocation;
+// warps 2-9 = softmax, two threads per query row: thread `ch` of a
 // row takes the 64 columns of piece `ch` of every key tile.
 // Tensor memory: three score buffers of 128 columns and one output accumulator of 128.  The
 // issuer runs Q K^T up to three tiles ahead, so the softmax threads find the next scores ready
@@ -24,7 +17,7 @@
 // columns -> O += P V (A operand from tensor memory).  The tree columns are masked with per-node
 // ancestor bitsets derived from parent[] on chip; masked scores are replaced, not added to, so
 // they contribute exactly zero.
-// Split-KV: the blocks (pairs) that share a row tile form one thread-block cluster; each stages
+// Split-KV: the blocks that share a row tile form one thread-block cluster; each stages
 // its accumulator in its own shared memory and every block finalises a share of the rows by
 // reading its peers' staging areas (distributed shared memory): no partial result touches global
 // memory.  Every wait is bounded: on expiry the block raises a flag, all roles leave their loops,
@@ -57,11 +50,10 @@ constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRowSumLimit = 256.0f;        // a thread's part of a row of P may sum to 2^8 before the reference is replaced
 
-template <int CG>
 struct Cfg {
-  static constexpr int KST = NSB;                        // a K buffer and a score buffer free together
-  static constexpr int VST = (CG == 2) ? NSB : 2;        // depth of the V ring
-  static constexpr uint32_t kStage = BN * HD * 2 / CG;   // bytes of this block's share of a K (or V) tile
+  static constexpr int KST = NSB;                   // a K buffer and a score buffer free together
+  static constexpr int VST = 2;                     // depth of the V ring
+  static constexpr uint32_t kStage = BN * HD * 2;   // bytes of a K (or V) tile
   static constexpr uint32_t kSmem = kQTile + (KST + VST) * kStage + 1024;
 };
 
@@ -75,9 +67,8 @@ struct Params {
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
   int longest_first;  // hand out sequences in order of decreasing context length
-  int row_groups;  // clusters along the row axis per (sequence, kv head); each covers CG row tiles
-  int tiles;       // row tiles per (sequence, kv head)
-  int splits;      // blocks (pairs) along the key axis; cluster size = CG * splits
+  int tiles;       // row tiles per (sequence, kv head); each is worked by one cluster
+  int splits;      // blocks along the key axis = cluster size
   float scale_log2;
   long long wait_limit;   // SM cycles a bounded wait may last
   unsigned* tickets;      // per sequence: [2b] blocks that have finished, [2b+1] error bits; zero between calls
@@ -114,32 +105,15 @@ __device__ __forceinline__ void named_barrier(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-template <int CG>
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-  if (CG == 2) umma_bf16_pair(d, a, b, idesc, acc);
-  else umma_bf16(d, a, b, idesc, acc);
-}
-template <int CG>
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-  if (CG == 2) umma_bf16_ts_pair(d, a, b, idesc, acc);
-  else umma_bf16_ts(d, a, b, idesc, acc);
-}
-// one arrival, once the MMAs issued so far are complete, at barrier `bar` of every block of the pair
-template <int CG>
-__device__ __forceinline__ void commit_all(uint32_t bar, uint16_t pair_mask) {
-  if (CG == 2) umma_commit_pair_both(bar, pair_mask);
-  else umma_commit(bar);
-}
-
 // Final combination of NSRC accumulators per output row, for the rows [first_row, first_row +
 // per_rank) of the tile that this block finalises.  The staged accumulators are fp16 (each row
 // scaled by a power of two of its own, which the weight undoes), 256 bytes per row.  One warp takes
 // 16 / NSRC rows at a time (16 remote 8-byte loads in flight per lane); lane j owns output
 // columns 4j .. 4j+3.  w[] holds the normalised weights divided by the rows' scales; source q of
-// a row lives in cluster rank q * rank_stride + rank_base.
+// a row lives in cluster rank q.
 template <int NSRC>
 __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank, int rot,
-                                           int rank_stride, int rank_base, int warp, int lane, int tile_row0,
+                                           int warp, int lane, int tile_row0,
                                            int RT, int rows_total, int G, int64_t seq_row0, int Hq, int head0,
                                            uint16_t* out) {
   constexpr int RB = 16 / NSRC;
@@ -152,7 +126,7 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
         const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
-        x[u * NSRC + j] = dsmem_ld8u(cluster_map(sO_addr + off, (uint32_t)(q * rank_stride + rank_base)));
+        x[u * NSRC + j] = dsmem_ld8u(cluster_map(sO_addr + off, (uint32_t)q));
       }
     }
 #pragma unroll
@@ -177,25 +151,21 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
 }
 
 // ------------------------------------------------------------------------------------ kernel
-template <int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                     const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
                     const __grid_constant__ CUtensorMap tm_vt, const Params p) {
-  constexpr int KST = Cfg<CG>::KST, VST = Cfg<CG>::VST;
-  constexpr uint32_t kStage = Cfg<CG>::kStage;
-  constexpr uint32_t kKHalf = kStage / 2;   // K stage: [64-wide half of d][keys of this block][64 d]
-  constexpr bool kVOwnRing = (VST != NSB);  // V buffers then have hand-back barriers of their own
-  constexpr uint32_t kIdescQK = make_idesc(BM * CG, BN, false);  // S[rows x 128 keys] = Q K^T
-  constexpr uint32_t kIdescPV = make_idesc(BM * CG, HD, true);   // O[rows x 128 d] += P V
+  constexpr int KST = Cfg::KST, VST = Cfg::VST;
+  constexpr uint32_t kStage = Cfg::kStage;
+  constexpr uint32_t kHalf = kStage / 2;    // a stage holds [64-wide half of d][128 keys][64 d]
+  constexpr uint32_t kIdescQK = make_idesc(BM, BN, false);  // S[128 rows x 128 keys] = Q K^T
+  constexpr uint32_t kIdescPV = make_idesc(BM, HD, true);   // O[128 rows x 128 d] += P V
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_anc[CLV_MAX_NODES][4];
   __shared__ int s_parent[CLV_MAX_NODES];
-  // barriers: K full [KST] | V full [VST] | S full [NSB] | P full [NSB] | P V done [NSB] | V empty [VST] | Q |
-  //           drain | the peer's K [KST], V [VST] and Q have landed (arrivals of the relay; even block only)
+  // barriers: K full [KST] | V full [VST] | S full [NSB] | P full [NSB] | P V done [NSB] | V empty [VST] | Q | drain
   constexpr int B_KF = 0, B_VF = B_KF + KST, B_SF = B_VF + VST, B_PF = B_SF + NSB, B_PV = B_PF + NSB,
-                B_VE = B_PV + NSB, B_Q = B_VE + VST, B_DR = B_Q + 1, B_KP = B_DR + 1, B_VP = B_KP + KST,
-                B_QP = B_VP + VST, NBAR = B_QP + 1;
+                B_VE = B_PV + NSB, B_Q = B_VE + VST, B_DR = B_Q + 1, NBAR = B_DR + 1;
   __shared__ __align__(8) unsigned long long s_bar[NBAR];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -208,21 +178,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ int s_seq;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int CS = CG * p.splits;                       // cluster size
-  const int crank = (int)(blockIdx.x % (unsigned)CS); // rank in the cluster (clusters are laid along x)
-  const int c = (CG == 2) ? (crank & 1) : 0;          // block of the pair
-  const int split = crank / CG;
+  const int CS = p.splits;                            // cluster size
+  const int split = (int)(blockIdx.x % (unsigned)CS); // rank in the cluster (clusters are laid along x)
   const int cluster_id = (int)(blockIdx.x / (unsigned)CS);
-  const int unit = cluster_id / p.row_groups, rgrp = cluster_id - unit * p.row_groups;
+  const int unit = cluster_id / p.tiles, tile_idx = cluster_id - unit * p.tiles;   // this block's row tile
   int b = unit / p.Hkv;
   const int kvh = unit - b * p.Hkv;
   const int N = p.N, G = p.G, rows_total = G * N;
   const int RT = (BM / G) * G;                        // rows of a tile that hold whole nodes
-  const int tile_idx = rgrp * CG + c;                 // this block's row tile of the unit
-  const bool has_rows = tile_idx < p.tiles;
-  const bool leader = (c == 0);
-  const uint32_t leader_rank = (uint32_t)(crank & ~(CG - 1));
-  const uint16_t pair_mask = (uint16_t)((CG == 2 ? 3u : 1u) << leader_rank);
 
   // ---- set-up that reads no global memory: barriers, tensor memory, descriptor prefetch.  The
   //      kernel is launched with programmatic stream serialisation, so this part may run while the
@@ -230,33 +193,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   auto bar = [&](int idx) { return bar0 + 8u * (uint32_t)idx; };
   if (tid == 0) {
-    for (int i = 0; i < KST; ++i) { mbar_init(bar(B_KF + i), 1); mbar_init(bar(B_KP + i), 1); }
-    for (int i = 0; i < VST; ++i) {
-      mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1); mbar_init(bar(B_VP + i), 1);
-    }
+    for (int i = 0; i < KST; ++i) mbar_init(bar(B_KF + i), 1);
+    for (int i = 0; i < VST; ++i) { mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1); }
     for (int i = 0; i < NSB; ++i) {
       mbar_init(bar(B_SF + i), 1);
-      mbar_init(bar(B_PF + i), 8u * CG);   // one arrival per softmax warp of the pair
+      mbar_init(bar(B_PF + i), 8);   // one arrival per softmax warp
       mbar_init(bar(B_PV + i), 1);
     }
     mbar_init(bar(B_Q), 1);
-    mbar_init(bar(B_QP), 1);
     mbar_init(bar(B_DR), 1);
     s_abort = 0;
     for (int i = 0; i < 8; ++i) { s_redo[i] = -1; s_fail[i] = 0; }
     fence_barrier_init();
     fence_async_smem();
   }
-  if (warp == 1) {
-    if (CG == 2) tmem_alloc_pair(smem_u32(&s_tmem), kTmemCols);
-    else tmem_alloc(smem_u32(&s_tmem), kTmemCols);
-  }
+  if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
   if (tid == 64) {
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
     tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
   }
-  __syncthreads();                     // this block's barriers exist ...
-  if (CG == 2) cluster_arrive();       // ... and the peer learns of it at the matching wait below
   cudaGridDependencySynchronize();
 
   if (p.longest_first) {
@@ -292,9 +247,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_before();
   const int seq_bad = __syncthreads_or(bad ? 1 : 0);  // same verdict in every block of the sequence
   tc_fence_after();
-  if (CG == 2) cluster_wait();         // the peer's barriers exist: remote arrivals may begin
   const uint32_t tmem = s_tmem;
-  const bool reporter = (rgrp == 0 && crank == 0 && kvh == 0);
+  const bool reporter = (tile_idx == 0 && split == 0 && kvh == 0);
   // status[b] is written once, by whichever block of the sequence finishes last: every block adds
   // its error bits (1 malformed input, 2 a wait ran out) to the sequence's word in the workspace
   // and then takes a ticket; the holder of the last ticket turns the bits into the status code and
@@ -310,10 +264,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const unsigned bits = atomicExch(p.tickets + 2 * b + 1, 0u);
     p.status[b] = (bits & 1u) ? CLV_ERR_TREE : (bits & 2u) ? CLV_ERR_TIMEOUT : CLV_OK;
   };
-  auto release_tmem = [&]() {   // warp 1 of every block of the pair
-    if (CG == 2) tmem_dealloc_pair(tmem, kTmemCols);
-    else tmem_dealloc(tmem, kTmemCols);
-  };
+  auto release_tmem = [&]() { tmem_dealloc(tmem, kTmemCols); };   // warp 1
   if (seq_bad) {  // the whole cluster leaves together; nothing has been issued yet
     if (warp == 1) release_tmem();
     if (tid == 0) publish(report(1u));
@@ -350,7 +301,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int quarter = warp & 3;                  // TMEM lanes this warp may touch
   const int row = quarter * 32 + lane;           // row inside the 128-row tile
   const int r_glob = tile_idx * RT + row;
-  const bool row_valid = has_rows && row < RT && r_glob < rows_total;
+  const bool row_valid = row < RT && r_glob < rows_total;
   const int node = row_valid ? r_glob / G : 0;
   const int gq = row_valid ? r_glob - node * G : 0;
   const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
@@ -387,7 +338,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int g = g0 + j;
             int pg = __shfl_sync(0xFFFFFFFFu, pk_page, (g - pk_base) & 31);
             is_tree[j] = g >= p_cache;
-            if (g >= pc_end || (CG == 2 && j != c)) row0[j] = -1;     // absent, or the peer's piece
+            if (g >= pc_end) row0[j] = -1;     // the range ended inside this tile
             else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
             else if (p.paged) { if (pg < 0 || pg >= p.n_pages) pg = 0; row0[j] = pg * PG; }
             else row0[j] = b * p.cap_tokens + g * PG;
@@ -401,9 +352,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
               const CUtensorMap* mk = is_tree[j] ? &tm_kt : &tm_kc;
-              const uint32_t dst = sK + st * kStage + (CG == 2 ? 0u : (uint32_t)j * kPiece);
+              const uint32_t dst = sK + st * kStage + (uint32_t)j * kPiece;
               tma_load_3d(dst, mk, 0, kvh, row0[j], bar(B_KF + st));
-              tma_load_3d(dst + kKHalf, mk, 64, kvh, row0[j], bar(B_KF + st));
+              tma_load_3d(dst + kHalf, mk, 64, kvh, row0[j], bar(B_KF + st));
             }
           }
           ++kt;
@@ -411,12 +362,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           progress = true;
         }
       }
-      // ---- V of tile vt: CG = 1: both pieces, both halves of d;  CG = 2: both pieces, half c of d
+      // ---- V of tile vt
       if (vt < T) {
         const int st = vt % VST;
         int ready = 1;
         if (vt >= VST && lane == 0)
-          ready = mbar_test(bar((kVOwnRing ? B_VE : B_PV) + st), ((vt / VST) - 1) & 1) ? 1 : 0;
+          ready = mbar_test(bar(B_VE + st), ((vt / VST) - 1) & 1) ? 1 : 0;
         ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
         if (ready) {
           const int g0 = pc_begin + vt * PPT;
@@ -443,18 +394,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int n_pieces = 0;
 #pragma unroll
             for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
-            mbar_expect_tx(bar(B_VF + st), (uint32_t)n_pieces * (CG == 2 ? 1u : 2u) * kPiece);
+            mbar_expect_tx(bar(B_VF + st), (uint32_t)n_pieces * 2u * kPiece);
 #pragma unroll
             for (int j = 0; j < PPT; ++j) {
               if (row0[j] < 0) continue;
               const CUtensorMap* mv = is_tree[j] ? &tm_vt : &tm_vc;
               const uint32_t dst = sV + st * kStage + (uint32_t)j * kPiece;
-              if (CG == 2) {
-                tma_load_3d(dst, mv, 64 * c, kvh, row0[j], bar(B_VF + st));
-              } else {
-                tma_load_3d(dst, mv, 0, kvh, row0[j], bar(B_VF + st));
-                tma_load_3d(dst + kStage / 2, mv, 64, kvh, row0[j], bar(B_VF + st));
-              }
+              tma_load_3d(dst, mv, 0, kvh, row0[j], bar(B_VF + st));
+              tma_load_3d(dst + kHalf, mv, 64, kvh, row0[j], bar(B_VF + st));
             }
           }
           ++vt;
@@ -474,92 +421,55 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
     }
   } else if (warp == 1) {
-    if (leader) {
-      // =========================== MMA issuer ===================================================
-      if (lane == 0 && T > 0) {
-        // a tile is ready when this block's copies have landed and, in a pair, the relay has
-        // reported the peer's
-        auto wait_both = [&](int own, int peer, uint32_t parity) -> bool {
-          if (!mbar_wait(bar(own), parity, abort_flag, wlim)) return false;
-          return CG == 1 || mbar_wait_cluster(bar(peer), parity, abort_flag, wlim);
-        };
-        bool ok = wait_both(B_Q, B_QP, 0);
+    // =========================== MMA issuer ===================================================
+    if (lane == 0 && T > 0) {
+      bool ok = mbar_wait(bar(B_Q), 0, abort_flag, wlim);
+      tc_fence_after();
+      // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
+      // constant (the address field counts 16-byte units and never carries out of its 14 bits).
+      const uint64_t q_desc = smem_desc(sQ, 16, 1024);
+      const uint64_t k_desc = smem_desc(sK, 16, 1024);
+      const uint64_t v_desc = smem_desc(sV, kHalf, 1024);   // lbo: the other half of d
+      auto issue_qk = [&](int t) -> bool {
+        const int st = t % KST;
+        if (!mbar_wait(bar(B_KF + st), (t / KST) & 1, abort_flag, wlim)) return false;
         tc_fence_after();
-        // Descriptors are built once; inside the loops an operand's descriptor is a base plus a
-        // constant (the address field counts 16-byte units and never carries out of its 14 bits).
-        const uint64_t q_desc = smem_desc(sQ, 16, 1024);
-        const uint64_t k_desc = smem_desc(sK, 16, 1024);
-        const uint64_t v_desc = smem_desc(sV, kStage / 2, 1024);   // lbo: the other half of d (CG = 1)
-        auto issue_qk = [&](int t) -> bool {
-          const int st = t % KST;
-          if (!wait_both(B_KF + st, B_KP + st, (t / KST) & 1)) return false;
-          tc_fence_after();
-          const uint64_t kd = k_desc + (uint64_t)((st * kStage) >> 4);
+        const uint64_t kd = k_desc + (uint64_t)((st * kStage) >> 4);
 #pragma unroll
-          for (int ks = 0; ks < HD / 16; ++ks) {
-            const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
-            const uint32_t ko = (ks >> 2) * kKHalf + (ks & 3) * 32;
-            mma_ss<CG>(tmem_S(t % NSB), q_desc + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
-          }
-          commit_all<CG>(bar(B_SF + t % NSB), pair_mask);   // scores ready; this K buffer is free
-          return true;
-        };
-        for (int t = 0; t < NSB && t < T && ok; ++t) ok = issue_qk(t);
-        for (int t = 0; t < T && ok; ++t) {
-          const int buf = t % NSB, st = t % VST;
-          ok = mbar_wait_cluster(bar(B_PF + buf), (t / NSB) & 1, abort_flag, wlim);
-          if (!ok) break;
-          ok = wait_both(B_VF + st, B_VP + st, (t / VST) & 1);
-          if (!ok) break;
-          tc_fence_after();
-          const int n_kk = min(PPT, pc_end - (pc_begin + t * PPT)) * (PG / 16);   // a missing piece is skipped
-          const uint64_t vd = v_desc + (uint64_t)((st * kStage) >> 4);
-          // P of piece j of the tile sits in the first 32 columns of that piece's 64 score columns
-          for (int kk = 0; kk < n_kk; ++kk)
-            mma_ts<CG>(tmem_O, tmem_S(buf) + (kk >> 2) * 64 + (kk & 3) * 8, vd + (uint64_t)((kk * 2048) >> 4),
-                       kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
-          commit_all<CG>(bar(B_PV + buf), pair_mask);   // O holds tile t; P buffer (and with it the V buffer) free
-          if (kVOwnRing) commit_all<CG>(bar(B_VE + st), pair_mask);
-          if (t + NSB < T) ok = issue_qk(t + NSB);
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t qo = (ks >> 2) * (kQTile / 2) + (ks & 3) * 32;
+          const uint32_t ko = (ks >> 2) * kHalf + (ks & 3) * 32;
+          umma_bf16(tmem_S(t % NSB), q_desc + (qo >> 4), kd + (ko >> 4), kIdescQK, ks > 0 ? 1u : 0u);
         }
-      }
-    } else {
-      // =========================== relay (odd block of a pair) ==================================
-      // forwards "my share of this tile has landed" to the barriers of the block that issues
-      if (lane == 0 && T > 0) {
-        bool ok = mbar_wait(bar(B_Q), 0, abort_flag, wlim);
-        if (ok) mbar_arrive_cluster(cluster_map(bar(B_QP), leader_rank));
-        int kt = 0, vt = 0;
-        long long t_idle = clock64();
-        while (ok && (kt < T || vt < T)) {
-          bool progress = false;
-          if (kt < T && mbar_test(bar(B_KF + kt % KST), (kt / KST) & 1)) {
-            mbar_arrive_cluster(cluster_map(bar(B_KP + kt % KST), leader_rank));
-            ++kt;
-            progress = true;
-          }
-          if (vt < T && mbar_test(bar(B_VF + vt % VST), (vt / VST) & 1)) {
-            mbar_arrive_cluster(cluster_map(bar(B_VP + vt % VST), leader_rank));
-            ++vt;
-            progress = true;
-          }
-          if (progress) t_idle = clock64();
-          else if (*abort_flag) ok = false;
-          else if (clock64() - t_idle > wlim) { *abort_flag = 1; ok = false; }
-        }
+        umma_commit(bar(B_SF + t % NSB));   // scores ready; this K buffer is free
+        return true;
+      };
+      for (int t = 0; t < NSB && t < T && ok; ++t) ok = issue_qk(t);
+      for (int t = 0; t < T && ok; ++t) {
+        const int buf = t % NSB, st = t % VST;
+        ok = mbar_wait(bar(B_PF + buf), (t / NSB) & 1, abort_flag, wlim);
+        if (!ok) break;
+        ok = mbar_wait(bar(B_VF + st), (t / VST) & 1, abort_flag, wlim);
+        if (!ok) break;
+        tc_fence_after();
+        const int n_kk = min(PPT, pc_end - (pc_begin + t * PPT)) * (PG / 16);   // a missing piece is skipped
+        const uint64_t vd = v_desc + (uint64_t)((st * kStage) >> 4);
+        // P of piece j of the tile sits in the first 32 columns of that piece's 64 score columns
+        for (int kk = 0; kk < n_kk; ++kk)
+          umma_bf16_ts(tmem_O, tmem_S(buf) + (kk >> 2) * 64 + (kk & 3) * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                     kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bar(B_PV + buf));   // O holds tile t
+        umma_commit(bar(B_VE + st));    // this V buffer is free
+        if (t + NSB < T) ok = issue_qk(t + NSB);
       }
     }
   } else {
     // =========================== softmax threads ==============================================
     if (warp == 2 && T > 0 && lane == 0) {  // the Q tile: issued here so that the producer starts with K/V
-      if (has_rows) {
-        mbar_expect_tx(bar(B_Q), (uint32_t)(RT * HD * 2));   // the boxes hold RT rows
-        const int node0 = b * N + tile_idx * (BM / G);
-        tma_load_3d(sQ, &tm_q, 0, kvh * G, node0, bar(B_Q));
-        tma_load_3d(sQ + kQTile / 2, &tm_q, 64, kvh * G, node0, bar(B_Q));
-      } else {
-        mbar_arrive(bar(B_Q));   // a block without rows (odd number of row tiles) loads no Q
-      }
+      mbar_expect_tx(bar(B_Q), (uint32_t)(RT * HD * 2));   // the boxes hold RT rows
+      const int node0 = b * N + tile_idx * (BM / G);
+      tma_load_3d(sQ, &tm_q, 0, kvh * G, node0, bar(B_Q));
+      tma_load_3d(sQ + kQTile / 2, &tm_q, 64, kvh * G, node0, bar(B_Q));
     }
     // ancestor bitsets (row i of the tree's topology matrix), built while the first tiles are on
     // their way; the 256 threads meet at a named barrier of their own
@@ -584,7 +494,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (lane == 0 && pbad) atomicOr(p.tickets + 2 * b + 1, 1u);  // before this block's ticket
     }
     named_barrier(1, kSoftmaxThreads);
-    const uint32_t pf_leader0 = cluster_map(bar(B_PF), leader_rank);
 
     // A wait that runs out raises the block's abort flag and sets `fail`; the thread then skips
     // the work but keeps walking through the named barriers it shares with its partner warp, and
@@ -741,7 +650,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (!fail) {
           uint8_t* vt = sV_gen + vst * kStage;
           const int me = tid - 64;   // 0 .. 255 among the softmax threads
-          constexpr int kHalves = (CG == 2) ? 1 : 2;   // halves of the head dimension held here
+          constexpr int kHalves = 2;   // halves of the head dimension
 #pragma unroll
           for (int j = 0; j < PPT; ++j) {
             if (valid[j] < 0) continue;
@@ -749,7 +658,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int cidx = me; cidx < kHalves * per_half; cidx += kSoftmaxThreads) {
               const int half = cidx / per_half, rem = cidx - half * per_half;
               const int vr = j * PG + valid[j] + (rem >> 3), chk = rem & 7;
-              *reinterpret_cast<uint4*>(vt + half * (kStage / 2) + vr * 128 + chk * 16) = make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4*>(vt + half * kHalf + vr * 128 + chk * 16) = make_uint4(0, 0, 0, 0);
             }
           }
           fence_async_smem();   // cleared V rows visible to the tensor core's reads
@@ -757,7 +666,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0 && !fail) mbar_arrive_cluster(pf_leader0 + 8u * (uint32_t)buf);
+      if (lane == 0 && !fail) mbar_arrive(bar(B_PF + buf));
       buf = nbuf;
       ph = nph;
     }
@@ -776,9 +685,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int i = max(0, issued_k - KST); i < issued_k; ++i) mbar_drain(bar(B_KF + i % KST), (i / KST) & 1);
       for (int i = max(0, issued_v - VST); i < issued_v; ++i) mbar_drain(bar(B_VF + i % VST), (i / VST) & 1);
     }
-    if (warp == 2 && lane == 0 && T > 0 && has_rows) mbar_drain(bar(B_Q), 0);
-    if (warp == 1 && lane == 0 && leader) {
-      if (CG == 2) umma_commit_pair(bar(B_DR)); else umma_commit(bar(B_DR));
+    if (warp == 2 && lane == 0 && T > 0) mbar_drain(bar(B_Q), 0);
+    if (warp == 1 && lane == 0) {
+      umma_commit(bar(B_DR));
       mbar_drain(bar(B_DR), 0);  // completes when every MMA issued so far has finished
     }
   }
@@ -887,7 +796,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   cluster.sync();  // every block's staging area is complete and its MMAs are done (also reached by an aborted block)
   if (n_src > 1 && !aborted) {
     // ---- merge across the key splits through distributed shared memory: split j finalises rows
-    //      [j, j+1) * 128 / splits of the tile; source q of a row lives in cluster rank q CG + c ----
+    //      [j, j+1) * 128 / splits of the tile; source q of a row lives in cluster rank q ----
     const int per_rank = BM / p.splits;
     const int first_row = split * per_rank;
     // (a) thread (k, q) fetches the (maximum, sum, scale) of source q of row k; the n_src lanes of
@@ -895,7 +804,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (tid < BM) {
       const int k = tid / n_src, q = tid - k * n_src;
       const int trow = first_row + k;
-      const float4 ml = dsmem_ld16(cluster_map(smem_u32(&s_ml[trow]), (uint32_t)(q * CG + c)));
+      const float4 ml = dsmem_ld16(cluster_map(smem_u32(&s_ml[trow]), (uint32_t)q));
       float mmax = ml.x;
       for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
       const float mu = (mmax == -INFINITY) ? 0.f : mmax;
@@ -904,21 +813,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int o = 1; o < n_src; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
       s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
       const int rg = tile_idx * RT + trow;
-      if (q == 0 && p.lse != nullptr && has_rows && trow < RT && rg < rows_total) {
+      if (q == 0 && p.lse != nullptr && trow < RT && rg < rows_total) {
         const int onode = rg / G, ogq = rg - onode * G;
         p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
       }
     }
     __syncthreads();
     // (b) weighted sums, rows spread over the warps
-    if (has_rows) {
+    {
       const uint32_t sO_addr = smem_u32(sO);
       const int rot = split + 1;  // first source read: the next split's
       const int64_t seq_row0 = (int64_t)b * N;
       switch (n_src) {
-        case 2: merge_rows<2>(sO_addr, s_w, first_row, per_rank, rot, CG, c, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-        case 4: merge_rows<4>(sO_addr, s_w, first_row, per_rank, rot, CG, c, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-        default: merge_rows<8>(sO_addr, s_w, first_row, per_rank, rot, CG, c, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+        case 2: merge_rows<2>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+        case 4: merge_rows<4>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+        default: merge_rows<8>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
       }
     }
   }
@@ -959,17 +868,14 @@ bool tc_attn_supported(const clv_shape& s, const clv_kv_cache& c) {
 
 AttnPlan tc_attn_plan(const clv_shape& s, int max_ctx_len) {
   AttnPlan pl;
-  const int tiles = row_tiles(s);
-  const int cgrp = tiles > 1 ? 2 : 1;                  // units of several row tiles are worked by pairs
-  pl.m_tiles = (tiles + cgrp - 1) / cgrp;
-  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * pl.m_tiles * cgrp;
+  pl.m_tiles = row_tiles(s);
+  const int64_t ctas = (int64_t)s.batch * s.n_kv_heads * pl.m_tiles;
   const int key_tiles = (max_ctx_len > 0 ? (max_ctx_len + BN - 1) / BN : 0) + (s.n_nodes + BN - 1) / BN;
   // The key axis is split over a thread-block cluster (merged through distributed shared memory):
-  // a power of two that keeps the cluster within the portable size of 8 and the grid within one
-  // block per SM, and leaves every block at least two key tiles.
+  // a power of two up to the portable cluster size of 8 that keeps the grid within one block per
+  // SM and leaves every block at least two key tiles.
   int splits = 1;
-  while (cgrp * splits * 2 <= 8 && ctas * (splits * 2) <= sm_count() && key_tiles / (splits * 2) >= 2)
-    splits *= 2;
+  while (splits * 2 <= 8 && ctas * (splits * 2) <= sm_count() && key_tiles / (splits * 2) >= 2) splits *= 2;
   pl.splits = splits;
   pl.tickets = 0;
   pl.scratch_bytes = 0;  // nothing goes through global memory
@@ -983,15 +889,10 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 cudaStream_t stream) {
   (void)scratch;
   const int G = s.n_q_heads / s.n_kv_heads;
-  const int tiles = row_tiles(s);
-  const int cgrp = tiles > 1 ? 2 : 1;   // as in tc_attn_plan
   static OncePerDevice once;
   cudaError_t e0 = run_once_per_device(once, [] {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)Cfg<1>::kSmem);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tree_attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)Cfg<2>::kSmem);
+    return cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)Cfg::kSmem);
   });
   if (e0 != cudaSuccess) return e0;
   alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt;
@@ -1011,35 +912,32 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.status = status;
-  const int cs = cgrp * plan.splits;
   const int64_t clusters = (int64_t)s.batch * s.n_kv_heads * plan.m_tiles;
   p.B = s.batch; p.N = s.n_nodes; p.Hq = s.n_q_heads; p.Hkv = s.n_kv_heads; p.G = G;
   p.paged = c.paged; p.cap_tokens = c.cap_tokens; p.n_pages = c.n_pages; p.max_pages = c.max_pages_per_seq;
-  p.row_groups = plan.m_tiles;
-  p.tiles = tiles;
+  p.tiles = plan.m_tiles;
   p.splits = plan.splits;
-  p.longest_first = (clusters * cs > sm_count() && s.batch > 1 && s.batch <= 256) ? 1 : 0;
+  p.longest_first = (clusters * plan.splits > sm_count() && s.batch > 1 && s.batch <= 256) ? 1 : 0;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.wait_limit = wait_limit_cycles();
   p.tickets = tickets;
-  p.blocks_per_seq = s.n_kv_heads * plan.m_tiles * cs;
+  p.blocks_per_seq = s.n_kv_heads * plan.m_tiles * plan.splits;
 
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(clusters * cs), 1, 1);
+  cfg.gridDim = dim3((unsigned)(clusters * plan.splits), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = cgrp == 1 ? Cfg<1>::kSmem : Cfg<2>::kSmem;
+  cfg.dynamicSmemBytes = Cfg::kSmem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;  // the blocks that share one row group's keys
-  attr[0].val.clusterDim.x = (unsigned)cs;
+  attr[0].id = cudaLaunchAttributeClusterDimension;  // the blocks that share one row tile's keys
+  attr[0].val.clusterDim.x = (unsigned)plan.splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up overlaps the previous kernel's tail
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if (cgrp == 1) return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<1>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
-  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<2>, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
 }
 
 }  // namespace clv
