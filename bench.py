@@ -30,11 +30,8 @@ import numpy as np  # noqa: E402
 METRIC = "verify-step achieved HBM GB/s (algorithmic bytes / step time)"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-ROTATE = 4   # distinct input sets cycled between steps: 4 x 138 MB > 2 x L2 (126 MB)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/verify_step_C3.md; valid for the kernels as they were when that capture was taken
-NCU_TRAFFIC = {("C3", "tree_attn"): 71.7e6, ("C3", "accept_argmax"): 65.9e6}
-
+ROTATE = 32  # at most this many distinct input sets are cycled between steps
+L2_BYTES = 126e6
 
 def time_token_tree(batch, node_cap, dev):
     """clv_build_token_tree for `batch` sequences, 32 speculated sequences of up to 6 tokens each
@@ -244,14 +241,17 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def workload_config(w):
+def workload_config(w, input_sets=None):
     c = w.cfg
+    policy = "not applicable"
+    if input_sets is not None:
+        policy = ("one step's inputs are larger than twice the L2" if input_sets == 1 else
+                  "inputs rotate over %d distinct buffer sets (> 2x L2 in total) between steps" % input_sets)
     return {"workload": "%s: LLaMA3-8B-shaped verify step" % c.name if c.name == "C3" else c.name,
             "batch": c.batch, "n_q_heads": c.n_q_heads, "n_kv_heads": c.n_kv_heads,
             "head_dim": c.head_dim, "ctx_len": (int(w.ctx_len.min()), int(w.ctx_len.max())),
             "tree_nodes": c.n_nodes, "vocab": c.vocab, "paged": bool(c.paged),
-            "cache_policy": "inputs rotate over %d distinct buffer sets (> 2x L2) between steps"
-                            % ROTATE}
+            "cache_policy": policy}
 
 
 def reduce_over_ranks(dist, device, step_ms, e2e_ms, local_bytes):
@@ -268,30 +268,46 @@ def reduce_over_ranks(dist, device, step_ms, e2e_ms, local_bytes):
 
 
 # ----------------------------------------------------------------------------- device arm
-def run_clv(args):
+# Which roof binds the attention of each workload (arithmetic intensity against the machine's
+# ridge): few query rows per kv head leave it to the memory system, 256 rows (C3) sit on the ridge,
+# 512 rows (C5) make it a dense contraction.  The argmax is a pure stream everywhere.
+ATTN_BOUND = {"C1": "hbm", "C2": "hbm", "C3": "hbm", "C4": "hbm", "C5": "tensor"}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from ncu captures of the library whose
+# clv_version() is the first element; a different library version reports null instead
+NCU_TRAFFIC = {}
+MIN_TIMED_MS = 200.0   # the --steps loop is repeated until this much has been timed
+
+
+def all_peaks():
+    """(HBM GB/s, bf16 burst TFLOP/s, bf16 sustained TFLOP/s, 'measured' | 'fallback')."""
+    try:
+        d = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, 1590.0, 1400.0, "fallback"
+
+
+def attention_flops(w):
+    """4 B Hq N (L + N) D: Q K^T and P V over the context and the whole tree tile."""
+    c = w.cfg
+    return float(sum(4.0 * c.n_q_heads * c.n_nodes * (int(L) + c.n_nodes) * c.head_dim for L in w.ctx_len))
+
+
+def measure_workload(name, args, dev, rank, dist, clocks_index, lib_version):
+    """Step time and per-call times of one workload on this rank's GPU (inputs resident, CUDA-graph
+    replay over rotating input sets, CUDA events on the launching stream)."""
+    import dataclasses
     import torch
-    from paper_2408_00264_b200 import binding as clv
     from paper_2408_00264_b200 import workloads as W
     from paper_2408_00264_b200.step import VerifyStep
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    clv.lib()
-
-    import dataclasses
-    cfg = dataclasses.replace(W.CONFIGS[args.workload], seed=W.CONFIGS[args.workload].seed + rank)
+    cfg = dataclasses.replace(W.CONFIGS[name], seed=W.CONFIGS[name].seed + rank)
     w = W.generate(cfg)
-    sets = [VerifyStep(w, device=dev, with_lse=False) for _ in range(ROTATE)]
     nbytes = w.algorithmic_bytes()
+    # enough distinct input sets that their bytes exceed twice the L2, so that every step is cold
+    # (C3: 4 x 138 MB; a workload larger than the L2 needs no second set)
+    rotate = 1 if nbytes["total"] > 2 * L2_BYTES else max(1, min(ROTATE, int(4 * L2_BYTES // nbytes["total"]) + 1))
+    sets = [VerifyStep(w, device=dev, with_lse=False) for _ in range(rotate)]
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -300,51 +316,63 @@ def run_clv(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    # ---- whole step, inputs resident -------------------------------------------------------
-    for i in range(max(args.warmup, 3)):
-        sets[i % ROTATE].run()
+    warm = max(args.warmup, 3)
+    for i in range(warm):
+        sets[i % rotate].run()
     torch.cuda.synchronize()
     graphs = None
     if not args.no_graph:
         graphs = []
-        for s in sets:
+        for st in sets:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                s.run()
+                st.run()
             graphs.append(g)
-        for i in range(max(args.warmup, 3)):
-            graphs[i % ROTATE].replay()
+        for i in range(warm):
+            graphs[i % rotate].replay()
         stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps_ms = []
     barrier()
-    with ClockSampler(local) as clocks:
-        e0.record(stream)
-        if graphs is not None:
+    with ClockSampler(clocks_index) as clocks:
+        total = 0.0
+        while True:   # exactly --steps steps per repeat; repeats until enough has been timed
+            barrier()
+            e0.record(stream)
             for i in range(args.steps):
-                graphs[i % ROTATE].replay()
-        else:
-            for i in range(args.steps):
-                sets[i % ROTATE].run()
-        e1.record(stream)
-        barrier()
-    step_ms = e0.elapsed_time(e1) / args.steps
+                if graphs is not None:
+                    graphs[i % rotate].replay()
+                else:
+                    sets[i % rotate].run()
+            e1.record(stream)
+            barrier()
+            ms = e0.elapsed_time(e1)
+            reps_ms.append(ms / args.steps)
+            total += ms
+            # every rank must take the same number of repeats: the slowest clock decides
+            go = total < MIN_TIMED_MS and len(reps_ms) < 200
+            if dist is not None:
+                t = torch.tensor([1.0 if go else 0.0], device=dev)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                go = bool(t.item() > 0)
+            if not go:
+                break
+    step_ms = statistics.median(reps_ms)
 
-    # ---- each call alone, back to back over the rotating sets (same stream) -----------------
-    def time_call(name, n):
-        """Microseconds per launch of one call, back to back over the rotating input sets.  The
-        launches are replayed from a CUDA graph (one launch per input set) so that host launch
-        overhead does not set the pace of the short kernels."""
+    def time_call(call, n):
+        """Microseconds per launch of one call, back to back over the rotating input sets, replayed
+        from a CUDA graph so that host launch overhead does not set the pace of short kernels."""
         for i in range(3):
-            getattr(sets[i % ROTATE], name)()
+            getattr(sets[i % rotate], call)()
         torch.cuda.synchronize()
         if args.no_graph:
-            run, per = (lambda: [getattr(sets[i], name)() for i in range(ROTATE)]), ROTATE
+            run, per = (lambda: [getattr(sets[i], call)() for i in range(rotate)]), rotate
         else:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                for i in range(ROTATE):
-                    getattr(sets[i], name)()
-            run, per = g.replay, ROTATE
+                for i in range(rotate):
+                    getattr(sets[i], call)()
+            run, per = g.replay, rotate
         run()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         cur = torch.cuda.current_stream()
@@ -357,7 +385,72 @@ def run_clv(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / (reps * per) * 1e3
     n_k = max(20, min(args.steps, 400))
-    call_us = {k: time_call(k, n_k) for k in ("tree_attn", "accept_argmax", "accept_walk", "kv_commit")}
+    call_us = {k: time_call(k, n_k) for k in ("tree_attn", "accept_argmax", "accept_walk", "kv_commit",
+                                              "accept_walk_commit")}
+
+    hbm, tf_burst, tf_sust, kind = all_peaks()
+    flops = attention_flops(w)
+    attn_gbs = nbytes["attn"] / call_us["tree_attn"] / 1e3
+    attn_tf = flops / call_us["tree_attn"] / 1e6
+    arg_gbs = nbytes["logits"] / call_us["accept_argmax"] / 1e3
+    dom = "tree_attn" if call_us["tree_attn"] >= call_us["accept_argmax"] else "accept_argmax"
+    bound = ATTN_BOUND[name] if dom == "tree_attn" else "hbm"
+    traffic = NCU_TRAFFIC.get((lib_version, name, dom))
+    if bound == "tensor":
+        # a kernel of most of a millisecond at the power cap: the sustained rate is its roof
+        roof = {"kernel": dom, "bound": "tensor", "achieved": attn_tf, "peak": tf_sust,
+                "peak_source": kind + " (sustained)", "unit": "TFLOP/s", "frac": attn_tf / tf_sust,
+                "traffic": traffic}
+    else:
+        ach = attn_gbs if dom == "tree_attn" else arg_gbs
+        roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": hbm, "peak_source": kind,
+                "unit": "GB/s", "frac": ach / hbm, "traffic": traffic}
+    res = {
+        "workload": name, "step_us": step_ms * 1e3, "step_us_min": min(reps_ms) * 1e3,
+        "repeats": len(reps_ms), "timed_ms": sum(reps_ms) * args.steps, "input_sets": rotate,
+        "call_us": call_us, "algorithmic_bytes": nbytes, "attention_flops": flops,
+        "step_gbs": nbytes["total"] / (step_ms * 1e-3) / 1e9,
+        "roofline": roof,
+        "attention": {"gbs": attn_gbs, "frac_of_hbm_%s" % kind: attn_gbs / hbm, "tflops": attn_tf,
+                      "frac_of_bf16_burst_%s" % kind: attn_tf / tf_burst,
+                      "frac_of_bf16_sustained_%s" % kind: attn_tf / tf_sust},
+        "argmax": {"gbs": arg_gbs, "frac_of_hbm_%s" % kind: arg_gbs / hbm},
+        "clocks": clocks.summary(),
+    }
+    return w, sets, res, reps_ms, graphs is not None
+
+
+def run_clv(args):
+    import torch
+    from paper_2408_00264_b200 import binding as clv
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if local >= torch.cuda.device_count():
+        raise SystemExit("bench.py: rank %d has no GPU (%d visible)" % (rank, torch.cuda.device_count()))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    L = clv.lib()
+    version = int(L.clv_version())
+
+    w, sets, main_res, reps_ms, graphed = measure_workload(args.workload, args, dev, rank, dist, local, version)
+    nbytes = main_res["algorithmic_bytes"]
+    step_ms = main_res["step_us"] * 1e-3
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
 
     # ---- end to end from pinned host buffers ------------------------------------------------
     c = w.cfg
@@ -404,6 +497,20 @@ def run_clv(args):
         lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
         tree_us = time_token_tree(B, 128, dev)
 
+    # ---- the other stated workloads, one after the other on rank 0's GPU (single-GPU runs) ------
+    others = {}
+    if world == 1 and args.all_workloads:
+        del sets, s0, staging, host
+        torch.cuda.empty_cache()
+        for name in ("C1", "C2", "C3", "C4", "C5"):
+            if name == args.workload:
+                continue
+            o_w, o_sets, o_res, _, _ = measure_workload(name, args, dev, rank, None, local, version)
+            o_res["config"] = workload_config(o_w, o_res["input_sets"])
+            others[name] = o_res
+            del o_w, o_sets
+            torch.cuda.empty_cache()
+
     # ---- max over ranks ------------------------------------------------------------------------
     step_ms, e2e_ms, job_bytes = reduce_over_ranks(dist, dev, step_ms, e2e_ms, float(nbytes["total"]))
     if rank != 0:
@@ -411,32 +518,33 @@ def run_clv(args):
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peaks()
+    hbm, tf_burst, tf_sust, peak_kind = all_peaks()
     value = job_bytes / (step_ms * 1e-3) / 1e9
-    dom = "tree_attn" if call_us["tree_attn"] >= call_us["accept_argmax"] else "accept_argmax"
-    dom_bytes = nbytes["attn"] if dom == "tree_attn" else nbytes["logits"]
-    achieved = dom_bytes / (call_us[dom] * 1e-6) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": workload_config(w),
-        "step_us": step_ms * 1e3,
+        "config": workload_config(w, main_res["input_sets"]),
+        "step_us": step_ms * 1e3, "step_us_min": main_res["step_us_min"], "repeats": main_res["repeats"],
+        "timed_ms": main_res["timed_ms"],
+        "timing": "--steps steps per repeat, repeats until %.0f ms are timed; ms_per_step is the median repeat "
+                  "(max over ranks)" % MIN_TIMED_MS,
         "tree_tokens_per_s": world * B * N / (step_ms * 1e-3),
-        "frac_of_hbm_peak": {"of_%s_%.0f_GBps" % (peak_kind, peak): value / world / peak,
+        "frac_of_hbm_peak": {"of_%s_%.0f_GBps" % (peak_kind, hbm): value / world / hbm,
                              "of_nominal_8000_GBps": value / world / NOMINAL_HBM_GBS},
-        "call_us": call_us, "launch_mode": "per-call" if graphs is None else "cuda-graph replay",
+        "call_us": main_res["call_us"], "launch_mode": "cuda-graph replay" if graphed else "per-call",
         "step_schedule": "clv_tree_attn, clv_accept_argmax, clv_accept_walk_commit (walk and commit in one launch) on one stream",
-        "algorithmic_bytes": nbytes,
-        "roofline": {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC.get((args.workload, dom))},
+        "algorithmic_bytes": nbytes, "attention_flops": main_res["attention_flops"],
+        "roofline": main_res["roofline"],
+        "attention": main_res["attention"], "argmax": main_res["argmax"],
+        "library_version": version,
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
         "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us},
-        "gpu_launches": 3 * args.steps,   # attention, argmax, walk + commit in one launch
-        "clocks": clocks.summary(),
+        "other_workloads": others,
+        "gpu_launches": 3 * args.steps * main_res["repeats"],   # attention, argmax, walk + commit in one launch
+        "clocks": main_res["clocks"],
     }
     if not args.no_cpu_baseline and world == 1:
         import oracle as orc
@@ -449,19 +557,53 @@ def run_clv(args):
         dist.destroy_process_group()
 
 
-def main():
+# ----------------------------------------------------------------------------- ranks
+def rank_env(rank, world, port):
+    """The environment a launcher would give rank `rank` of `world` on this node."""
+    return {"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world),
+            "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)}
+
+
+def _rank_entry(rank, world, port, argv):
+    """One spawned rank: the launcher's environment, then the ordinary main."""
+    os.environ.update(rank_env(rank, world, port))
+    main(argv)
+
+
+def free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def launch_ranks(world, argv, entry=_rank_entry):
+    """`--gpus N` without a launcher: start N processes on this node, one per GPU."""
+    import torch.multiprocessing as mp
+    mp.spawn(entry, args=(world, free_port(), argv), nprocs=world, join=True)
+
+
+def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--impl", default="clv", choices=["clv", "reference"])
-    ap.add_argument("--no-graph", action="store_true", help="launch the four calls per step directly")
+    ap.add_argument("--no-graph", action="store_true", help="launch the calls of a step directly")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lm-head", action="store_true",
                     help="skip the timing of clv_lm_head_argmax (hidden 4096, the workload's rows and vocabulary)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiling runs)")
-    args = ap.parse_args()
+    ap.add_argument("--no-other-workloads", dest="all_workloads", action="store_false",
+                    help="time only --workload (by default a single-GPU run also times the other four)")
+    args = ap.parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        if args.impl == "reference":   # the CPU arm runs on rank 0 alone
+            run_reference(args)
+            return
+        launch_ranks(args.gpus, list(sys.argv[1:] if argv is None else argv))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

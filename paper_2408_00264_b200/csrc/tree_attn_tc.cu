@@ -447,17 +447,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int t = 0; t < NSB && t < T && ok; ++t) ok = issue_qk(t);
       for (int t = 0; t < T && ok; ++t) {
         const int buf = t % NSB, st = t % VST;
-        ok = mbar_wait(bar(B_PF + buf), (t / NSB) & 1, abort_flag, wlim);
-        if (!ok) break;
-        ok = mbar_wait(bar(B_VF + st), (t / VST) & 1, abort_flag, wlim);
+        // both tests are issued together; the bounded waits follow only if one of them fails
+        const bool p_in = mbar_test(bar(B_PF + buf), (t / NSB) & 1);
+        const bool v_in = mbar_test(bar(B_VF + st), (t / VST) & 1);
+        if (!p_in) ok = mbar_wait(bar(B_PF + buf), (t / NSB) & 1, abort_flag, wlim);
+        if (ok && !v_in) ok = mbar_wait(bar(B_VF + st), (t / VST) & 1, abort_flag, wlim);
         if (!ok) break;
         tc_fence_after();
         const int n_kk = min(PPT, pc_end - (pc_begin + t * PPT)) * (PG / 16);   // a missing piece is skipped
         const uint64_t vd = v_desc + (uint64_t)((st * kStage) >> 4);
         // P of piece j of the tile sits in the first 32 columns of that piece's 64 score columns
-        for (int kk = 0; kk < n_kk; ++kk)
-          umma_bf16_ts(tmem_O, tmem_S(buf) + (kk >> 2) * 64 + (kk & 3) * 8, vd + (uint64_t)((kk * 2048) >> 4),
-                     kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+        for (int kk = 0; kk < BN / 16; ++kk)
+          if (kk < n_kk)
+            umma_bf16_ts(tmem_O, tmem_S(buf) + (kk >> 2) * 64 + (kk & 3) * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                         kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
         umma_commit(bar(B_PV + buf));   // O holds tile t
         umma_commit(bar(B_VE + st));    // this V buffer is free
         if (t + NSB < T) ok = issue_qk(t + NSB);

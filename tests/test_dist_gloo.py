@@ -39,3 +39,27 @@ def test_two_ranks_shard_and_reduce():
     gathered, step, e2e, nbytes = out.get()
     assert sorted(gathered[0] + gathered[1]) == list(range(7)) and not set(gathered[0]) & set(gathered[1])
     assert step == 11.0 and e2e == 100.0 and nbytes == 3000.0
+
+
+def test_gpus_flag_without_a_launcher_starts_its_own_ranks(monkeypatch):
+    """`bench.py --gpus N` with no WORLD_SIZE in the environment must start N ranks itself (one per
+    GPU, rendezvous on 127.0.0.1); under a launcher (WORLD_SIZE set) it must not."""
+    import bench
+    calls = []
+    monkeypatch.setattr(bench, "launch_ranks", lambda world, argv: calls.append((world, list(argv))))
+    monkeypatch.setattr(bench, "run_clv", lambda args: calls.append(("run", args.gpus)))
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    bench.main(["--gpus", "4", "--steps", "7"])
+    assert calls == [(4, ["--gpus", "4", "--steps", "7"])]
+    calls.clear()
+    monkeypatch.setenv("WORLD_SIZE", "4")
+    bench.main(["--gpus", "4", "--steps", "7"])
+    assert calls == [("run", 4)]
+    calls.clear()
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    bench.main(["--gpus", "1"])
+    assert calls == [("run", 1)]
+    env = bench.rank_env(2, 4, 29511)
+    assert env == {"RANK": "2", "LOCAL_RANK": "2", "WORLD_SIZE": "4", "MASTER_ADDR": "127.0.0.1",
+                   "MASTER_PORT": "29511"}
+    assert 1024 < bench.free_port() < 65536

@@ -306,6 +306,41 @@ def test_argmax_ties_zeros_and_infinities(clv, oracle):
     assert np.array_equal(st.ids.cpu().numpy(), ref)
 
 
+@pytest.mark.parametrize("rows_b,rows_n,vocab", [(3, 7, 40008), (1, 1, 8), (2, 64, 9000), (5, 3, 2051), (1, 128, 33)])
+def test_argmax_cuts_ties_and_ragged_rows(clv, oracle, rows_b, rows_n, vocab):
+    # A row is scanned in pieces by several blocks, wherever the cuts fall: equal maxima planted far
+    # apart (first index wins), maxima in the ragged last elements of a row (vocab not a multiple
+    # of 8), and a second call on the same workspace.
+    ld = (vocab + 7) // 8 * 8 + 8
+    rng = np.random.default_rng(vocab * 31 + rows_n)
+    rows = rows_b * rows_n
+    lg = np.empty((rows, ld), np.uint16)
+    lg[:] = W.f32_to_bf16_bits(rng.standard_normal((rows, ld)).astype(np.float32))
+    big = int(W.f32_to_bf16_bits(np.array([9.0], np.float32))[0])
+    for r in range(rows):
+        k = r % 4
+        if k == 0:
+            pos = sorted(set(int(x) for x in rng.integers(0, vocab, size=5)))
+            lg[r, pos] = big                      # ties far apart
+        elif k == 1:
+            lg[r, vocab - 1] = big                # the very last (possibly ragged) element
+        elif k == 2:
+            lg[r, max(0, vocab - 3)] = big
+            lg[r, vocab // 2] = big               # tie between the middle and the ragged end
+        # k == 3: plain random row
+    lg[:, vocab:] = 0x7F00                        # huge values in the padding must be ignored
+    shape = clv.make_shape(rows_b, rows_n, 1, 1, vocab, 1)
+    ws = clv.new_workspace(shape, None, 0)
+    d = torch.from_numpy(lg.view(np.int16)).cuda()
+    ids = torch.full((rows_b, rows_n), -5, dtype=torch.int32, device="cuda")
+    ref = oracle.argmax(lg, vocab)
+    for _ in range(2):
+        clv.clv_accept_argmax(shape, d, ld, ids, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(ids.cpu().numpy().reshape(-1), ref)
+        ids.fill_(-5)
+
+
 # ------------------------------------------------------------------ walk and commit
 def test_walk_random_trees_and_errors(clv, oracle):
     rng = np.random.default_rng(5)
