@@ -73,7 +73,8 @@ size_t clv_workspace_bytes(const clv_shape* shape, const clv_kv_cache* cache, in
   (void)cache;
   if (check_shape(shape) != CLV_OK) return 0;
   if (max_ctx_len < 0) max_ctx_len = 0;
-  size_t scratch = tc_attn_plan(*shape, max_ctx_len).scratch_bytes;
+  size_t scratch = (tc2_attn_wanted(*shape) ? tc2_attn_plan(*shape, max_ctx_len)
+                                            : tc_attn_plan(*shape, max_ctx_len)).scratch_bytes;
   if (shape->vocab > 0) {
     const ArgmaxPlan gp = argmax_plan(shape->batch * shape->n_nodes, shape->vocab);
     if (gp.scratch_bytes > scratch) scratch = gp.scratch_bytes;
@@ -104,7 +105,7 @@ static clv_status validate_tree_attn(const clv_shape* shape, const clv_kv_cache*
   if (max_ctx_len < 0) return CLV_ERR_SHAPE;
   if (shape->n_q_heads / shape->n_kv_heads > 128) return CLV_ERR_UNSUPPORTED;
   if (shape->batch > kTickets / 2) return CLV_ERR_UNSUPPORTED;   // two counters per sequence
-  *plan = tc_attn_plan(*shape, max_ctx_len);
+  *plan = tc2_attn_wanted(*shape) ? tc2_attn_plan(*shape, max_ctx_len) : tc_attn_plan(*shape, max_ctx_len);
   if (!workspace || workspace_bytes < kWsFixedBytes + plan->scratch_bytes) return CLV_ERR_WORKSPACE;
   if (!aligned16(workspace)) return CLV_ERR_ALIGN;
   if (!tc_attn_supported(*shape, *cache)) return CLV_ERR_UNSUPPORTED;   // asks the driver: last
@@ -120,9 +121,13 @@ clv_status clv_tree_attn(const clv_shape* shape, const clv_kv_cache* cache, cons
   const clv_status st = validate_tree_attn(shape, cache, q, k_tree, v_tree, parent, ctx_len, max_ctx_len,
                                            out, status, workspace, workspace_bytes, &plan);
   if (st != CLV_OK) return st;
-  cudaError_t e = launch_tree_attn_tc(plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len,
-                                      softmax_scale, out, lse, status, ws_tickets(workspace),
-                                      ws_scratch(workspace), static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = tc2_attn_wanted(*shape)
+                      ? launch_tree_attn_tc2(plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len, softmax_scale,
+                                             out, lse, status, ws_tickets(workspace), ws_scratch(workspace),
+                                             static_cast<cudaStream_t>(cuda_stream))
+                      : launch_tree_attn_tc(plan, *shape, *cache, q, k_tree, v_tree, parent, ctx_len, softmax_scale,
+                                            out, lse, status, ws_tickets(workspace), ws_scratch(workspace),
+                                            static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 

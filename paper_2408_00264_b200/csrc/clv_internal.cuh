@@ -69,6 +69,15 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
                                 cudaStream_t stream);
+// units of four or more row tiles per (sequence, kv head): blocks of two row tiles that share every
+// staged K/V tile (same results, same plan fields; m_tiles counts pairs of row tiles)
+bool tc2_attn_wanted(const clv_shape& s);
+AttnPlan tc2_attn_plan(const clv_shape& s, int max_ctx_len);
+cudaError_t launch_tree_attn_tc2(const AttnPlan& plan, const clv_shape& s, const clv_kv_cache& c,
+                                 const void* q, const void* k_tree, const void* v_tree,
+                                 const int32_t* parent, const int32_t* ctx_len, float scale, void* out,
+                                 float* lse, int32_t* status, unsigned* tickets, void* scratch,
+                                 cudaStream_t stream);
 
 // ---- LM head fused with the argmax (tcgen05 GEMM whose logits stay in tensor memory) ---------------
 bool lm_head_supported(int rows, int hidden, int vocab);

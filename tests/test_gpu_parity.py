@@ -234,13 +234,27 @@ def test_attention_flags_bad_sequences(clv, oracle):
     assert_attn_close(bits(st.out)[0], ref[0], "valid sequence beside bad ones")
 
 
-def test_attention_wait_that_runs_out_is_reported_and_leaves_the_library_usable(clv, oracle):
+@pytest.mark.parametrize("paged", [False, True])
+def test_attention_units_of_many_row_tiles(clv, oracle, paged):
+    # four row tiles per (sequence, kv head) (GQA 4 x 128 nodes = 512 rows): such units are worked
+    # by blocks of two row tiles; ragged contexts, one of them shorter than a key tile, key splits
+    cfg = W.small_config(batch=3, n_q_heads=8, n_kv_heads=2, ctx=(50, 1300), n_nodes=128, vocab=64,
+                         paged=paged, seed=W.BASE_SEED + 512)
+    w = W.generate(cfg)
+    st = make_step(w)
+    st.tree_attn()
+    torch.cuda.synchronize()
+    check_attention(oracle, w, st)
+
+
+@pytest.mark.parametrize("n_nodes", [24, 128])   # one row tile per block / two row tiles per block
+def test_attention_wait_that_runs_out_is_reported_and_leaves_the_library_usable(clv, oracle, n_nodes):
     # Every on-chip wait of the attention kernel is bounded.  With the bound cut to a few dozen SM
     # cycles the ordinary wait for the first tile (a load from device memory takes far longer)
     # runs out: the blocks must leave in order - copies and tensor-core work in flight waited for,
     # tensor memory released - the call itself succeeds, and status[] says CLV_ERR_TIMEOUT.
     # Nothing faults; the next call, on the same workspace, is an ordinary one.
-    cfg = W.small_config(batch=2, n_q_heads=8, n_kv_heads=2, ctx=(300, 700), n_nodes=24, vocab=64,
+    cfg = W.small_config(batch=2, n_q_heads=8, n_kv_heads=2, ctx=(300, 700), n_nodes=n_nodes, vocab=64,
                          seed=W.BASE_SEED + 404)
     w = W.generate(cfg)
     st = make_step(w)
