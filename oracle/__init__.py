@@ -191,6 +191,31 @@ def accept_walk(parent, tokens, ids, path_cap: int):
     return alen, aidx, nxt, status
 
 
+def accept_sample(logits, vocab: int, parent, tokens, uniforms, temperature: float, path_cap: int):
+    """Stochastic acceptance (temperature > 0).  logits: uint16 bf16 bits [B, N, ld]; uniforms:
+    float32 [B, N + 1].  Returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
+    status [B], margin [B]): margin is the smallest distance between a uniform and the threshold it
+    was compared with, over the decisions of the sequence."""
+    lib = _load()
+    lg = _c(logits, np.uint16)
+    parent = _c(parent, np.int32); tokens = _c(tokens, np.int32)
+    uniforms = _c(uniforms, np.float32)
+    B, N = parent.shape
+    assert lg.shape[0] == B and lg.shape[1] == N and uniforms.shape == (B, N + 1)
+    ld = lg.shape[-1]
+    alen = np.empty(B, dtype=np.int32)
+    aidx = np.empty((B, path_cap), dtype=np.int32)
+    nxt = np.empty(B, dtype=np.int32)
+    status = np.empty(B, dtype=np.int32)
+    margin = np.empty(B, dtype=np.float64)
+    rc = lib.orc_accept_sample(ctypes.c_int(B), ctypes.c_int(N), ctypes.c_int(vocab), ctypes.c_int64(ld),
+                               ctypes.c_int(path_cap), _p(lg), _p(parent), _p(tokens), _p(uniforms),
+                               ctypes.c_double(float(temperature)), _p(alen), _p(aidx), _p(nxt), _p(status),
+                               _p(margin))
+    assert rc == 0
+    return alen, aidx, nxt, status, margin
+
+
 def kv_commit(k_cache, v_cache, k_tree, v_tree, accept_idx, accept_len, ctx_len, *,
               block_table=None):
     """Returns (k_cache', v_cache', ctx_len_out, status); the inputs are not modified."""

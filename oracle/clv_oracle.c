@@ -22,6 +22,14 @@
  *   orc_accept_walk   - Sec. 2.1 verification phase (the target filters out wrong drafted
  *                       tokens; the output equals plain decoding) with the greedy rule of the
  *                       tree-sampling algorithm Sec. 4.1 adopts.
+ *   orc_accept_sample - Sec. 4.1 / 4.2 (Table 1, temperature 1): the paper adopts the tree sampling
+ *                       algorithm of its baseline system and prints no formula; this is the
+ *                       speculative-sampling rule for drafts that are proposed deterministically
+ *                       (each child of a node is one proposed token): a child is accepted with its
+ *                       probability under what is left of the target's distribution, a rejected
+ *                       token is struck from it, and when every child is rejected the next token
+ *                       is drawn from the remainder.  The emitted tokens then follow the target's
+ *                       distribution exactly.
  *   orc_kv_commit     - derived from the equivalence requirement of Sec. 2.1: after a step the
  *                       cache holds exactly what plain decoding of the accepted tokens would.
  *
@@ -29,8 +37,11 @@
  * decodes, a float64 library attention with an explicit boolean mask, convex-hull and
  * log-sum-exp identities, mask exactness under perturbation, brute-force path enumeration,
  * numpy's first-occurrence argmax, the commit/append equivalence, and for the LM head a float64
- * library matrix product, a one-hot weight matrix and planted rounding ties.  No function here is
- * "parity unpinned".
+ * library matrix product, a one-hot weight matrix and planted rounding ties; for the stochastic
+ * acceptance the exact outcome probabilities of small trees (computed by a separate recursive
+ * enumeration) against frequencies over many draws, the emitted token's distribution against the
+ * target's softmax, the low-temperature limit against the greedy walk, and certain / impossible
+ * drafts.  No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -316,4 +327,103 @@ int orc_kv_commit(int B, int N, int Hkv, int D, int path_cap, uint16_t *kc, uint
 }
 
 /* Exposed so a test can pin the rounding helper against an independent bf16 conversion. */
+/*
+ * Stochastic acceptance at temperature T > 0.  Node 0 is the root (always accepted).  At the current
+ * node the target's distribution is p = softmax(logits[cur] / T) over the vocabulary.  Its
+ * children are looked at in increasing node index; child c carries token x = tokens[c] and is
+ * accepted if  u[c] < p(x) / (1 - mass of the tokens rejected at this node so far);  an accepted
+ * child becomes the current node (with a fresh distribution).  A rejected token is struck from the
+ * distribution.  When no child is accepted (or there is none), the next token is drawn from what
+ * is left: the first v, in vocabulary order and not struck, whose running sum of p exceeds
+ * u[N] * (1 - rejected mass).  u: [B, N + 1] uniforms in [0, 1) supplied by the caller (u[b][c]
+ * decides child c, u[b][N] draws the next token).  A struck token cannot be proposed again at the
+ * same node (siblings carry distinct tokens; if they do not, the repeat is rejected).
+ * margin[b] receives the smallest |u - threshold| of the decisions taken (accept tests: in
+ * probability units; the final draw: distance of the target to the two running sums that bracket
+ * it, divided by the remaining mass), so that a caller can tell results that rounding cannot
+ * change from those it can.  Malformed trees are reported like orc_accept_walk does.
+ */
+int orc_accept_sample(int B, int N, int vocab, int64_t ld, int path_cap, const uint16_t *logits,
+                      const int32_t *parent, const int32_t *tokens, const float *u, double temperature,
+                      int32_t *accept_len, int32_t *accept_idx, int32_t *next_token, int32_t *status,
+                      double *margin) {
+  double *p = (double *)malloc(sizeof(double) * (size_t)vocab);
+  if (!p) return 1;
+  for (int b = 0; b < B; ++b) {
+    const int32_t *par = parent + (int64_t)b * N, *tok = tokens + (int64_t)b * N;
+    const float *ub = u + (int64_t)b * (N + 1);
+    int32_t *path = accept_idx + (int64_t)b * path_cap;
+    for (int j = 0; j < path_cap; ++j) path[j] = -1;
+    status[b] = ORC_OK;
+    margin[b] = 1.0;
+    int ok = tree_ok(par, N, 0) && path_cap >= 1 && temperature > 0.0;
+    int len = 0, cur = 0, nxt = -1;
+    if (ok) {
+      path[len++] = 0;
+      for (;;) {
+        /* the target's distribution at the current node */
+        const uint16_t *row = logits + ((int64_t)b * N + cur) * ld;
+        double m = -INFINITY, z = 0.0;
+        for (int v = 0; v < vocab; ++v) { double l = bf16_to_f64(row[v]) / temperature; if (l > m) m = l; }
+        for (int v = 0; v < vocab; ++v) { p[v] = exp(bf16_to_f64(row[v]) / temperature - m); z += p[v]; }
+        for (int v = 0; v < vocab; ++v) p[v] /= z;
+        double rejected = 0.0;
+        int found = -1;
+        for (int c = cur + 1; c < N && found < 0; ++c) {
+          if (par[c] != cur) continue;
+          const int x = tok[c];
+          double a = 0.0;
+          if (x >= 0 && x < vocab && rejected < 1.0) a = p[x] / (1.0 - rejected);
+          const double d = fabs((double)ub[c] - a);
+          if (d < margin[b]) margin[b] = d;
+          if ((double)ub[c] < a) {
+            found = c;
+          } else if (x >= 0 && x < vocab) {
+            rejected += p[x];
+            p[x] = 0.0;
+          }
+        }
+        if (found >= 0) {
+          if (len == path_cap) { ok = 0; break; }
+          path[len++] = found;
+          cur = found;
+          continue;
+        }
+        /* every child rejected (or no child): draw from what is left */
+        double left = 0.0;
+        for (int v = 0; v < vocab; ++v) left += p[v];
+        const double target = (double)ub[N] * left;
+        double run = 0.0;
+        nxt = -1;
+        int last = -1;
+        for (int v = 0; v < vocab; ++v) {
+          if (p[v] <= 0.0) continue;
+          last = v;
+          const double before = run;
+          run += p[v];
+          if (run > target) {
+            nxt = v;
+            double d = (target - before < run - target ? target - before : run - target) / left;
+            if (before == 0.0) d = (run - target) / left;   /* nothing below the first candidate */
+            if (d < margin[b]) margin[b] = d;
+            break;
+          }
+        }
+        if (nxt < 0) nxt = last;   /* rounding left the running sum a hair short of the target */
+        break;
+      }
+    }
+    if (!ok) {
+      for (int j = 0; j < path_cap; ++j) path[j] = -1;
+      len = 0;
+      nxt = -1;
+      status[b] = ORC_ERR_TREE;
+    }
+    accept_len[b] = len;
+    next_token[b] = nxt;
+  }
+  free(p);
+  return 0;
+}
+
 uint16_t orc_f64_to_bf16(double d) { return f64_to_bf16(d); }
