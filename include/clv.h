@@ -184,6 +184,39 @@ clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* ca
                                   void* cuda_stream);
 
 /*
+ * Stochastic acceptance at temperature T > 0 (Sec. 4.1 / 4.2, Table 1 "Temperature = 1": the paper
+ * uses its baseline's tree sampling algorithm and prints no formula; the reading taken is
+ * speculative sampling for drafts that are proposed deterministically, one token per child).
+ * For every sequence, starting at the root (always accepted): p = softmax(logits[cur] / T); the
+ * children of the current node are tried in increasing node index, child c with token x being
+ * accepted if  uniforms[b][c] < p(x) / (1 - mass of the tokens rejected at this node so far);
+ * an accepted child becomes current, a rejected token is struck from p.  When every child is
+ * rejected (or there is none), next_token = the first v, in vocabulary order and not struck, whose
+ * running sum of p exceeds uniforms[b][N] * (mass left).  The tokens emitted this way follow the
+ * target's distribution exactly, whatever the drafts.  Use clv_kv_commit on the result as after
+ * clv_accept_walk.
+ * logits: device, bf16 [B*N, ld] as for clv_accept_argmax (no NaN: a precondition; the kernels
+ * give such an entry no probability);
+ * uniforms: device, fp32 [B, N + 1], every value in [0, 1), supplied by the caller (the library
+ * draws no random numbers); temperature: host, finite and > 0.
+ * accept_len / accept_idx / next_token / status: as clv_accept_walk (status CLV_ERR_TREE for a
+ * malformed parent[] or a path longer than path_cap; next_token -1 then, and also for a row
+ * without any probability mass).  Arithmetic: fp32 with hardware exp2; a decision whose uniform
+ * lies within rounding distance of its threshold (relative 1e-5) may fall either way.
+ * workspace: as returned by clv_workspace_bytes for this shape (with vocab set), initialised.
+ * Errors: CLV_ERR_NULL, CLV_ERR_SHAPE (also temperature <= 0), CLV_ERR_ALIGN, CLV_ERR_WORKSPACE.
+ */
+clv_status clv_accept_sample(const clv_shape* shape,
+                             const void* logits, /* bf16 [B*N, ld] */
+                             int64_t ld,
+                             const int32_t* parent, const int32_t* tokens, /* [B, N] */
+                             const float* uniforms,                        /* [B, N + 1] */
+                             float temperature,
+                             int32_t* accept_len, int32_t* accept_idx, int32_t* next_token,
+                             int32_t* status,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * LM head fused with the greedy choice (Sec. 3.1: the target's final norm and LM head produce the
  * logits of every tree node; Sec. 4.2: greedy decoding at temperature 0):
  *   argmax_ids[r] = the lowest v that maximises round_bf16(sum_k hidden[r][k] * weight[v][k]),

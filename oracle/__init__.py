@@ -194,8 +194,9 @@ def accept_walk(parent, tokens, ids, path_cap: int):
 def accept_sample(logits, vocab: int, parent, tokens, uniforms, temperature: float, path_cap: int):
     """Stochastic acceptance (temperature > 0).  logits: uint16 bf16 bits [B, N, ld]; uniforms:
     float32 [B, N + 1].  Returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
-    status [B], margin [B]): margin is the smallest distance between a uniform and the threshold it
-    was compared with, over the decisions of the sequence."""
+    status [B], margin [B, 2]): margin[:, 0] is the smallest distance between a uniform and the
+    probability it was compared with over the accept tests of the sequence, margin[:, 1] the distance
+    of the final draw's target to the nearer running sum around it (as a fraction of the mass left)."""
     lib = _load()
     lg = _c(logits, np.uint16)
     parent = _c(parent, np.int32); tokens = _c(tokens, np.int32)
@@ -207,7 +208,7 @@ def accept_sample(logits, vocab: int, parent, tokens, uniforms, temperature: flo
     aidx = np.empty((B, path_cap), dtype=np.int32)
     nxt = np.empty(B, dtype=np.int32)
     status = np.empty(B, dtype=np.int32)
-    margin = np.empty(B, dtype=np.float64)
+    margin = np.empty((B, 2), dtype=np.float64)
     rc = lib.orc_accept_sample(ctypes.c_int(B), ctypes.c_int(N), ctypes.c_int(vocab), ctypes.c_int64(ld),
                                ctypes.c_int(path_cap), _p(lg), _p(parent), _p(tokens), _p(uniforms),
                                ctypes.c_double(float(temperature)), _p(alen), _p(aidx), _p(nxt), _p(status),

@@ -338,10 +338,11 @@ int orc_kv_commit(int B, int N, int Hkv, int D, int path_cap, uint16_t *kc, uint
  * u[N] * (1 - rejected mass).  u: [B, N + 1] uniforms in [0, 1) supplied by the caller (u[b][c]
  * decides child c, u[b][N] draws the next token).  A struck token cannot be proposed again at the
  * same node (siblings carry distinct tokens; if they do not, the repeat is rejected).
- * margin[b] receives the smallest |u - threshold| of the decisions taken (accept tests: in
- * probability units; the final draw: distance of the target to the two running sums that bracket
- * it, divided by the remaining mass), so that a caller can tell results that rounding cannot
- * change from those it can.  Malformed trees are reported like orc_accept_walk does.
+ * margin[b][0] receives the smallest |u - threshold| over the accept tests of the sequence (in
+ * probability units), margin[b][1] the distance of the final draw's target to the nearer of the
+ * two running sums that bracket it, divided by the remaining mass, so that a caller can tell
+ * results that rounding cannot change from those it can.  Malformed trees are reported like
+ * orc_accept_walk does.
  */
 int orc_accept_sample(int B, int N, int vocab, int64_t ld, int path_cap, const uint16_t *logits,
                       const int32_t *parent, const int32_t *tokens, const float *u, double temperature,
@@ -355,7 +356,8 @@ int orc_accept_sample(int B, int N, int vocab, int64_t ld, int path_cap, const u
     int32_t *path = accept_idx + (int64_t)b * path_cap;
     for (int j = 0; j < path_cap; ++j) path[j] = -1;
     status[b] = ORC_OK;
-    margin[b] = 1.0;
+    margin[2 * b] = 1.0;
+    margin[2 * b + 1] = 1.0;
     int ok = tree_ok(par, N, 0) && path_cap >= 1 && temperature > 0.0;
     int len = 0, cur = 0, nxt = -1;
     if (ok) {
@@ -375,7 +377,7 @@ int orc_accept_sample(int B, int N, int vocab, int64_t ld, int path_cap, const u
           double a = 0.0;
           if (x >= 0 && x < vocab && rejected < 1.0) a = p[x] / (1.0 - rejected);
           const double d = fabs((double)ub[c] - a);
-          if (d < margin[b]) margin[b] = d;
+          if (d < margin[2 * b]) margin[2 * b] = d;
           if ((double)ub[c] < a) {
             found = c;
           } else if (x >= 0 && x < vocab) {
@@ -405,7 +407,7 @@ int orc_accept_sample(int B, int N, int vocab, int64_t ld, int path_cap, const u
             nxt = v;
             double d = (target - before < run - target ? target - before : run - target) / left;
             if (before == 0.0) d = (run - target) / left;   /* nothing below the first candidate */
-            if (d < margin[b]) margin[b] = d;
+            if (d < margin[2 * b + 1]) margin[2 * b + 1] = d;
             break;
           }
         }

@@ -24,7 +24,7 @@ EXPORTS = (
     "clv_workspace_bytes", "clv_workspace_init", "clv_tree_attn", "clv_accept_argmax",
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
-    "clv_lm_head_argmax", "clv_build_token_tree", "clv_accept_walk_commit",
+    "clv_lm_head_argmax", "clv_build_token_tree", "clv_accept_walk_commit", "clv_accept_sample",
     "clv_test_set_wait_limit",
 )
 
@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.clv_lm_head_argmax.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp]
         L.clv_accept_walk_commit.restype = i32
         L.clv_accept_walk_commit.argtypes = [vp] * 15
+        L.clv_accept_sample.restype = i32
+        L.clv_accept_sample.argtypes = [vp, vp, i64, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, vp]
         L.clv_build_token_tree.restype = i32
         L.clv_build_token_tree.argtypes = [i32, i32, i32, i32] + [vp] * 9
         L.clv_accept_walk.restype = i32
@@ -205,6 +207,18 @@ def clv_accept_walk_commit(shape, cache, parent, tokens, argmax_ids, k_tree, v_t
                                         _stream(stream))
     if check:
         _check(code, "clv_accept_walk_commit")
+    return code
+
+
+def clv_accept_sample(shape, logits, ld, parent, tokens, uniforms, temperature, accept_len, accept_idx,
+                      next_token, status, workspace, stream=None, check=True) -> int:
+    """uniforms: float32 [B, N + 1] in [0, 1); temperature: python float > 0."""
+    code = lib().clv_accept_sample(_ref(shape), _ptr(logits), int(ld), _ptr(parent), _ptr(tokens),
+                                   _ptr(uniforms), float(temperature), _ptr(accept_len), _ptr(accept_idx),
+                                   _ptr(next_token), _ptr(status), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream(stream))
+    if check:
+        _check(code, "clv_accept_sample")
     return code
 
 

@@ -1,5 +1,6 @@
 // C ABI of libclv: argument checks and dispatch.  No device memory is allocated here, nothing
 // synchronises, every launch goes to the caller's stream.
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -78,6 +79,8 @@ size_t clv_workspace_bytes(const clv_shape* shape, const clv_kv_cache* cache, in
   if (shape->vocab > 0) {
     const ArgmaxPlan gp = argmax_plan(shape->batch * shape->n_nodes, shape->vocab);
     if (gp.scratch_bytes > scratch) scratch = gp.scratch_bytes;
+    const size_t sb = sample_scratch_bytes(shape->batch * shape->n_nodes, shape->vocab);
+    if (sb > scratch) scratch = sb;
   }
   return kWsFixedBytes + round_up(scratch, 256);
 }
@@ -219,6 +222,28 @@ clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* ca
   cudaError_t e = launch_walk_commit(*shape, *cache, parent, tokens, argmax_ids, k_tree, v_tree, ctx_len,
                                      accept_len, accept_idx, next_token, ctx_len_out, walk_status,
                                      commit_status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+clv_status clv_accept_sample(const clv_shape* shape, const void* logits, int64_t ld, const int32_t* parent,
+                             const int32_t* tokens, const float* uniforms, float temperature,
+                             int32_t* accept_len, int32_t* accept_idx, int32_t* next_token, int32_t* status,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  if (!logits || !parent || !tokens || !uniforms || !accept_len || !accept_idx || !next_token || !status)
+    return CLV_ERR_NULL;
+  if (shape->vocab < 1 || ld < shape->vocab || shape->path_cap < 1) return CLV_ERR_SHAPE;
+  if (!(temperature > 0.0f) || !(temperature < INFINITY)) return CLV_ERR_SHAPE;
+  if (!aligned16(logits) || (ld % 8) != 0) return CLV_ERR_ALIGN;
+  const int64_t rows = (int64_t)shape->batch * shape->n_nodes;
+  if (rows > INT32_MAX / 64) return CLV_ERR_UNSUPPORTED;
+  const size_t need = kWsFixedBytes + sample_scratch_bytes((int)rows, shape->vocab);
+  if (!workspace || workspace_bytes < need) return CLV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  cudaError_t e = launch_accept_sample(*shape, logits, ld, parent, tokens, uniforms, temperature, accept_len,
+                                       accept_idx, next_token, status, ws_scratch(workspace),
+                                       static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 

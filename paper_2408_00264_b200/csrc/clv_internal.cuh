@@ -40,6 +40,13 @@ bool argmax_static_fits(int rows, int vocab);
 cudaError_t launch_argmax_static(const void* logits, int64_t ld, int rows, int vocab, int32_t* ids,
                                  cudaStream_t stream);
 
+// ---- stochastic acceptance (temperature > 0): statistics pass over the logits + per-sequence walk
+size_t sample_scratch_bytes(int rows, int vocab);
+cudaError_t launch_accept_sample(const clv_shape& s, const void* logits, int64_t ld, const int32_t* parent,
+                                 const int32_t* tokens, const float* uniforms, float temperature,
+                                 int32_t* accept_len, int32_t* accept_idx, int32_t* next_token, int32_t* status,
+                                 void* scratch, cudaStream_t stream);
+
 // ---- walk / commit ----------------------------------------------------------------------------
 cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
                         const int32_t* ids, int32_t* accept_len, int32_t* accept_idx,

@@ -294,6 +294,14 @@ def make_candidates(batch: int, n_cand: int, max_len: int, vocab: int, seed: int
     return root, cand, lens
 
 
+def make_uniforms(batch: int, n_nodes: int, seed: int) -> np.ndarray:
+    """Uniform numbers in [0, 1) for the stochastic acceptance: float32 [batch, n_nodes + 1] (entry
+    c decides drafted node c, the last one draws the next token).  Multiples of 2^-24, so that the
+    float32 value is exactly what a float64 reader sees."""
+    rng = np.random.default_rng(seed)
+    return (rng.integers(0, 1 << 24, size=(batch, n_nodes + 1)).astype(np.float64) / float(1 << 24)).astype(np.float32)
+
+
 def make_lm_head(rows: int, hidden_dim: int, vocab: int, seed: int, planted: float = 12.0):
     """Inputs of the LM head for ``rows`` tree nodes: hidden states N(0,1) and a weight matrix
     N(0, 1/hidden_dim) (so that logits are about N(0,1)), both rounded to bf16 and returned as bit

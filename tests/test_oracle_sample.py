@@ -127,9 +127,9 @@ def test_certain_and_impossible_drafts_and_the_final_draw():
     lg3[0, :, 2:vocab] = 0xFF80                              # two tokens of probability 1/2 each
     par, tok = np.array([[-1, 0]], np.int32), np.array([[0, 1]], np.int32)
     a, _, nx, _, mg = oracle.accept_sample(lg3, vocab, par, tok, np.array([[0, 0.5, 0.3]], np.float32), 1.0, 2)
-    assert a.tolist() == [1] and nx.tolist() == [0] and mg[0] == 0.0
+    assert a.tolist() == [1] and nx.tolist() == [0] and mg[0, 0] == 0.0
     a, _, _, _, mg = oracle.accept_sample(lg3, vocab, par, tok, np.array([[0, 0.4990, 0.3]], np.float32), 1.0, 2)
-    assert a.tolist() == [2] and abs(mg[0] - 0.001) < 1e-6
+    assert a.tolist() == [2] and abs(mg[0, 0] - 0.001) < 1e-6
 
 
 def test_rejected_tokens_are_struck_before_the_next_sibling():
