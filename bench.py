@@ -64,6 +64,46 @@ def time_token_tree(batch, node_cap, dev):
             "us": a.elapsed_time(b) / 160 * 1e3, "nodes": outs[2].cpu().tolist()[:4]}
 
 
+def time_accept_sample(w, dev):
+    """clv_accept_sample (temperature 1) on the workload's logits and trees: microseconds per call
+    (two launches: the statistics pass streams every logit once, then one block per sequence walks),
+    replayed from a CUDA graph over two copies of the logits."""
+    import torch
+    from paper_2408_00264_b200 import binding as clv
+    from paper_2408_00264_b200 import workloads as W
+    c = w.cfg
+    B, N = c.batch, c.n_nodes
+    shape = clv.make_shape(B, N, c.n_q_heads, c.n_kv_heads, c.vocab, w.path_cap)
+    ws = clv.new_workspace(shape, None, 0, dev)
+    lg = [torch.from_numpy(w.logits.view(np.int16)).to(dev)]
+    lg.append(lg[0].clone())
+    t = lambda a: torch.from_numpy(a).to(dev)  # noqa: E731
+    parent, tokens, u = t(w.parent), t(w.tokens), t(W.make_uniforms(B, N, seed=W.BASE_SEED + 3))
+    i32 = dict(dtype=torch.int32, device=dev)
+    outs = [torch.zeros(B, **i32), torch.zeros(B, w.path_cap, **i32), torch.zeros(B, **i32), torch.zeros(B, **i32)]
+    call = lambda i: clv.clv_accept_sample(shape, lg[i], w.logits.shape[-1], parent, tokens, u, 1.0, *outs, ws)  # noqa: E731
+    for i in range(4):
+        call(i % 2)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(2):
+            call(i)
+    g.replay()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    a.record(cur)
+    for _ in range(20):
+        g.replay()
+    b.record(cur)
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) / 40 * 1e3
+    nbytes = B * N * c.vocab * 2
+    return {"batch": B, "n_nodes": N, "vocab": c.vocab, "temperature": 1.0, "us": us, "launches_per_call": 2,
+            "accept_len": outs[0].cpu().tolist()[:8], "logits_bytes": nbytes, "gbs_of_logits_stream": nbytes / us / 1e3}
+
+
 def time_lm_head(rows, hidden, vocab, dev, args):
     """clv_lm_head_argmax on `rows` tree nodes: microseconds per launch (CUDA events, launches
     replayed from a CUDA graph over two copies of the weight matrix, 2 x 1.05 GB at vocabulary
@@ -493,9 +533,11 @@ def run_clv(args):
     # ---- the step before the argmax: LM head fused with the greedy choice (rank 0 only) ---------
     lm_head = None
     tree_us = None
+    sample_us = None
     if rank == 0 and not args.no_lm_head:
         lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
         tree_us = time_token_tree(B, 128, dev)
+        sample_us = time_accept_sample(w, dev)
 
     # ---- the other stated workloads, one after the other on rank 0's GPU (single-GPU runs) ------
     others = {}
@@ -541,7 +583,7 @@ def run_clv(args):
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
-        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us},
+        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us, "accept_sample": sample_us},
         "other_workloads": others,
         "gpu_launches": 3 * args.steps * main_res["repeats"],   # attention, argmax, walk + commit in one launch
         "clocks": main_res["clocks"],

@@ -14,7 +14,7 @@
 // update, in base-2 units.  (2) One block per sequence walks the tree: per level it combines the
 // pieces of the current row, fetches the logits of all children's tokens at once (one round trip
 // to memory), and one thread runs the accept chain; the final draw sums 256 slices of the row,
-// locates the slice by a running sum and walks that slice.
+// locates the slice by a running sum and then scans that slice with the whole block.
 #include <limits.h>
 #include <math.h>
 
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
   __shared__ float su[CLV_MAX_NODES + 1], se[CLV_MAX_NODES];
   __shared__ float s_slice[kThreads];
   __shared__ float s_m, s_S, s_before, s_target;
-  __shared__ int s_found, s_bad, s_pick;
+  __shared__ int s_found, s_bad, s_pick, s_lastv;
   const int b = blockIdx.x, tid = threadIdx.x, N = p.N;
   const int64_t o = (int64_t)b * N;
   cudaGridDependencySynchronize();
@@ -215,39 +215,38 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
     const uint16_t* row = p.logits + (o + cur) * p.ld;
     const int per = ((p.vocab + kThreads - 1) / kThreads + 7) & ~7;
     const int v0 = min(p.vocab, tid * per), v1 = min(p.vocab, v0 + per);
-    // struck tokens inside this slice (usually none)
-    int struck[8];
-    int n_struck = 0;
-    bool many = false;
-    for (int c = cur + 1; c < N; ++c)
-      if (sp[c] == cur && st[c] >= v0 && st[c] < v1) {
-        if (n_struck < 8) struck[n_struck++] = st[c]; else many = true;
-      }
-    auto is_struck = [&](int v) -> bool {
-      for (int j = 0; j < n_struck; ++j) if (struck[j] == v) return true;
-      if (many) for (int c = cur + 1; c < N; ++c) if (sp[c] == cur && st[c] == v) return true;
-      return false;
-    };
     auto weight = [&](int v) -> float {
       const float l = __uint_as_float((uint32_t)row[v] << 16) * p.k;
       return (l == l && m > -INFINITY) ? ex2(l - m) : 0.f;
     };
+    // the slice's sum with 16-byte reads, four in flight (v0 is a multiple of 8, rows are 16-byte
+    // aligned); the weights of struck tokens inside the slice are taken out again afterwards
     float sum = 0.f;
-    if (n_struck == 0 && !many) {
+    {
       int v = v0;
-      for (; v + 8 <= v1; v += 8) {   // 16-byte reads (v0 is a multiple of 8, rows are 16-byte aligned)
-        const uint4 w = *reinterpret_cast<const uint4*>(row + v);
-        const float x[8] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y),
-                            bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w)};
+      for (; v + 32 <= v1; v += 32) {
+        uint4 w[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float l = x[j] * p.k;
-          sum += (l == l && m > -INFINITY) ? ex2(l - m) : 0.f;
+        for (int q = 0; q < 4; ++q) w[q] = *reinterpret_cast<const uint4*>(row + v + 8 * q);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float x[8] = {bf16_lo(w[q].x), bf16_hi(w[q].x), bf16_lo(w[q].y), bf16_hi(w[q].y),
+                              bf16_lo(w[q].z), bf16_hi(w[q].z), bf16_lo(w[q].w), bf16_hi(w[q].w)};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float l = x[j] * p.k;
+            sum += (l == l && m > -INFINITY) ? ex2(l - m) : 0.f;
+          }
         }
       }
       for (; v < v1; ++v) sum += weight(v);
-    } else {
-      for (int v = v0; v < v1; ++v) sum += is_struck(v) ? 0.f : weight(v);
+      for (int c = cur + 1; c < N; ++c) {
+        if (sp[c] != cur || st[c] < v0 || st[c] >= v1) continue;
+        bool repeat = false;   // a token carried by two siblings is struck once
+        for (int d = cur + 1; d < c; ++d) repeat |= (sp[d] == cur && st[d] == st[c]);
+        if (!repeat) sum -= weight(st[c]);
+      }
+      sum = fmaxf(sum, 0.f);
     }
     s_slice[tid] = sum;
     __syncthreads();
@@ -270,23 +269,50 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
       }
       s_pick = pick;
       s_target = target;
+      s_found = INT_MAX;   // first element of the slice whose running sum exceeds the target
+      s_lastv = -1;        // last element of the slice that carries any weight
     }
     __syncthreads();
-    if (s_pick >= 0 && tid == s_pick) {
+    const int pick = s_pick;
+    if (pick >= 0) {
+      // ---- the whole block walks the chosen slice, 256 elements at a time: weights, a running sum
+      //      across the block (warp scans + the warps' totals), the first element past the target
       const float target = s_target;
-      float run = s_before;
-      int next = -1, lastv = -1;
-      for (int v = v0; v < v1; ++v) {
-        if (is_struck(v)) continue;
-        const float e = weight(v);
-        if (e <= 0.f) continue;
-        lastv = v;
-        run += e;
-        if (run > target) { next = v; break; }
+      const int q0 = min(p.vocab, pick * per), q1 = min(p.vocab, q0 + per);
+      const int lane = tid & 31, warp = tid >> 5;
+      float before = s_before;
+      for (int base = q0; base < q1; base += kThreads) {
+        const int v = base + tid;
+        float e = 0.f;
+        if (v < q1) {
+          bool hit = false;
+          for (int c = cur + 1; c < N; ++c) hit |= (sp[c] == cur && st[c] == v);
+          e = hit ? 0.f : weight(v);
+        }
+        float incl = e;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const float up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+          if (lane >= off) incl += up;
+        }
+        if (lane == 31) s_slice[warp] = incl;
+        __syncthreads();
+        float wbase = before;
+        for (int w = 0; w < warp; ++w) wbase += s_slice[w];
+        float round_total = 0.f;
+        for (int w = 0; w < kThreads / 32; ++w) round_total += s_slice[w];
+        if (e > 0.f) {
+          atomicMax(&s_lastv, v);
+          if (wbase + incl > target) atomicMin(&s_found, v);
+        }
+        __syncthreads();
+        if (s_found != INT_MAX) break;   // same verdict in every thread
+        before += round_total;
       }
-      p.next_token[b] = next >= 0 ? next : lastv;
+      if (tid == 0) p.next_token[b] = (s_found != INT_MAX) ? s_found : s_lastv;
+    } else if (tid == 0) {
+      p.next_token[b] = -1;   // a row without any mass
     }
-    if (s_pick < 0 && tid == 0) p.next_token[b] = -1;   // a row without any mass
   }
   __syncthreads();
   if (bad) len = 0;
