@@ -176,6 +176,76 @@ def build_token_tree(root_token, cand, cand_len, node_cap: int):
     return tokens, parent, n_nodes, node_of, status
 
 
+def tree_to_intervals(parent):
+    """Compressed (linear) form of the tree mask (App. A.1: "a numerical comparison" instead of an
+    N x N matrix; the figure is missing, the encoding taken is depth-first entry/exit labels): tin
+    = position of the node in a depth-first walk that visits children in increasing node index
+    (several roots: one after the other), tout = tin + size of the node's subtree.  Then j is an
+    ancestor of i, or i itself, exactly if tin[j] <= tin[i] < tout[j].  Written as a recursive
+    walk.  Returns tin, tout [B, N], status [B] (7 for a malformed parent[], labels -1)."""
+    parent = np.asarray(parent, dtype=np.int32)
+    B, N = parent.shape
+    tin = np.full((B, N), -1, np.int32)
+    tout = np.full((B, N), -1, np.int32)
+    status = np.zeros(B, np.int32)
+    for b in range(B):
+        par = parent[b]
+        if any(par[i] < -1 or par[i] >= i for i in range(N)):
+            status[b] = 7
+            continue
+        kids = [[] for _ in range(N)]
+        roots = []
+        for i in range(N):
+            (roots if par[i] < 0 else kids[par[i]]).append(i)
+        clock = [0]
+
+        def visit(v):
+            tin[b, v] = clock[0]
+            clock[0] += 1
+            for c in kids[v]:
+                visit(c)
+            tout[b, v] = clock[0]
+        for r in roots:
+            visit(r)
+    return tin, tout, status
+
+
+def tree_from_intervals(tin, tout):
+    """parent[] from depth-first labels: the parent of i is the node j != i whose interval
+    [tin[j], tout[j]) contains tin[i] and is the narrowest such interval; -1 if there is none.
+    Status 7 (parent all -1) if the labels are not those of a forest in topological node order:
+    an empty interval, two nodes with the same tin, intervals that overlap without nesting, or a
+    parent that does not come before its child."""
+    tin = np.asarray(tin, dtype=np.int64)
+    tout = np.asarray(tout, dtype=np.int64)
+    B, N = tin.shape
+    parent = np.full((B, N), -1, np.int32)
+    status = np.zeros(B, np.int32)
+    for b in range(B):
+        ok = all(tout[b, i] > tin[b, i] for i in range(N)) and len(set(tin[b].tolist())) == N
+        for i in range(N):
+            for j in range(N):
+                if not ok or i == j:
+                    continue
+                a0, a1, b0, b1 = tin[b, i], tout[b, i], tin[b, j], tout[b, j]
+                if a0 < b0 < a1 < b1:          # overlap without nesting
+                    ok = False
+        if ok:
+            for i in range(N):
+                best = -1
+                for j in range(N):
+                    if j != i and tin[b, j] <= tin[b, i] < tout[b, j]:
+                        if best < 0 or tout[b, j] - tin[b, j] < tout[b, best] - tin[b, best]:
+                            best = j
+                if best >= i:
+                    ok = False
+                parent[b, i] = best
+        if not ok:
+            parent[b] = -1
+            status[b] = 7
+    return parent, status
+
+
 def accept_walk(parent, tokens, ids, path_cap: int):
     """Greedy acceptance walk; returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
     status [B])."""

@@ -19,6 +19,9 @@
  *                       greedy choice, the logit held in bf16 like a logits tensor.
  *   build_token_tree (in the Python wrapper, plain loops over a dictionary) - Sec. 2.1 and the
  *                       caption of Fig. 2: speculations merged by prefix matching into a tree.
+ *   tree_to_intervals / tree_from_intervals (in the Python wrapper, a recursive walk and plain
+ *                       loops) - App. A.1: the compressed, linear form of the tree mask, taken
+ *                       as depth-first entry/exit labels.
  *   orc_accept_walk   - Sec. 2.1 verification phase (the target filters out wrong drafted
  *                       tokens; the output equals plain decoding) with the greedy rule of the
  *                       tree-sampling algorithm Sec. 4.1 adopts.
