@@ -104,6 +104,41 @@ def time_accept_sample(w, dev):
             "accept_len": outs[0].cpu().tolist()[:8], "logits_bytes": nbytes, "gbs_of_logits_stream": nbytes / us / 1e3}
 
 
+def time_model_step(w, n_layers, dev):
+    """Whole-model verify step on the workload's shape: clv_tree_attn per layer (each layer its own
+    Q, tree K/V and cache), clv_lm_head_argmax (hidden 4096), walk, one commit for all layers; one
+    CUDA graph, replayed.  With 32 layers of C3 the caches alone are 2.1 GB, so every launch is cold."""
+    import torch
+    from paper_2408_00264_b200 import workloads as W
+    from paper_2408_00264_b200.step import ModelVerifyStep
+    c = w.cfg
+    layers = W.layer_tensors(w, n_layers)
+    h, wt, _ = W.make_lm_head(c.batch * c.n_nodes, 4096, c.vocab, seed=W.BASE_SEED + 78)
+    st = ModelVerifyStep(w, layers, h, wt, device=dev)
+    for _ in range(2):
+        st.run()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        st.run()
+    g.replay()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    reps = 10
+    a.record(cur)
+    for _ in range(reps):
+        g.replay()
+    b.record(cur)
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) / reps * 1e3
+    nb = w.algorithmic_bytes()
+    total = n_layers * nb["attn"] + (c.vocab + c.batch * c.n_nodes) * 4096 * 2
+    return {"layers": n_layers, "us": us, "launches": n_layers + 3, "status_max": int(st.status.max().item()),
+            "accept_len": st.accept_len.cpu().tolist()[:8], "algorithmic_bytes": total,
+            "gbs": total / us / 1e3}
+
+
 def time_lm_head(rows, hidden, vocab, dev, args):
     """clv_lm_head_argmax on `rows` tree nodes: microseconds per launch (CUDA events, launches
     replayed from a CUDA graph over two copies of the weight matrix, 2 x 1.05 GB at vocabulary
@@ -539,10 +574,12 @@ def run_clv(args):
     lm_head = None
     tree_us = None
     sample_us = None
+    model_us = None
     if rank == 0 and not args.no_lm_head:
         lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
         tree_us = time_token_tree(B, 128, dev)
         sample_us = time_accept_sample(w, dev)
+        model_us = time_model_step(w, 32, dev) if args.workload in ("C1", "C2", "C3") else None
 
     # ---- the other stated workloads, one after the other on rank 0's GPU (single-GPU runs) ------
     others = {}
@@ -588,7 +625,7 @@ def run_clv(args):
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
-        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us, "accept_sample": sample_us},
+        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us, "accept_sample": sample_us, "model_step": model_us},
         "other_workloads": others,
         "gpu_launches": 3 * args.steps * main_res["repeats"],   # attention, argmax, walk + commit in one launch
         "clocks": main_res["clocks"],

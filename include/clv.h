@@ -217,6 +217,43 @@ clv_status clv_accept_sample(const clv_shape* shape,
                              void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The compressed, linear form of the tree mask (App. A.1: a mask that is a numerical comparison
+ * instead of an N x N matrix; the figure is missing, the encoding taken is depth-first entry/exit
+ * labels).  tin[b][i] = position of node i in a depth-first walk of the tree that visits children
+ * in increasing node index (several roots one after the other), tout = tin + size of the node's
+ * subtree; node j is an ancestor of node i, or i itself, exactly if tin[j] <= tin[i] < tout[j].
+ * clv_tree_to_intervals writes the labels of parent[]; clv_tree_from_intervals gives parent[]
+ * back from any labels that nest properly (parent of i = the node with the narrowest interval
+ * around tin[i]), so that a caller holding labels can feed clv_tree_attn, the walk and the commit.
+ * All arrays: device, int32 [B, N], N <= 128.  status[b] = CLV_ERR_TREE (outputs of that sequence
+ * all -1) for a malformed parent[] (parent[i] >= i or < -1), or for labels that are not those of a
+ * forest in topological node order: an empty interval, two equal tin, intervals that overlap
+ * without nesting, a parent that would not come before its child.
+ */
+clv_status clv_tree_to_intervals(int32_t batch, int32_t n_nodes, const int32_t* parent,
+                                 int32_t* tin, int32_t* tout, int32_t* status, void* cuda_stream);
+clv_status clv_tree_from_intervals(int32_t batch, int32_t n_nodes, const int32_t* tin, const int32_t* tout,
+                                   int32_t* parent, int32_t* status, void* cuda_stream);
+
+/*
+ * clv_kv_commit for all layers of a model in one launch (Sec. 2.1: attention is the only block
+ * with a sequence dependency, so a verify step runs clv_tree_attn once per layer and can defer the
+ * commit of every layer's accepted rows to the end of the step).  Layer l's cache buffers start
+ * cache_layer_stride elements (bf16) after layer l-1's - `cache` describes layer 0 -, its tree
+ * K/V tree_layer_stride elements after layer l-1's; all layers share accept_idx / accept_len,
+ * ctx_len and, for a paged cache, the block table.  Results per layer are those of clv_kv_commit;
+ * status and ctx_len_out are written once per sequence (the same for every layer).  Both strides
+ * must be multiples of 8 and at least the size of one layer's buffer; ctx_len_out must not alias
+ * ctx_len here (CLV_ERR_UNSUPPORTED), nor may tree and cache buffers overlap.
+ */
+clv_status clv_kv_commit_layers(const clv_shape* shape, const clv_kv_cache* cache, int32_t n_layers,
+                                int64_t cache_layer_stride,
+                                const void* k_tree, const void* v_tree, int64_t tree_layer_stride,
+                                const int32_t* accept_idx, const int32_t* accept_len,
+                                const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status,
+                                void* cuda_stream);
+
+/*
  * LM head fused with the greedy choice (Sec. 3.1: the target's final norm and LM head produce the
  * logits of every tree node; Sec. 4.2: greedy decoding at temperature 0):
  *   argmax_ids[r] = the lowest v that maximises round_bf16(sum_k hidden[r][k] * weight[v][k]),

@@ -25,6 +25,7 @@ EXPORTS = (
     "clv_accept_walk", "clv_kv_commit", "clv_staging_bytes", "clv_verify_step_host",
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
     "clv_lm_head_argmax", "clv_build_token_tree", "clv_accept_walk_commit", "clv_accept_sample",
+    "clv_tree_to_intervals", "clv_tree_from_intervals", "clv_kv_commit_layers",
     "clv_test_set_wait_limit",
 )
 
@@ -92,6 +93,12 @@ def lib() -> ctypes.CDLL:
         L.clv_lm_head_argmax.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp]
         L.clv_accept_walk_commit.restype = i32
         L.clv_accept_walk_commit.argtypes = [vp] * 15
+        L.clv_tree_to_intervals.restype = i32
+        L.clv_tree_to_intervals.argtypes = [i32, i32, vp, vp, vp, vp, vp]
+        L.clv_tree_from_intervals.restype = i32
+        L.clv_tree_from_intervals.argtypes = [i32, i32, vp, vp, vp, vp, vp]
+        L.clv_kv_commit_layers.restype = i32
+        L.clv_kv_commit_layers.argtypes = [vp, vp, i32, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp]
         L.clv_accept_sample.restype = i32
         L.clv_accept_sample.argtypes = [vp, vp, i64, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, vp]
         L.clv_build_token_tree.restype = i32
@@ -219,6 +226,37 @@ def clv_accept_sample(shape, logits, ld, parent, tokens, uniforms, temperature, 
                                    workspace.numel() * workspace.element_size(), _stream(stream))
     if check:
         _check(code, "clv_accept_sample")
+    return code
+
+
+def clv_tree_to_intervals(parent, tin, tout, status, stream=None, check=True) -> int:
+    """parent, tin, tout: int32 [B, N]; status int32 [B]."""
+    B, N = parent.shape
+    code = lib().clv_tree_to_intervals(int(B), int(N), _ptr(parent), _ptr(tin), _ptr(tout), _ptr(status),
+                                       _stream(stream))
+    if check:
+        _check(code, "clv_tree_to_intervals")
+    return code
+
+
+def clv_tree_from_intervals(tin, tout, parent, status, stream=None, check=True) -> int:
+    B, N = tin.shape
+    code = lib().clv_tree_from_intervals(int(B), int(N), _ptr(tin), _ptr(tout), _ptr(parent), _ptr(status),
+                                         _stream(stream))
+    if check:
+        _check(code, "clv_tree_from_intervals")
+    return code
+
+
+def clv_kv_commit_layers(shape, cache, n_layers, cache_layer_stride, k_tree, v_tree, tree_layer_stride,
+                         accept_idx, accept_len, ctx_len, ctx_len_out, status, stream=None, check=True) -> int:
+    """cache: descriptor of layer 0; the strides are in bf16 elements between consecutive layers."""
+    code = lib().clv_kv_commit_layers(_ref(shape), _ref(cache), int(n_layers), int(cache_layer_stride),
+                                      _ptr(k_tree), _ptr(v_tree), int(tree_layer_stride), _ptr(accept_idx),
+                                      _ptr(accept_len), _ptr(ctx_len), _ptr(ctx_len_out), _ptr(status),
+                                      _stream(stream))
+    if check:
+        _check(code, "clv_kv_commit_layers")
     return code
 
 

@@ -247,6 +247,55 @@ clv_status clv_accept_sample(const clv_shape* shape, const void* logits, int64_t
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
+clv_status clv_tree_to_intervals(int32_t batch, int32_t n_nodes, const int32_t* parent, int32_t* tin,
+                                 int32_t* tout, int32_t* status, void* cuda_stream) {
+  if (!parent || !tin || !tout || !status) return CLV_ERR_NULL;
+  if (batch < 1 || n_nodes < 1) return CLV_ERR_SHAPE;
+  if (n_nodes > CLV_MAX_NODES) return CLV_ERR_UNSUPPORTED;
+  cudaError_t e = launch_tree_to_intervals(batch, n_nodes, parent, tin, tout, status,
+                                           static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+clv_status clv_tree_from_intervals(int32_t batch, int32_t n_nodes, const int32_t* tin, const int32_t* tout,
+                                   int32_t* parent, int32_t* status, void* cuda_stream) {
+  if (!parent || !tin || !tout || !status) return CLV_ERR_NULL;
+  if (batch < 1 || n_nodes < 1) return CLV_ERR_SHAPE;
+  if (n_nodes > CLV_MAX_NODES) return CLV_ERR_UNSUPPORTED;
+  cudaError_t e = launch_tree_from_intervals(batch, n_nodes, tin, tout, parent, status,
+                                             static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
+clv_status clv_kv_commit_layers(const clv_shape* shape, const clv_kv_cache* cache, int32_t n_layers,
+                                int64_t cache_layer_stride, const void* k_tree, const void* v_tree,
+                                int64_t tree_layer_stride, const int32_t* accept_idx, const int32_t* accept_len,
+                                const int32_t* ctx_len, int32_t* ctx_len_out, int32_t* status, void* cuda_stream) {
+  clv_status st = check_shape(shape);
+  if (st != CLV_OK) return st;
+  st = check_cache(cache);
+  if (st != CLV_OK) return st;
+  if (!k_tree || !v_tree || !accept_idx || !accept_len || !ctx_len || !ctx_len_out || !status) return CLV_ERR_NULL;
+  if (!aligned16(k_tree) || !aligned16(v_tree)) return CLV_ERR_ALIGN;
+  if (shape->path_cap < 1 || n_layers < 1 || n_layers > 65535) return CLV_ERR_SHAPE;
+  const int64_t row = (int64_t)shape->n_kv_heads * CLV_HEAD_DIM;   // elements per token row
+  const int64_t tree_elems = (int64_t)shape->batch * shape->n_nodes * row;
+  const int64_t cache_elems = cache->paged ? (int64_t)cache->n_pages * CLV_PAGE_SIZE * row
+                                           : (int64_t)shape->batch * cache->cap_tokens * row;
+  if (n_layers > 1 && (cache_layer_stride < cache_elems || tree_layer_stride < tree_elems)) return CLV_ERR_SHAPE;
+  if ((cache_layer_stride % 8) != 0 || (tree_layer_stride % 8) != 0) return CLV_ERR_ALIGN;
+  if (ctx_len_out == ctx_len) return CLV_ERR_UNSUPPORTED;   // every layer's block reads ctx_len
+  const size_t tree_bytes = (size_t)(((int64_t)n_layers - 1) * tree_layer_stride + tree_elems) * 2;
+  const size_t cache_bytes = (size_t)(((int64_t)n_layers - 1) * cache_layer_stride + cache_elems) * 2;
+  if (overlaps(k_tree, tree_bytes, cache->k, cache_bytes) || overlaps(k_tree, tree_bytes, cache->v, cache_bytes) ||
+      overlaps(v_tree, tree_bytes, cache->k, cache_bytes) || overlaps(v_tree, tree_bytes, cache->v, cache_bytes))
+    return CLV_ERR_UNSUPPORTED;
+  cudaError_t e = launch_commit_layers(*shape, *cache, n_layers, cache_layer_stride, k_tree, v_tree,
+                                       tree_layer_stride, accept_idx, accept_len, ctx_len, ctx_len_out, status,
+                                       static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CLV_OK : cuda_fail(e);
+}
+
 clv_status clv_build_token_tree(int32_t batch, int32_t n_cand, int32_t max_len, int32_t node_cap,
                                 const int32_t* root_token, const int32_t* cand, const int32_t* cand_len,
                                 int32_t* tokens, int32_t* parent, int32_t* n_nodes, int32_t* node_of,

@@ -62,6 +62,17 @@ cudaError_t launch_walk_commit(const clv_shape& s, const clv_kv_cache& c, const 
                                int32_t* accept_idx, int32_t* next_token, int32_t* ctx_len_out,
                                int32_t* walk_status, int32_t* commit_status, cudaStream_t stream);
 
+cudaError_t launch_commit_layers(const clv_shape& s, const clv_kv_cache& c, int n_layers, int64_t cache_layer_stride,
+                                 const void* k_tree, const void* v_tree, int64_t tree_layer_stride,
+                                 const int32_t* accept_idx, const int32_t* accept_len, const int32_t* ctx_len,
+                                 int32_t* ctx_len_out, int32_t* status, cudaStream_t stream);
+
+// ---- interval (depth-first label) form of the tree mask
+cudaError_t launch_tree_to_intervals(int batch, int n_nodes, const int32_t* parent, int32_t* tin, int32_t* tout,
+                                     int32_t* status, cudaStream_t stream);
+cudaError_t launch_tree_from_intervals(int batch, int n_nodes, const int32_t* tin, const int32_t* tout,
+                                       int32_t* parent, int32_t* status, cudaStream_t stream);
+
 // ---- tree attention (tcgen05 / TMA; a row tile holds whole nodes: any group size G up to 128) -------
 struct AttnPlan {
   int m_tiles;   // row tiles per (sequence, kv head)

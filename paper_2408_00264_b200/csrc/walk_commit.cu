@@ -172,6 +172,23 @@ __global__ void __launch_bounds__(256) walk_commit_kernel(WalkArgs w, CommitPara
   commit_sequence(csm, p, blockIdx.x, threadIdx.x);
 }
 
+// The commit of every layer of a model in one launch: block (b, layer) copies the accepted rows of
+// sequence b in that layer's tree buffers into that layer's cache.  All layers share the accepted
+// path, the context lengths and (paged) the block table, so every block of a sequence reaches the
+// same verdict; ctx_len_out and status are written by each of them with the same values.
+__global__ void __launch_bounds__(256) commit_layers_kernel(CommitParams p, long long cache_stride_vec,
+                                                            long long tree_stride_vec) {
+  __shared__ CommitSmem sm;
+  cudaGridDependencySynchronize();
+  cudaTriggerProgrammaticLaunchCompletion();
+  const long long layer = blockIdx.y;
+  p.kc += layer * cache_stride_vec;
+  p.vc += layer * cache_stride_vec;
+  p.k_tree += layer * tree_stride_vec;
+  p.v_tree += layer * tree_stride_vec;
+  commit_sequence(sm, p, blockIdx.x, threadIdx.x);
+}
+
 }  // namespace
 
 cudaError_t launch_walk(const clv_shape& s, const int32_t* parent, const int32_t* tokens,
@@ -260,6 +277,24 @@ cudaError_t launch_walk_commit(const clv_shape& s, const clv_kv_cache& c, const 
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, walk_commit_kernel, w, p);
+}
+
+cudaError_t launch_commit_layers(const clv_shape& s, const clv_kv_cache& c, int n_layers, int64_t cache_layer_stride,
+                                 const void* k_tree, const void* v_tree, int64_t tree_layer_stride,
+                                 const int32_t* accept_idx, const int32_t* accept_len, const int32_t* ctx_len,
+                                 int32_t* ctx_len_out, int32_t* status, cudaStream_t stream) {
+  const CommitParams p = commit_params(s, c, k_tree, v_tree, accept_idx, accept_len, ctx_len, ctx_len_out, status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)s.batch, (unsigned)n_layers, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, commit_layers_kernel, p, (long long)(cache_layer_stride / 8),
+                            (long long)(tree_layer_stride / 8));
 }
 
 }  // namespace clv

@@ -400,6 +400,19 @@ def generate(cfg: VerifyConfig, ld_pad: int = 0, extra_cap: int = 0,
                     path_cap=path_cap)
 
 
+def layer_tensors(w: Workload, n_layers: int):
+    """Per-layer Q, tree K/V and cache K/V for a whole-model verify step on the trees, contexts and
+    (paged) block table of ``w``: layer 0 is ``w`` itself, every further layer draws fresh N(0,1)
+    tensors of the same shapes.  Returns uint16 arrays with a leading layer axis."""
+    s0 = w.cfg.seed * 7919
+    out = []
+    for name, off in (("q", 1), ("k_tree", 2), ("v_tree", 3), ("k_cache", 4), ("v_cache", 5)):
+        base = getattr(w, name)
+        layers = [base] + [_normal_bf16(base.shape, s0 + 1000 * l + off) for l in range(1, n_layers)]
+        out.append(np.stack(layers))
+    return tuple(out)
+
+
 def small_config(name: str = "small", **kw) -> VerifyConfig:
     """A reduced configuration for tests; keyword arguments override the defaults."""
     base = dict(name=name, batch=2, n_q_heads=8, n_kv_heads=2, ctx=200, n_nodes=24, max_depth=5,
