@@ -246,6 +246,55 @@ def tree_from_intervals(tin, tout):
     return parent, status
 
 
+def draft_head_step(h, e, wts, k_top: int, eps: float = 1e-5):
+    """One step of a Clover-2 draft head for every row (Sec. 3.1; App. A.3 prints the Attention
+    Decoder), in float64 numpy, written as the definition.  h: [R, H] hidden states (of the target,
+    or of the previous head), e: [R, H] embeddings of the previously emitted tokens; both uint16
+    bf16 bits, like every weight in ``wts`` (a dict):
+      norm1 [H], wq, wk, wv [H, H], bq, bk, bv [H], n_heads (int), wfc [H, 2H], bfc [H], norm2 [H],
+      lm_head [V, H].
+    Attention Decoder:  x = RMSNorm(h; norm1);  q = x wq^T + bq;  k = e wk^T + bk;  v = e wv^T + bv;
+    per head j (H / n_heads consecutive features): gate_j = <q_j, k_j> / max(|q_j| |k_j|, 1e-8);
+    a = h + v * gate (the gate broadcast over its head's features; no activation).
+    Output projector: p = [a, e] wfc^T + bfc (a fully connected layer over the decoder's output and
+    the token embedding).  Logits = RMSNorm(p; norm2) lm_head^T; the head's proposals are the k_top
+    largest logits of each row, highest first, lower index first among equals.
+    Returns (p float64 [R, H], top ids int32 [R, k_top], top logits float64 [R, k_top], logits [R, V])."""
+    f = lambda a: _bits_to_f64(np.asarray(a))  # noqa: E731
+    h64, e64 = f(h), f(e)
+    R, H = h64.shape
+    nh = int(wts["n_heads"])
+    hd = H // nh
+
+    def rms(x, g):
+        return x / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps) * f(g)
+    x = rms(h64, wts["norm1"])
+    q = x @ f(wts["wq"]).T + f(wts["bq"])
+    k = e64 @ f(wts["wk"]).T + f(wts["bk"])
+    v = e64 @ f(wts["wv"]).T + f(wts["bv"])
+    a = np.empty_like(h64)
+    for r in range(R):
+        for j in range(nh):
+            sl = slice(j * hd, (j + 1) * hd)
+            den = max(np.sqrt((q[r, sl] ** 2).sum()) * np.sqrt((k[r, sl] ** 2).sum()), 1e-8)
+            gate = float(q[r, sl] @ k[r, sl]) / den
+            a[r, sl] = h64[r, sl] + v[r, sl] * gate
+    p = np.concatenate([a, e64], axis=1) @ f(wts["wfc"]).T + f(wts["bfc"])
+    logits = rms(p, wts["norm2"]) @ f(wts["lm_head"]).T
+    V = logits.shape[1]
+    ids = np.empty((R, k_top), np.int32)
+    vals = np.empty((R, k_top), np.float64)
+    for r in range(R):
+        order = sorted(range(V), key=lambda t: (-logits[r, t], t))[:k_top]
+        ids[r] = order
+        vals[r] = logits[r, order]
+    return p, ids, vals, logits
+
+
+def _bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
 def accept_walk(parent, tokens, ids, path_cap: int):
     """Greedy acceptance walk; returns (accept_len [B], accept_idx [B,path_cap], next_token [B],
     status [B])."""

@@ -22,6 +22,10 @@
  *   tree_to_intervals / tree_from_intervals (in the Python wrapper, a recursive walk and plain
  *                       loops) - App. A.1: the compressed, linear form of the tree mask, taken
  *                       as depth-first entry/exit labels.
+ *   draft_head_step (in the Python wrapper, float64 numpy) - Sec. 3.1 and App. A.3: the Attention
+ *                       Decoder (RMSNorm, q/k/v projections, per-head cosine gate, residual), the
+ *                       fully connected output projector over its output and the token
+ *                       embedding, then norm + LM head and the head's top-k proposals.
  *   orc_accept_walk   - Sec. 2.1 verification phase (the target filters out wrong drafted
  *                       tokens; the output equals plain decoding) with the greedy rule of the
  *                       tree-sampling algorithm Sec. 4.1 adopts.

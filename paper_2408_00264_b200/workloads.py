@@ -413,6 +413,27 @@ def layer_tensors(w: Workload, n_layers: int):
     return tuple(out)
 
 
+def make_draft_head(rows: int, hidden_dim: int, n_heads: int, vocab: int, seed: int):
+    """Random inputs and weights of one Clover-2 draft-head step (trained heads are not available):
+    hidden states and token embeddings N(0,1), projection weights N(0, 1/fan_in), small biases,
+    norm gains around 1, all rounded to bf16.  Returns (h, e, weights dict) as uint16 bit patterns."""
+    s = seed * 7919
+    H = hidden_dim
+
+    def scaled(shape, k, factor):
+        x = bf16_bits_to_f32(_normal_bf16(shape, s + k)) * np.float32(factor)
+        return f32_to_bf16_bits(x)
+    inv = 1.0 / math.sqrt(H)
+    wts = {"n_heads": n_heads,
+           "norm1": f32_to_bf16_bits(1.0 + 0.1 * bf16_bits_to_f32(_normal_bf16((H,), s + 10))),
+           "norm2": f32_to_bf16_bits(1.0 + 0.1 * bf16_bits_to_f32(_normal_bf16((H,), s + 11))),
+           "wq": scaled((H, H), 12, inv), "wk": scaled((H, H), 13, inv), "wv": scaled((H, H), 14, inv),
+           "bq": scaled((H,), 15, 0.1), "bk": scaled((H,), 16, 0.1), "bv": scaled((H,), 17, 0.1),
+           "wfc": scaled((H, 2 * H), 18, 1.0 / math.sqrt(2 * H)), "bfc": scaled((H,), 19, 0.1),
+           "lm_head": scaled((vocab, H), 20, inv)}
+    return _normal_bf16((rows, H), s + 1), _normal_bf16((rows, H), s + 2), wts
+
+
 def small_config(name: str = "small", **kw) -> VerifyConfig:
     """A reduced configuration for tests; keyword arguments override the defaults."""
     base = dict(name=name, batch=2, n_q_heads=8, n_kv_heads=2, ctx=200, n_nodes=24, max_depth=5,
