@@ -139,6 +139,49 @@ def time_model_step(w, n_layers, dev):
             "gbs": total / us / 1e3}
 
 
+def time_draft_head(rows, hidden, n_heads, vocab, dev):
+    """clv_draft_head_step (Attention Decoder, output projector, norm + LM head, top-8) on `rows`
+    rows with random weights: microseconds per step (9 launches, replayed from a CUDA graph) and the
+    rate at which the step streams its weights (1.22 GB at hidden 4096 and vocabulary 128256: far
+    larger than the L2, so every step reads them from HBM)."""
+    import torch
+    from paper_2408_00264_b200 import binding as clv
+    from paper_2408_00264_b200 import workloads as W
+    h, e, wts = W.make_draft_head(rows, hidden, n_heads, vocab, seed=W.BASE_SEED + 31)
+    dw = {n: (v if n == "n_heads" else W.as_torch_bf16(v).to(dev)) for n, v in wts.items()}
+    head = clv.make_draft_head(dw)
+    ws = clv.new_draft_head_workspace(rows, hidden, vocab, dev)
+    k = 8
+    hid = torch.empty(rows, hidden, dtype=torch.bfloat16, device=dev)
+    ids = torch.zeros(rows, k, dtype=torch.int32, device=dev)
+    vals = torch.zeros(rows, k, dtype=torch.float32, device=dev)
+    st = torch.zeros(5, dtype=torch.int32, device=dev)
+    dh, de = W.as_torch_bf16(h).to(dev), W.as_torch_bf16(e).to(dev)
+    call = lambda: clv.clv_draft_head_step(head, dh, de, k, hid, ids, vals, st, ws)  # noqa: E731
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        call()
+    g.replay()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    reps = 20
+    a.record(cur)
+    for _ in range(reps):
+        g.replay()
+    b.record(cur)
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) / reps * 1e3
+    wbytes = (3 * hidden * hidden + 2 * hidden * hidden + vocab * hidden) * 2
+    bw_peak, bw_kind = measured_peaks()
+    return {"rows": rows, "hidden": hidden, "n_heads": n_heads, "vocab": vocab, "k_top": k, "us": us,
+            "launches": 9, "status": st.cpu().tolist(), "weight_bytes": wbytes, "gbs": wbytes / us / 1e3,
+            "frac_of_hbm_peak": {"of_%s_%.0f_GBps" % (bw_kind, bw_peak): wbytes / us / 1e3 / bw_peak}}
+
+
 def time_lm_head(rows, hidden, vocab, dev, args):
     """clv_lm_head_argmax on `rows` tree nodes: microseconds per launch (CUDA events, launches
     replayed from a CUDA graph over two copies of the weight matrix, 2 x 1.05 GB at vocabulary
@@ -575,11 +618,13 @@ def run_clv(args):
     tree_us = None
     sample_us = None
     model_us = None
+    head_us = None
     if rank == 0 and not args.no_lm_head:
         lm_head = time_lm_head(B * N, 4096, c.vocab, dev, args)
         tree_us = time_token_tree(B, 128, dev)
         sample_us = time_accept_sample(w, dev)
         model_us = time_model_step(w, 32, dev) if args.workload in ("C1", "C2", "C3") else None
+        head_us = time_draft_head(B, 4096, 32, c.vocab, dev)
 
     # ---- the other stated workloads, one after the other on rank 0's GPU (single-GPU runs) ------
     others = {}
@@ -625,7 +670,7 @@ def run_clv(args):
         "e2e": {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "steps": n_e2e},
-        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us, "accept_sample": sample_us, "model_step": model_us},
+        "next_rows": {"lm_head_argmax": lm_head, "build_token_tree": tree_us, "accept_sample": sample_us, "model_step": model_us, "draft_head_step": head_us},
         "other_workloads": others,
         "gpu_launches": 3 * args.steps * main_res["repeats"],   # attention, argmax, walk + commit in one launch
         "clocks": main_res["clocks"],

@@ -254,6 +254,46 @@ clv_status clv_kv_commit_layers(const clv_shape* shape, const clv_kv_cache* cach
                                 void* cuda_stream);
 
 /*
+ * One step of a Clover-2 draft head (Sec. 3.1 "Attention Decoder output projector", "Other
+ * Details"; App. A.3 prints the Attention Decoder) for `rows` rows, one per sequence and candidate:
+ *   x = RMSNorm(h; norm1);  q = x wq^T + bq;  k = e wk^T + bk;  v = e wv^T + bv;
+ *   per head j (hidden_dim / n_heads consecutive features):
+ *       gate_j = <q_j, k_j> / max(|q_j| |k_j|, 1e-8);      a = h + v * gate   (no activation)
+ *   p = [a, e] wfc^T + bfc             (the fully connected output projector over the decoder's
+ *                                       output and the token embedding)
+ *   logits = RMSNorm(p; norm2) lm_head^T;   top_ids / top_logits = the k_top largest logits of each
+ *   row, highest first, lower index first among equals;   hidden_out = p (bf16), the hidden state
+ *   the next head regresses on.
+ * h: the target's last hidden state (first head) or the previous head's hidden_out; e: embedding
+ * of the previously emitted token (the paper takes it from the transposed LM head).  The paper's
+ * listing names its norm inconsistently and cuts one line short; the reading taken is RMSNorm
+ * (eps = rms_eps) before the q projection and before the LM head, linear layers with bias.
+ * Arithmetic: the operands of every product are bf16 (x, a, RMSNorm(p) are rounded once), sums,
+ * gates and logits fp32 (tensor cores).  All pointers device; h, e, hidden_out bf16 [rows,
+ * hidden_dim]; top_ids int32 and top_logits fp32 [rows, k_top]; status int32 [5] (one word per
+ * product: CLV_OK or CLV_ERR_TIMEOUT).  rows <= 256, hidden_dim a multiple of 64 and of n_heads,
+ * 1 <= k_top <= 64.  workspace: at least clv_draft_head_workspace_bytes(), initialised with
+ * clv_workspace_init.  The step streams every weight once (1.22 GB at hidden 4096, vocabulary
+ * 128256) and is bound by that.
+ */
+typedef struct {
+  int32_t hidden_dim, n_heads, vocab;
+  float rms_eps;
+  const void* norm1; const void* norm2;                 /* bf16 [hidden_dim]                  */
+  const void* wq; const void* wk; const void* wv;       /* bf16 [hidden_dim, hidden_dim]      */
+  const void* bq; const void* bk; const void* bv;       /* bf16 [hidden_dim]                  */
+  const void* wfc;                                      /* bf16 [hidden_dim, 2 * hidden_dim]  */
+  const void* bfc;                                      /* bf16 [hidden_dim]                  */
+  const void* lm_head;                                  /* bf16 [vocab, hidden_dim]           */
+} clv_draft_head;
+
+size_t clv_draft_head_workspace_bytes(int32_t rows, int32_t hidden_dim, int32_t vocab);
+clv_status clv_draft_head_step(const clv_draft_head* head, int32_t rows,
+                               const void* h, const void* e, int32_t k_top,
+                               void* hidden_out, int32_t* top_ids, float* top_logits, int32_t* status,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * LM head fused with the greedy choice (Sec. 3.1: the target's final norm and LM head produce the
  * logits of every tree node; Sec. 4.2: greedy decoding at temperature 0):
  *   argmax_ids[r] = the lowest v that maximises round_bf16(sum_k hidden[r][k] * weight[v][k]),

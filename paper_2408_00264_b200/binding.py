@@ -26,6 +26,7 @@ EXPORTS = (
     "clv_status_string", "clv_last_cuda_error", "clv_version", "clv_accept_argmax_noalloc",
     "clv_lm_head_argmax", "clv_build_token_tree", "clv_accept_walk_commit", "clv_accept_sample",
     "clv_tree_to_intervals", "clv_tree_from_intervals", "clv_kv_commit_layers",
+    "clv_draft_head_step", "clv_draft_head_workspace_bytes",
     "clv_test_set_wait_limit",
 )
 
@@ -54,6 +55,12 @@ class ClvHostOutputs(ctypes.Structure):
     _fields_ = [("out", ctypes.c_void_p), ("argmax_ids", ctypes.c_void_p),
                 ("accept_len", ctypes.c_void_p), ("accept_idx", ctypes.c_void_p),
                 ("next_token", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+class ClvDraftHead(ctypes.Structure):
+    _fields_ = [("hidden_dim", ctypes.c_int32), ("n_heads", ctypes.c_int32), ("vocab", ctypes.c_int32),
+                ("rms_eps", ctypes.c_float)] + [(n, ctypes.c_void_p) for n in (
+                    "norm1", "norm2", "wq", "wk", "wv", "bq", "bk", "bv", "wfc", "bfc", "lm_head")]
 
 
 class ClvError(RuntimeError):
@@ -99,6 +106,10 @@ def lib() -> ctypes.CDLL:
         L.clv_tree_from_intervals.argtypes = [i32, i32, vp, vp, vp, vp, vp]
         L.clv_kv_commit_layers.restype = i32
         L.clv_kv_commit_layers.argtypes = [vp, vp, i32, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp]
+        L.clv_draft_head_workspace_bytes.restype = sz
+        L.clv_draft_head_workspace_bytes.argtypes = [i32, i32, i32]
+        L.clv_draft_head_step.restype = i32
+        L.clv_draft_head_step.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
         L.clv_accept_sample.restype = i32
         L.clv_accept_sample.argtypes = [vp, vp, i64, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, vp]
         L.clv_build_token_tree.restype = i32
@@ -258,6 +269,34 @@ def clv_kv_commit_layers(shape, cache, n_layers, cache_layer_stride, k_tree, v_t
     if check:
         _check(code, "clv_kv_commit_layers")
     return code
+
+
+def make_draft_head(weights: dict, rms_eps: float = 1e-5) -> ClvDraftHead:
+    """weights: torch bf16 CUDA tensors under the names of ClvDraftHead's pointer fields, plus
+    ``n_heads``; the tensors must stay alive while the descriptor is used."""
+    H = weights["wq"].shape[0]
+    d = ClvDraftHead(int(H), int(weights["n_heads"]), int(weights["lm_head"].shape[0]), float(rms_eps))
+    for n in ("norm1", "norm2", "wq", "wk", "wv", "bq", "bk", "bv", "wfc", "bfc", "lm_head"):
+        setattr(d, n, weights[n].data_ptr())
+    return d
+
+
+def clv_draft_head_step(head, h, e, k_top, hidden_out, top_ids, top_logits, status, workspace, stream=None,
+                        check=True) -> int:
+    """h, e, hidden_out: bf16 [rows, hidden]; top_ids int32 / top_logits float32 [rows, k_top]; status int32 [5]."""
+    code = lib().clv_draft_head_step(_ref(head), int(h.shape[0]), _ptr(h), _ptr(e), int(k_top), _ptr(hidden_out),
+                                     _ptr(top_ids), _ptr(top_logits), _ptr(status), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream))
+    if check:
+        _check(code, "clv_draft_head_step")
+    return code
+
+
+def new_draft_head_workspace(rows: int, hidden_dim: int, vocab: int, device="cuda") -> torch.Tensor:
+    n = int(lib().clv_draft_head_workspace_bytes(int(rows), int(hidden_dim), int(vocab)))
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    clv_workspace_init(ws)
+    return ws
 
 
 def clv_build_token_tree(root_token, cand, cand_len, tokens, parent, n_nodes, node_of, status,

@@ -296,6 +296,34 @@ clv_status clv_kv_commit_layers(const clv_shape* shape, const clv_kv_cache* cach
   return e == cudaSuccess ? CLV_OK : cuda_fail(e);
 }
 
+size_t clv_draft_head_workspace_bytes(int32_t rows, int32_t hidden_dim, int32_t vocab) {
+  if (rows < 1 || hidden_dim < 1 || vocab < 1) return 0;
+  return kWsFixedBytes + draft_head_scratch_bytes(rows, hidden_dim, vocab);
+}
+
+clv_status clv_draft_head_step(const clv_draft_head* head, int32_t rows, const void* h, const void* e,
+                               int32_t k_top, void* hidden_out, int32_t* top_ids, float* top_logits,
+                               int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!head || !h || !e || !hidden_out || !top_ids || !top_logits || !status) return CLV_ERR_NULL;
+  if (!head->norm1 || !head->norm2 || !head->wq || !head->wk || !head->wv || !head->bq || !head->bk || !head->bv ||
+      !head->wfc || !head->bfc || !head->lm_head)
+    return CLV_ERR_NULL;
+  const int H = head->hidden_dim;
+  if (rows < 1 || H < 1 || head->n_heads < 1 || head->vocab < 1 || k_top < 1 || k_top > head->vocab) return CLV_ERR_SHAPE;
+  if (!(head->rms_eps > 0.f)) return CLV_ERR_SHAPE;
+  if (rows > 256 || (H % 64) != 0 || (H % head->n_heads) != 0 || k_top > 64) return CLV_ERR_UNSUPPORTED;
+  if (!lm_head_supported(rows, H, head->vocab)) return CLV_ERR_UNSUPPORTED;
+  const void* ptrs[] = {h, e, hidden_out, head->wq, head->wk, head->wv, head->wfc, head->lm_head};
+  for (const void* q : ptrs) if (!aligned16(q)) return CLV_ERR_ALIGN;
+  if (!workspace || workspace_bytes < kWsFixedBytes + draft_head_scratch_bytes(rows, H, head->vocab))
+    return CLV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return CLV_ERR_ALIGN;
+  cudaError_t err = launch_draft_head_step(*head, rows, h, e, k_top, hidden_out, top_ids, top_logits, status,
+                                           ws_tickets(workspace), ws_scratch(workspace),
+                                           static_cast<cudaStream_t>(cuda_stream));
+  return err == cudaSuccess ? CLV_OK : cuda_fail(err);
+}
+
 clv_status clv_build_token_tree(int32_t batch, int32_t n_cand, int32_t max_len, int32_t node_cap,
                                 const int32_t* root_token, const int32_t* cand, const int32_t* cand_len,
                                 int32_t* tokens, int32_t* parent, int32_t* n_nodes, int32_t* node_of,

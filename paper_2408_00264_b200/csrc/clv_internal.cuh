@@ -103,6 +103,17 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
                                   int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
                                   unsigned* tickets, cudaStream_t stream);
 
+int rows_linear_splits(int rows, int in_dim, int out_dim);
+cudaError_t launch_rows_linear(const void* x, int64_t ld_x, const void* weight, int64_t ld_weight, const void* bias,
+                               int rows, int in_dim, int out_dim, float* out, int64_t ld_out, int splits,
+                               int64_t split_stride, int32_t* status, unsigned* tickets, cudaStream_t stream);
+
+// ---- one step of a Clover-2 draft head
+size_t draft_head_scratch_bytes(int rows, int hidden, int vocab);
+cudaError_t launch_draft_head_step(const clv_draft_head& w, int rows, const void* h, const void* e, int k_top,
+                                   void* hidden_out, int32_t* top_ids, float* top_logits, int32_t* status,
+                                   unsigned* tickets, void* scratch, cudaStream_t stream);
+
 // ---- token tree from speculated sequences -------------------------------------------------------
 cudaError_t launch_token_tree(int batch, int n_cand, int max_len, int node_cap, const int32_t* root_token,
                               const int32_t* cand, const int32_t* cand_len, int32_t* tokens, int32_t* parent,

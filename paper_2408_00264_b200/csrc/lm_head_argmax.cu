@@ -40,6 +40,11 @@ struct Params {
   int full_items;   // work items that are whole tiles; the rest are half tiles (128 vocabulary entries)
   int n_items;
   int32_t* ids;
+  float* out;                 // not NULL: the products (+ bias) are written here, fp32 [M, ld_out], and no argmax is taken
+  int64_t ld_out;
+  int k_splits;               // with `out`: the K axis is cut in this many parts, part s writes its partial
+  int64_t out_split_stride;   //   products to out + s * out_split_stride (the reader adds the parts up)
+  const uint16_t* bias;       // bf16 [V] or NULL (only with `out`)
   unsigned long long* keys;   // [M], zero between calls
   unsigned* counter;          // zero between calls
   unsigned* aborts;           // blocks that gave up a wait; zero between calls
@@ -118,8 +123,8 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   auto sA = [&](int s, int mt) { return smem_base + (uint32_t)s * kStageBytes + (uint32_t)mt * kATile; };
   auto sW = [&](int s) { return smem_base + (uint32_t)s * kStageBytes + 2 * kATile; };
 
-  const int n_items = p.n_items;
-  const int k_chunks = p.K / BK;
+  const int n_items = p.n_items * p.k_splits;   // (tile, row block, part of the K axis)
+  const int k_chunks = p.K / BK / p.k_splits;
   int issued = 0;  // ring stages filled by the producer (for the drain)
 
   if (warp == 0) {
@@ -128,7 +133,8 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       bool ok = true;
       int it = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item wi = decode_item(p, item);
+        const Item wi = decode_item(p, item / p.k_splits);
+        const int kc0 = (item % p.k_splits) * k_chunks;
         const int mb = wi.mb;
         const int rows_left = p.M - mb * MB;
         const int m_tiles = rows_left > BM ? 2 : 1;
@@ -138,9 +144,9 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
           if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag, wlim);
           if (!ok) break;
           mbar_expect_tx(bar_full(s), w_bytes + (uint32_t)m_tiles * kATile);
-          tma_load_2d(sW(s), wi.cols == BN ? &tm_w : &tm_w_half, kc * BK, wi.col0, bar_full(s));
+          tma_load_2d(sW(s), wi.cols == BN ? &tm_w : &tm_w_half, (kc0 + kc) * BK, wi.col0, bar_full(s));
           for (int mt = 0; mt < m_tiles; ++mt)
-            tma_load_2d(sA(s, mt), &tm_a, kc * BK, mb * MB + mt * BM, bar_full(s));
+            tma_load_2d(sA(s, mt), &tm_a, (kc0 + kc) * BK, mb * MB + mt * BM, bar_full(s));
           issued = it + 1;
         }
       }
@@ -151,7 +157,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       bool ok = true;
       int it = 0, tile = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
-        const Item wi = decode_item(p, item);
+        const Item wi = decode_item(p, item / p.k_splits);
         const int m_tiles = (p.M - wi.mb * MB) > BM ? 2 : 1;
         const uint32_t idesc = wi.cols == BN ? kIdesc : kIdescHalf;
         if (tile > 0) {  // the epilogue has taken the previous tile out of tensor memory
@@ -186,7 +192,8 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     bool ok = true;
     int tile = 0;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
-      const Item wi = decode_item(p, item);
+      const Item wi = decode_item(p, item / p.k_splits);
+      const int part = item % p.k_splits;
       const int mb = wi.mb;
       const int row = mb * MB + mt * BM + row_in_tile;
       const bool row_valid = row < p.M;
@@ -204,6 +211,19 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
           uint32_t x[32];
           tmem_ld_x32(tmem + lane_addr + (uint32_t)(mt * BN + c), x);
           tmem_wait_ld();
+          if (p.out != nullptr) {   // plain product: this row's 32 values (+ bias) go to memory
+            if (row_valid) {
+              float* dst = p.out + part * p.out_split_stride + (int64_t)row * p.ld_out + col0 + c;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + c + j >= p.V) continue;
+                float v = __uint_as_float(x[j]);
+                if (p.bias != nullptr && part == 0) v += __uint_as_float((uint32_t)p.bias[col0 + c + j] << 16);
+                dst[j] = v;
+              }
+            }
+            continue;
+          }
           // rounding to bf16 is monotonic: the chunk's maximum first, the position only if it wins
           float m = -INFINITY;
 #pragma unroll
@@ -253,6 +273,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   // the last block turns the keys into indices and leaves keys and counters zero for the next call
   __threadfence();
   if (tid == 0) *p.status = atomicExch(p.aborts, 0u) ? (int)CLV_ERR_TIMEOUT : (int)CLV_OK;
+  if (p.out != nullptr) return;   // no keys were written
   for (int r = tid; r < p.M; r += kThreads) {
     const unsigned long long key = atomicExch(p.keys + r, 0ull);
     const int idx = (int)(0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull));
@@ -280,9 +301,11 @@ bool lm_head_supported(int rows, int hidden, int vocab) {
          encode_fn() != nullptr;
 }
 
-cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
-                                  int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
-                                  unsigned* tickets, cudaStream_t stream) {
+namespace {
+cudaError_t launch_rows_times_weights(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
+                                      int rows, int hidden_dim, int vocab, int32_t* ids, float* out, int64_t ld_out,
+                                      const void* bias, int k_splits, int64_t out_split_stride, int32_t* status,
+                                      unsigned* tickets, cudaStream_t stream) {
   static OncePerDevice once;
   cudaError_t e0 = run_once_per_device(once, [] {
     return cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
@@ -300,15 +323,21 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
   p.n_tiles = (vocab + BN - 1) / BN;
   p.m_blocks = (rows + MB - 1) / MB;
   p.ids = ids;
+  p.out = out;
+  p.ld_out = ld_out;
+  p.bias = static_cast<const uint16_t*>(bias);
+  p.k_splits = k_splits;
+  p.out_split_stride = out_split_stride;
   p.counter = tickets;
   p.aborts = tickets + 1;
   p.keys = reinterpret_cast<unsigned long long*>(tickets + 2);
   p.status = status;
   p.wait_limit = wait_limit_cycles();
   const int tiles = p.n_tiles * p.m_blocks;
-  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const int work = tiles * k_splits;
+  const int grid = work < sm_count() ? work : sm_count();
   const int rem = tiles % grid;   // tiles of the last, incomplete round
-  const int split = (rem > 0 && 2 * rem <= grid) ? rem : 0;
+  const int split = (k_splits == 1 && rem > 0 && 2 * rem <= grid) ? rem : 0;
   p.full_items = tiles - split;
   p.n_items = tiles + split;
   cudaLaunchConfig_t cfg = {};
@@ -322,6 +351,33 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, lm_head_argmax_kernel, tm_a, tm_w, tm_w_half, p);
+}
+}  // namespace
+
+cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
+                                  int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
+                                  unsigned* tickets, cudaStream_t stream) {
+  return launch_rows_times_weights(hidden, ld_hidden, weight, ld_weight, rows, hidden_dim, vocab, ids, nullptr, 0,
+                                   nullptr, 1, 0, status, tickets, stream);
+}
+
+// How many parts the K axis of a product with few output features is cut into, so that the launch
+// covers the machine: a power of two up to 8 that divides the number of 64-wide K chunks.
+int rows_linear_splits(int rows, int in_dim, int out_dim) {
+  const int tiles = ((out_dim + BN - 1) / BN) * ((rows + MB - 1) / MB);
+  int s = 1;
+  while (s < 8 && tiles * s * 2 <= sm_count() && (in_dim / BK) % (s * 2) == 0) s *= 2;
+  return s;
+}
+
+// out[part][r][o] = sum over part's share of k of x[r][k] * weight[o][k] (+ bias[o] in part 0):
+// the same kernel with its accumulators written out (fp32) instead of reduced to an argmax.  The
+// reader adds the `splits` parts up (a fixed order: the result does not depend on scheduling).
+cudaError_t launch_rows_linear(const void* x, int64_t ld_x, const void* weight, int64_t ld_weight, const void* bias,
+                               int rows, int in_dim, int out_dim, float* out, int64_t ld_out, int splits,
+                               int64_t split_stride, int32_t* status, unsigned* tickets, cudaStream_t stream) {
+  return launch_rows_times_weights(x, ld_x, weight, ld_weight, rows, in_dim, out_dim, nullptr, out, ld_out, bias,
+                                   splits, split_stride, status, tickets, stream);
 }
 
 }  // namespace clv
