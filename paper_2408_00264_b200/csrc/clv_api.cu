@@ -311,9 +311,11 @@ clv_status clv_draft_head_step(const clv_draft_head* head, int32_t rows, const v
   const int H = head->hidden_dim;
   if (rows < 1 || H < 1 || head->n_heads < 1 || head->vocab < 1 || k_top < 1 || k_top > head->vocab) return CLV_ERR_SHAPE;
   if (!(head->rms_eps > 0.f)) return CLV_ERR_SHAPE;
-  if (rows > 256 || (H % 64) != 0 || (H % head->n_heads) != 0 || k_top > 64) return CLV_ERR_UNSUPPORTED;
+  if (rows > 256 || (H % 64) != 0 || (H % head->n_heads) != 0 || ((H / head->n_heads) % 4) != 0 || k_top > 64)
+    return CLV_ERR_UNSUPPORTED;
   if (!lm_head_supported(rows, H, head->vocab)) return CLV_ERR_UNSUPPORTED;
-  const void* ptrs[] = {h, e, hidden_out, head->wq, head->wk, head->wv, head->wfc, head->lm_head};
+  const void* ptrs[] = {h, e, hidden_out, head->wq, head->wk, head->wv, head->wfc, head->lm_head, head->norm1,
+                        head->norm2};
   for (const void* q : ptrs) if (!aligned16(q)) return CLV_ERR_ALIGN;
   if (!workspace || workspace_bytes < kWsFixedBytes + draft_head_scratch_bytes(rows, H, head->vocab))
     return CLV_ERR_WORKSPACE;

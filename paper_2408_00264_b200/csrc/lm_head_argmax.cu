@@ -45,6 +45,10 @@ struct Params {
   int k_splits;               // with `out`: the K axis is cut in this many parts, part s writes its partial
   int64_t out_split_stride;   //   products to out + s * out_split_stride (the reader adds the parts up)
   const uint16_t* bias;       // bf16 [V] or NULL (only with `out`)
+  int out_vec;                // `out`, its strides and `bias` allow 16-byte accesses
+  int two_acc;                // M <= 128: the two accumulators alternate between tiles, so that the
+                              //   epilogue of one tile runs under the MMAs of the next
+  uint32_t a_tile_bytes;      // bytes one load of the row operand brings (a box of 8..128 rows)
   unsigned long long* keys;   // [M], zero between calls
   unsigned* counter;          // zero between calls
   unsigned* aborts;           // blocks that gave up a wait; zero between calls
@@ -88,7 +92,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                       const __grid_constant__ CUtensorMap tm_w_half, const Params p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) unsigned long long s_bar[2 * kStages + 3];
+  __shared__ __align__(8) unsigned long long s_bar[2 * kStages + 5];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ int s_last;
@@ -97,13 +101,16 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   const uint32_t bar0 = smem_u32(&s_bar[0]);
   auto bar_full = [&](int s) { return bar0 + 8u * s; };
   auto bar_empty = [&](int s) { return bar0 + 8u * (kStages + s); };
-  const uint32_t bar_acc_full = bar0 + 8u * (2 * kStages);       // a tile's accumulators are complete
-  const uint32_t bar_acc_empty = bar0 + 8u * (2 * kStages + 1);  // the epilogue has read them
-  const uint32_t bar_drain = bar0 + 8u * (2 * kStages + 2);
+  // a tile's accumulators are complete / the epilogue has read them; index 1 only with two_acc
+  auto bar_acc_full = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto bar_acc_empty = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
+  const uint32_t bar_drain = bar0 + 8u * (2 * kStages + 4);
   if (tid == 0) {
     for (int i = 0; i < 2 * kStages; ++i) mbar_init(bar0 + 8u * i, 1);
-    mbar_init(bar_acc_full, 1);
-    mbar_init(bar_acc_empty, 2 * BM);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_acc_full(b), 1);
+      mbar_init(bar_acc_empty(b), p.two_acc ? BM : 2 * BM);
+    }
     mbar_init(bar_drain, 1);
     s_abort = 0;
     fence_barrier_init();
@@ -111,6 +118,15 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   }
   if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
   if (tid == 64) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_w); tma_prefetch_desc(&tm_w_half); }
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  if (p.a_tile_bytes < kATile) {
+    // a box of fewer than 128 rows leaves the rest of the operand tile as it was: make that zeros
+    uint8_t* base = smem_raw + (smem_base - smem_u32(smem_raw));
+    for (int s = 0; s < kStages; ++s)
+      for (uint32_t o = (uint32_t)tid * 16u; o < kATile; o += kThreads * 16u)
+        *reinterpret_cast<uint4*>(base + (size_t)s * kStageBytes + o) = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
+  }
   cudaGridDependencySynchronize();  // programmatic launch: the previous kernel's results are complete
   tc_fence_before();
   __syncthreads();
@@ -119,7 +135,6 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   volatile int* abort_flag = &s_abort;
   const long long wlim = p.wait_limit;
 
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   auto sA = [&](int s, int mt) { return smem_base + (uint32_t)s * kStageBytes + (uint32_t)mt * kATile; };
   auto sW = [&](int s) { return smem_base + (uint32_t)s * kStageBytes + 2 * kATile; };
 
@@ -143,7 +158,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
           const int s = it % kStages;
           if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag, wlim);
           if (!ok) break;
-          mbar_expect_tx(bar_full(s), w_bytes + (uint32_t)m_tiles * kATile);
+          mbar_expect_tx(bar_full(s), w_bytes + (uint32_t)m_tiles * p.a_tile_bytes);
           tma_load_2d(sW(s), wi.cols == BN ? &tm_w : &tm_w_half, (kc0 + kc) * BK, wi.col0, bar_full(s));
           for (int mt = 0; mt < m_tiles; ++mt)
             tma_load_2d(sA(s, mt), &tm_a, (kc0 + kc) * BK, mb * MB + mt * BM, bar_full(s));
@@ -160,8 +175,10 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         const Item wi = decode_item(p, item / p.k_splits);
         const int m_tiles = (p.M - wi.mb * MB) > BM ? 2 : 1;
         const uint32_t idesc = wi.cols == BN ? kIdesc : kIdescHalf;
-        if (tile > 0) {  // the epilogue has taken the previous tile out of tensor memory
-          ok = mbar_wait(bar_acc_empty, (tile - 1) & 1, abort_flag, wlim);
+        const int acc = p.two_acc ? (tile & 1) : 0;          // accumulator (pair) of this tile
+        const int use = p.two_acc ? (tile >> 1) : tile;      // how often it has been used before
+        if (use > 0) {  // the epilogue has taken its previous tile out of tensor memory
+          ok = mbar_wait(bar_acc_empty(acc), (use - 1) & 1, abort_flag, wlim);
           if (!ok) break;
           tc_fence_after();
         }
@@ -175,12 +192,12 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
             const uint64_t ad = smem_desc(sA(s, mt), 16, 1024);
 #pragma unroll
             for (int ks = 0; ks < BK / 16; ++ks)
-              umma_bf16(tmem + (uint32_t)(mt * BN), ad + (uint64_t)((ks * 32) >> 4), wd + (uint64_t)((ks * 32) >> 4),
+              umma_bf16(tmem + (uint32_t)((mt + acc) * BN), ad + (uint64_t)((ks * 32) >> 4), wd + (uint64_t)((ks * 32) >> 4),
                         idesc, (kc > 0 || ks > 0) ? 1u : 0u);
           }
           umma_commit(bar_empty(s));  // the stage is free once these MMAs have read it
         }
-        if (ok) umma_commit(bar_acc_full);
+        if (ok) umma_commit(bar_acc_full(acc));
       }
     }
   } else {
@@ -195,13 +212,16 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       const Item wi = decode_item(p, item / p.k_splits);
       const int part = item % p.k_splits;
       const int mb = wi.mb;
-      const int row = mb * MB + mt * BM + row_in_tile;
+      if (p.two_acc && (tile & 1) != mt) continue;   // the other group's tile
+      const int acc = p.two_acc ? mt : 0;
+      const int row = mb * MB + (p.two_acc ? 0 : mt * BM) + row_in_tile;
       const bool row_valid = row < p.M;
-      ok = mbar_wait(bar_acc_full, tile & 1, abort_flag, wlim);
+      ok = mbar_wait(bar_acc_full(acc), (p.two_acc ? (tile >> 1) : tile) & 1, abort_flag, wlim);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      const bool group_used = (p.M - mb * MB) > mt * BM;   // second accumulator unused for a short row block
+      // the second accumulator is unused for a short row block
+      const bool group_used = p.two_acc || (p.M - mb * MB) > mt * BM;
       float best_v = -INFINITY;
       int best_i = INT_MAX;
       if (group_used) {
@@ -214,12 +234,33 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
           if (p.out != nullptr) {   // plain product: this row's 32 values (+ bias) go to memory
             if (row_valid) {
               float* dst = p.out + part * p.out_split_stride + (int64_t)row * p.ld_out + col0 + c;
+              const bool add_bias = p.bias != nullptr && part == 0;
+              if (p.out_vec && col0 + c + 32 <= p.V) {   // 128 bytes of this row in eight stores
+                if (add_bias) {
+                  const uint4* b4 = reinterpret_cast<const uint4*>(p.bias + col0 + c);
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                if (col0 + c + j >= p.V) continue;
-                float v = __uint_as_float(x[j]);
-                if (p.bias != nullptr && part == 0) v += __uint_as_float((uint32_t)p.bias[col0 + c + j] << 16);
-                dst[j] = v;
+                  for (int j = 0; j < 4; ++j) {
+                    const uint4 b = b4[j];
+                    const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                      x[8 * j + 2 * t] = __float_as_uint(__uint_as_float(x[8 * j + 2 * t]) + __uint_as_float(w[t] << 16));
+                      x[8 * j + 2 * t + 1] =
+                          __float_as_uint(__uint_as_float(x[8 * j + 2 * t + 1]) + __uint_as_float(w[t] & 0xFFFF0000u));
+                    }
+                  }
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                  reinterpret_cast<uint4*>(dst)[j] = make_uint4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  if (col0 + c + j >= p.V) continue;
+                  float v = __uint_as_float(x[j]);
+                  if (add_bias) v += __uint_as_float((uint32_t)p.bias[col0 + c + j] << 16);
+                  dst[j] = v;
+                }
               }
             }
             continue;
@@ -244,7 +285,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         }
       }
       tc_fence_before();
-      mbar_arrive(bar_acc_empty);
+      mbar_arrive(bar_acc_empty(acc));
       if (row_valid && best_i != INT_MAX) atomicMax(p.keys + row, pack_key(best_v, best_i));
     }
   }
@@ -312,7 +353,9 @@ cudaError_t launch_rows_times_weights(const void* hidden, int64_t ld_hidden, con
   });
   if (e0 != cudaSuccess) return e0;
   CUtensorMap tm_a, tm_w, tm_w_half;
-  if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, BM) ||
+  int a_box = BM;   // rows one load of the row operand brings: the power of two that covers them, 8..128
+  while (a_box > 8 && a_box / 2 >= rows) a_box /= 2;
+  if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, (uint32_t)a_box) ||
       !make_map_2d(&tm_w, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN) ||
       !make_map_2d(&tm_w_half, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN / 2))
     return cudaErrorInvalidValue;
@@ -328,6 +371,10 @@ cudaError_t launch_rows_times_weights(const void* hidden, int64_t ld_hidden, con
   p.bias = static_cast<const uint16_t*>(bias);
   p.k_splits = k_splits;
   p.out_split_stride = out_split_stride;
+  p.out_vec = out != nullptr && (reinterpret_cast<uintptr_t>(out) % 16) == 0 && (ld_out % 4) == 0 &&
+              (out_split_stride % 4) == 0 && (reinterpret_cast<uintptr_t>(bias) % 16) == 0;
+  p.two_acc = rows <= BM;
+  p.a_tile_bytes = (uint32_t)a_box * BK * 2;
   p.counter = tickets;
   p.aborts = tickets + 1;
   p.keys = reinterpret_cast<unsigned long long*>(tickets + 2);
