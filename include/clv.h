@@ -272,9 +272,18 @@ clv_status clv_kv_commit_layers(const clv_shape* shape, const clv_kv_cache* cach
  * gates and logits fp32 (tensor cores).  All pointers device; h, e, hidden_out bf16 [rows,
  * hidden_dim]; top_ids int32 and top_logits fp32 [rows, k_top]; status int32 [5] (one word per
  * product: CLV_OK or CLV_ERR_TIMEOUT).  rows <= 256, hidden_dim a multiple of 64 and of n_heads,
- * 1 <= k_top <= 64.  workspace: at least clv_draft_head_workspace_bytes(), initialised with
- * clv_workspace_init.  The step streams every weight once (1.22 GB at hidden 4096, vocabulary
- * 128256) and is bound by that.
+ * the head size hidden_dim / n_heads a multiple of 4, 1 <= k_top <= 64 (up to 32 the selection
+ * is one pass over the logits; beyond, k_top passes).  h, e, hidden_out, the weight matrices and
+ * the two norm gains start on 16-byte boundaries (CLV_ERR_ALIGN otherwise); biases may start
+ * anywhere (16-byte aligned ones are read faster).  workspace: at least
+ * clv_draft_head_workspace_bytes(), initialised with clv_workspace_init; it holds every
+ * intermediate (the caller owns it and must not share it between calls that may overlap).  A
+ * NaN logit ranks after every number; if a row has fewer than k_top entries (vocab < k_top is
+ * rejected, so this never happens) the missing ids would read -1.  The step streams every weight
+ * once (1.22 GB at hidden 4096, vocabulary 128256) and is bound by that.
+ * Errors: CLV_ERR_NULL, CLV_ERR_SHAPE (a size below 1, k_top > vocab, rms_eps <= 0),
+ * CLV_ERR_UNSUPPORTED (the limits above, no tensor-map support in the driver), CLV_ERR_ALIGN,
+ * CLV_ERR_WORKSPACE, CLV_ERR_CUDA.  Nothing is launched on an error.
  */
 typedef struct {
   int32_t hidden_dim, n_heads, vocab;

@@ -51,7 +51,10 @@ def run_gpu(clv, h, e, wts, k_top):
 
 
 @pytest.mark.parametrize("R,H,nh,V,k", [(3, 64, 4, 500, 5), (16, 256, 8, 3000, 8), (5, 128, 2, 777, 1),
-                                         (130, 128, 4, 1000, 4), (8, 4096, 32, 128256, 8)])
+                                         (130, 128, 4, 1000, 4), (8, 4096, 32, 128256, 8),
+                                         (4, 64, 4, 9000, 32),      # the widest one-pass selection, two levels
+                                         (2, 64, 2, 3000, 40),      # beyond it: one pass per proposal
+                                         (70, 192, 48, 2049, 2)])   # head size 4; one entry in the second slice
 def test_draft_head_step(clv, oracle, R, H, nh, V, k):
     h, e, wts = W.make_draft_head(R, H, nh, V, seed=R + H + V)
     p, ids, vals, logits = oracle.draft_head_step(h, e, wts, k)
@@ -100,3 +103,24 @@ def test_draft_head_step_planted_proposals_and_errors(clv, oracle):
     assert clv.clv_draft_head_step(bad, *args, ws, check=False) == clv.CLV_ERR_UNSUPPORTED
     assert clv.clv_draft_head_step(head, t(R, H), t(R, H), 65, t(R, H), t(R, 65, dt=torch.int32),
                                    t(R, 65, dt=torch.float32), t(5, dt=torch.int32), ws, check=False) == clv.CLV_ERR_UNSUPPORTED
+
+
+def test_draft_head_step_equal_logits_rank_by_index(clv, oracle):
+    # vocabulary rows that are copies of one another give equal logits on both sides (the same
+    # products in the same order): the proposals must list them lower index first
+    R, H, nh, V, k = 4, 128, 4, 4500, 6
+    h, e, wts = W.make_draft_head(R, H, nh, V, seed=311)
+    p, _, _, _ = oracle.draft_head_step(h, e, wts, k)
+    y = p / np.sqrt((p * p).mean(-1, keepdims=True) + 1e-5) * W.bf16_bits_to_f64(wts["norm2"])
+    lm = W.bf16_bits_to_f64(wts["lm_head"]).copy()
+    copies = (4100, 17, 2047, 2048, 3333)                    # in different slices and next to a slice edge
+    for t in copies:
+        lm[t] = y[1] * 2.5 / np.sqrt(H)
+    wts["lm_head"] = W.f32_to_bf16_bits(lm.astype(np.float32))
+    _, ids, vals, logits = oracle.draft_head_step(h, e, wts, k)
+    assert ids[1, :5].tolist() == sorted(copies)
+    hid, g_ids, g_vals = run_gpu(clv, h, e, wts, k)
+    assert g_ids[1, :5].tolist() == sorted(copies) and (g_vals[1, :5] == g_vals[1, 0]).all()
+    for r in range(R):
+        same = np.diff(g_vals[r]) == 0
+        assert (np.diff(g_ids[r])[same] > 0).all()
