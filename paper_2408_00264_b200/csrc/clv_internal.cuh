@@ -103,10 +103,11 @@ cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const v
                                   int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
                                   unsigned* tickets, cudaStream_t stream);
 
-int rows_linear_splits(int rows, int in_dim, int out_dim);
-cudaError_t launch_rows_linear(const void* x, int64_t ld_x, const void* weight, int64_t ld_weight, const void* bias,
-                               int rows, int in_dim, int out_dim, float* out, int64_t ld_out, int splits,
-                               int64_t split_stride, int32_t* status, unsigned* tickets, cudaStream_t stream);
+int rows_linear_splits(int rows, int in_dim, int out_dim, int n);
+cudaError_t launch_rows_linear(int n, const void* const* x, int64_t ld_x, const void* const* weight,
+                               int64_t ld_weight, const void* const* bias, int rows, int in_dim, int out_dim,
+                               float* const* out, int64_t ld_out, int splits, int64_t split_stride, int32_t* status,
+                               unsigned* tickets, cudaStream_t stream);
 
 // ---- one step of a Clover-2 draft head
 size_t draft_head_scratch_bytes(int rows, int hidden, int vocab);

@@ -309,7 +309,7 @@ size_t topk_candidates(int vocab, int k_top) {
 // candidates, values then indices [R, cand] each   (S1, S2: parts of the K axis)
 size_t draft_head_scratch_bytes(int rows, int hidden, int vocab) {
   const size_t R = rows, H = hidden, ldl = (vocab + 7) / 8 * 8;
-  const size_t s1 = rows_linear_splits(rows, hidden, hidden), s2 = rows_linear_splits(rows, 2 * hidden, hidden);
+  const size_t s1 = rows_linear_splits(rows, hidden, hidden, 3), s2 = rows_linear_splits(rows, 2 * hidden, hidden, 1);
   return up256(R * H * 2) + 3 * up256(s1 * R * H * 4) + up256(R * 2 * H * 2) + up256(s2 * R * H * 4) +
          up256(R * H * 2) + up256(R * ldl * 4) + 4 * up256(R * topk_candidates(vocab, kListK) * 4);
 }
@@ -319,7 +319,7 @@ cudaError_t launch_draft_head_step(const clv_draft_head& w, int rows, const void
                                    unsigned* tickets, void* scratch, cudaStream_t stream) {
   const int H = w.hidden_dim, V = w.vocab;
   const size_t R = rows, ldl = (V + 7) / 8 * 8;
-  const int s1 = rows_linear_splits(rows, H, H), s2 = rows_linear_splits(rows, 2 * H, H);
+  const int s1 = rows_linear_splits(rows, H, H, 3), s2 = rows_linear_splits(rows, 2 * H, H, 1);
   const int64_t part = (int64_t)R * H;   // elements between the parts of a product
   const size_t cand = topk_candidates(V, kListK);
   char* s = static_cast<char*>(scratch);
@@ -345,16 +345,31 @@ cudaError_t launch_draft_head_step(const clv_draft_head& w, int rows, const void
   // status words: one per product (a wait of the GEMM kernel that ran out)
   CLV_TRY(launch_rows(rmsnorm_rows_kernel, per_row, kNormThreads, stream, H, h16, (const float*)nullptr, 1, (int64_t)0,
                       static_cast<const uint16_t*>(w.norm1), w.rms_eps, x, (uint16_t*)nullptr));
-  CLV_TRY(launch_rows_linear(x, H, w.wq, H, w.bq, rows, H, H, q, H, s1, part, status + 0, tickets, stream));
-  CLV_TRY(launch_rows_linear(e16, H, w.wk, H, w.bk, rows, H, H, k, H, s1, part, status + 1, tickets, stream));
-  CLV_TRY(launch_rows_linear(e16, H, w.wv, H, w.bv, rows, H, H, v, H, s1, part, status + 2, tickets, stream));
+  {   // q = x wq^T + bq, k = e wk^T + bk, v = e wv^T + bv: one launch
+    const void* const xs[3] = {x, e16, e16};
+    const void* const ws[3] = {w.wq, w.wk, w.wv};
+    const void* const bs[3] = {w.bq, w.bk, w.bv};
+    float* const outs[3] = {q, k, v};
+    CLV_TRY(launch_rows_linear(3, xs, H, ws, H, bs, rows, H, H, outs, H, s1, part, status + 0, tickets, stream));
+  }
   CLV_TRY(launch_rows(gate_residual_kernel, dim3((unsigned)rows, (unsigned)((w.n_heads + 7) / 8)), kThreads, stream, H,
                       (int)w.n_heads, (const float*)q, (const float*)k, (const float*)v, s1, part, h16, e16, cat));
-  CLV_TRY(launch_rows_linear(cat, 2 * H, w.wfc, 2 * H, w.bfc, rows, 2 * H, H, p, H, s2, part, status + 3, tickets, stream));
+  {
+    const void* const xs[1] = {cat};
+    const void* const bs[1] = {w.bfc};
+    float* const outs[1] = {p};
+    CLV_TRY(launch_rows_linear(1, xs, 2 * H, &w.wfc, 2 * H, bs, rows, 2 * H, H, outs, H, s2, part, status + 3, tickets,
+                               stream));
+  }
   CLV_TRY(launch_rows(rmsnorm_rows_kernel, per_row, kNormThreads, stream, H, (const uint16_t*)nullptr, (const float*)p,
                       s2, part, static_cast<const uint16_t*>(w.norm2), w.rms_eps, y, static_cast<uint16_t*>(hidden_out)));
-  CLV_TRY(launch_rows_linear(y, H, w.lm_head, H, nullptr, rows, H, V, logits, (int64_t)ldl, 1, 0, status + 4, tickets,
-                             stream));
+  {
+    const void* const xs[1] = {y};
+    const void* const bs[1] = {nullptr};
+    float* const outs[1] = {logits};
+    CLV_TRY(launch_rows_linear(1, xs, H, &w.lm_head, H, bs, rows, H, V, outs, (int64_t)ldl, 1, 0, status + 4, tickets,
+                               stream));
+  }
   if (k_top > kListK) {
     CLV_TRY(launch_rows(topk_passes_kernel, per_row, kThreads, stream, V, (int64_t)ldl, k_top, (const float*)logits,
                         top_ids, top_logits));

@@ -26,6 +26,7 @@ constexpr int MB = 2 * BM;           // rows per block step (two accumulators)
 constexpr int BN = 256;              // vocabulary entries per tile
 constexpr int BK = 64;               // K elements per ring stage (one 128-byte swizzle row)
 constexpr int kStages = 3;
+constexpr int kMaxProb = 3;          // products of one shape that one launch can take
 constexpr uint32_t kATile = BM * BK * 2;      // 16 KB
 constexpr uint32_t kWTile = BN * BK * 2;      // 32 KB
 constexpr uint32_t kStageBytes = 2 * kATile + kWTile;
@@ -41,10 +42,12 @@ struct Params {
   int n_items;
   int32_t* ids;
   float* out;                 // not NULL: the products (+ bias) are written here, fp32 [M, ld_out], and no argmax is taken
+  int n_prob;                 // with `out`: up to kMaxProb products of one shape in one launch, each with its own
+  float* outs[3];             //   operands (tensor maps), destination and bias; out == outs[0]
+  const uint16_t* biases[3];
   int64_t ld_out;
   int k_splits;               // with `out`: the K axis is cut in this many parts, part s writes its partial
   int64_t out_split_stride;   //   products to out + s * out_split_stride (the reader adds the parts up)
-  const uint16_t* bias;       // bf16 [V] or NULL (only with `out`)
   int out_vec;                // `out`, its strides and `bias` allow 16-byte accesses
   int two_acc;                // M <= 128: the two accumulators alternate between tiles, so that the
                               //   epilogue of one tile runs under the MMAs of the next
@@ -88,9 +91,12 @@ __device__ __forceinline__ Item decode_item(const Params& p, int item) {
   return it;
 }
 
+struct Maps {
+  CUtensorMap a[kMaxProb], w[kMaxProb], w_half;   // w_half: 128-entry boxes of w[0] (single product only)
+};
+
 __global__ void __launch_bounds__(kThreads, 1)
-lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
-                      const __grid_constant__ CUtensorMap tm_w_half, const Params p) {
+lm_head_argmax_kernel(const __grid_constant__ Maps tm, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) unsigned long long s_bar[2 * kStages + 5];
   __shared__ uint32_t s_tmem;
@@ -117,7 +123,11 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     fence_async_smem();
   }
   if (warp == 1) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
-  if (tid == 64) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_w); tma_prefetch_desc(&tm_w_half); }
+  if (tid >= 64 && tid < 64 + p.n_prob) {
+    tma_prefetch_desc(&tm.a[tid - 64]);
+    tma_prefetch_desc(&tm.w[tid - 64]);
+    if (tid == 64) tma_prefetch_desc(&tm.w_half);
+  }
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   if (p.a_tile_bytes < kATile) {
     // a box of fewer than 128 rows leaves the rest of the operand tile as it was: make that zeros
@@ -138,7 +148,10 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   auto sA = [&](int s, int mt) { return smem_base + (uint32_t)s * kStageBytes + (uint32_t)mt * kATile; };
   auto sW = [&](int s) { return smem_base + (uint32_t)s * kStageBytes + 2 * kATile; };
 
-  const int n_items = p.n_items * p.k_splits;   // (tile, row block, part of the K axis)
+  // work item -> (tile and row block, part of the K axis, product): products innermost, so that
+  // blocks working side by side read different weights
+  const int per_tile = p.k_splits * p.n_prob;
+  const int n_items = p.n_items * per_tile;
   const int k_chunks = p.K / BK / p.k_splits;
   int issued = 0;  // ring stages filled by the producer (for the drain)
 
@@ -148,8 +161,9 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       bool ok = true;
       int it = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item wi = decode_item(p, item / p.k_splits);
-        const int kc0 = (item % p.k_splits) * k_chunks;
+        const Item wi = decode_item(p, item / per_tile);
+        const int sub = item % per_tile, prob = sub % p.n_prob;
+        const int kc0 = (sub / p.n_prob) * k_chunks;
         const int mb = wi.mb;
         const int rows_left = p.M - mb * MB;
         const int m_tiles = rows_left > BM ? 2 : 1;
@@ -159,9 +173,9 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
           if (it >= kStages) ok = mbar_wait(bar_empty(s), ((it / kStages) - 1) & 1, abort_flag, wlim);
           if (!ok) break;
           mbar_expect_tx(bar_full(s), w_bytes + (uint32_t)m_tiles * p.a_tile_bytes);
-          tma_load_2d(sW(s), wi.cols == BN ? &tm_w : &tm_w_half, (kc0 + kc) * BK, wi.col0, bar_full(s));
+          tma_load_2d(sW(s), wi.cols == BN ? &tm.w[prob] : &tm.w_half, (kc0 + kc) * BK, wi.col0, bar_full(s));
           for (int mt = 0; mt < m_tiles; ++mt)
-            tma_load_2d(sA(s, mt), &tm_a, (kc0 + kc) * BK, mb * MB + mt * BM, bar_full(s));
+            tma_load_2d(sA(s, mt), &tm.a[prob], (kc0 + kc) * BK, mb * MB + mt * BM, bar_full(s));
           issued = it + 1;
         }
       }
@@ -172,7 +186,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
       bool ok = true;
       int it = 0, tile = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
-        const Item wi = decode_item(p, item / p.k_splits);
+        const Item wi = decode_item(p, item / per_tile);
         const int m_tiles = (p.M - wi.mb * MB) > BM ? 2 : 1;
         const uint32_t idesc = wi.cols == BN ? kIdesc : kIdescHalf;
         const int acc = p.two_acc ? (tile & 1) : 0;          // accumulator (pair) of this tile
@@ -209,8 +223,8 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     bool ok = true;
     int tile = 0;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile) {
-      const Item wi = decode_item(p, item / p.k_splits);
-      const int part = item % p.k_splits;
+      const Item wi = decode_item(p, item / per_tile);
+      const int sub = item % per_tile, prob = sub % p.n_prob, part = sub / p.n_prob;
       const int mb = wi.mb;
       if (p.two_acc && (tile & 1) != mt) continue;   // the other group's tile
       const int acc = p.two_acc ? mt : 0;
@@ -233,11 +247,15 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
           tmem_wait_ld();
           if (p.out != nullptr) {   // plain product: this row's 32 values (+ bias) go to memory
             if (row_valid) {
-              float* dst = p.out + part * p.out_split_stride + (int64_t)row * p.ld_out + col0 + c;
-              const bool add_bias = p.bias != nullptr && part == 0;
+              const uint16_t* bias = p.biases[0];
+              float* dst = p.outs[0];
+              if (prob == 1) { bias = p.biases[1]; dst = p.outs[1]; }
+              if (prob == 2) { bias = p.biases[2]; dst = p.outs[2]; }
+              dst += part * p.out_split_stride + (int64_t)row * p.ld_out + col0 + c;
+              const bool add_bias = bias != nullptr && part == 0;
               if (p.out_vec && col0 + c + 32 <= p.V) {   // 128 bytes of this row in eight stores
                 if (add_bias) {
-                  const uint4* b4 = reinterpret_cast<const uint4*>(p.bias + col0 + c);
+                  const uint4* b4 = reinterpret_cast<const uint4*>(bias + col0 + c);
 #pragma unroll
                   for (int j = 0; j < 4; ++j) {
                     const uint4 b = b4[j];
@@ -258,7 +276,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                 for (int j = 0; j < 32; ++j) {
                   if (col0 + c + j >= p.V) continue;
                   float v = __uint_as_float(x[j]);
-                  if (add_bias) v += __uint_as_float((uint32_t)p.bias[col0 + c + j] << 16);
+                  if (add_bias) v += __uint_as_float((uint32_t)bias[col0 + c + j] << 16);
                   dst[j] = v;
                 }
               }
@@ -313,7 +331,10 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
   if (!s_last) return;
   // the last block turns the keys into indices and leaves keys and counters zero for the next call
   __threadfence();
-  if (tid == 0) *p.status = atomicExch(p.aborts, 0u) ? (int)CLV_ERR_TIMEOUT : (int)CLV_OK;
+  if (tid == 0) {   // one status word per product
+    const int verdict = atomicExch(p.aborts, 0u) ? (int)CLV_ERR_TIMEOUT : (int)CLV_OK;
+    for (int i = 0; i < p.n_prob; ++i) p.status[i] = verdict;
+  }
   if (p.out != nullptr) return;   // no keys were written
   for (int r = tid; r < p.M; r += kThreads) {
     const unsigned long long key = atomicExch(p.keys + r, 0ull);
@@ -343,36 +364,51 @@ bool lm_head_supported(int rows, int hidden, int vocab) {
 }
 
 namespace {
-cudaError_t launch_rows_times_weights(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
-                                      int rows, int hidden_dim, int vocab, int32_t* ids, float* out, int64_t ld_out,
-                                      const void* bias, int k_splits, int64_t out_split_stride, int32_t* status,
-                                      unsigned* tickets, cudaStream_t stream) {
+struct Product {   // one product of a launch: rows x[rows, K] times weight[vocab, K]^T (+ bias) -> out
+  const void* x;
+  const void* weight;
+  const void* bias;
+  float* out;
+};
+
+cudaError_t launch_rows_times_weights(int n_prob, const Product* pr, int64_t ld_hidden, int64_t ld_weight, int rows,
+                                      int hidden_dim, int vocab, int32_t* ids, int64_t ld_out, int k_splits,
+                                      int64_t out_split_stride, int32_t* status, unsigned* tickets,
+                                      cudaStream_t stream) {
   static OncePerDevice once;
   cudaError_t e0 = run_once_per_device(once, [] {
     return cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
   });
   if (e0 != cudaSuccess) return e0;
-  CUtensorMap tm_a, tm_w, tm_w_half;
+  if (n_prob < 1 || n_prob > kMaxProb) return cudaErrorInvalidValue;
+  Maps tm;
   int a_box = BM;   // rows one load of the row operand brings: the power of two that covers them, 8..128
   while (a_box > 8 && a_box / 2 >= rows) a_box /= 2;
-  if (!make_map_2d(&tm_a, hidden, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, (uint32_t)a_box) ||
-      !make_map_2d(&tm_w, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN) ||
-      !make_map_2d(&tm_w_half, weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN / 2))
-    return cudaErrorInvalidValue;
   Params p;
+  bool vec = (ld_out % 4) == 0 && (out_split_stride % 4) == 0;
+  for (int i = 0; i < kMaxProb; ++i) {
+    const Product& q = pr[i < n_prob ? i : 0];   // unused slots repeat the first product
+    if (!make_map_2d(&tm.a[i], q.x, (uint64_t)rows, (uint64_t)hidden_dim, ld_hidden, (uint32_t)a_box) ||
+        !make_map_2d(&tm.w[i], q.weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN))
+      return cudaErrorInvalidValue;
+    p.outs[i] = q.out;
+    p.biases[i] = static_cast<const uint16_t*>(q.bias);
+    vec = vec && (reinterpret_cast<uintptr_t>(q.out) % 16) == 0 && (reinterpret_cast<uintptr_t>(q.bias) % 16) == 0;
+  }
+  if (!make_map_2d(&tm.w_half, pr[0].weight, (uint64_t)vocab, (uint64_t)hidden_dim, ld_weight, BN / 2))
+    return cudaErrorInvalidValue;
   p.M = rows;
   p.K = hidden_dim;
   p.V = vocab;
   p.n_tiles = (vocab + BN - 1) / BN;
   p.m_blocks = (rows + MB - 1) / MB;
   p.ids = ids;
-  p.out = out;
+  p.out = pr[0].out;
+  p.n_prob = n_prob;
   p.ld_out = ld_out;
-  p.bias = static_cast<const uint16_t*>(bias);
   p.k_splits = k_splits;
   p.out_split_stride = out_split_stride;
-  p.out_vec = out != nullptr && (reinterpret_cast<uintptr_t>(out) % 16) == 0 && (ld_out % 4) == 0 &&
-              (out_split_stride % 4) == 0 && (reinterpret_cast<uintptr_t>(bias) % 16) == 0;
+  p.out_vec = p.out != nullptr && vec;
   p.two_acc = rows <= BM;
   p.a_tile_bytes = (uint32_t)a_box * BK * 2;
   p.counter = tickets;
@@ -381,10 +417,10 @@ cudaError_t launch_rows_times_weights(const void* hidden, int64_t ld_hidden, con
   p.status = status;
   p.wait_limit = wait_limit_cycles();
   const int tiles = p.n_tiles * p.m_blocks;
-  const int work = tiles * k_splits;
+  const int work = tiles * k_splits * n_prob;
   const int grid = work < sm_count() ? work : sm_count();
   const int rem = tiles % grid;   // tiles of the last, incomplete round
-  const int split = (k_splits == 1 && rem > 0 && 2 * rem <= grid) ? rem : 0;
+  const int split = (k_splits == 1 && n_prob == 1 && rem > 0 && 2 * rem <= grid) ? rem : 0;
   p.full_items = tiles - split;
   p.n_items = tiles + split;
   cudaLaunchConfig_t cfg = {};
@@ -397,34 +433,42 @@ cudaError_t launch_rows_times_weights(const void* hidden, int64_t ld_hidden, con
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, lm_head_argmax_kernel, tm_a, tm_w, tm_w_half, p);
+  return cudaLaunchKernelEx(&cfg, lm_head_argmax_kernel, tm, p);
 }
 }  // namespace
 
 cudaError_t launch_lm_head_argmax(const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
                                   int rows, int hidden_dim, int vocab, int32_t* ids, int32_t* status,
                                   unsigned* tickets, cudaStream_t stream) {
-  return launch_rows_times_weights(hidden, ld_hidden, weight, ld_weight, rows, hidden_dim, vocab, ids, nullptr, 0,
-                                   nullptr, 1, 0, status, tickets, stream);
+  const Product pr = {hidden, weight, nullptr, nullptr};
+  return launch_rows_times_weights(1, &pr, ld_hidden, ld_weight, rows, hidden_dim, vocab, ids, 0, 1, 0, status,
+                                   tickets, stream);
 }
 
 // How many parts the K axis of a product with few output features is cut into, so that the launch
 // covers the machine: a power of two up to 8 that divides the number of 64-wide K chunks.
-int rows_linear_splits(int rows, int in_dim, int out_dim) {
-  const int tiles = ((out_dim + BN - 1) / BN) * ((rows + MB - 1) / MB);
+// `n` products of one shape share the launch; up to three rounds of blocks are accepted.
+int rows_linear_splits(int rows, int in_dim, int out_dim, int n) {
+  const int tiles = ((out_dim + BN - 1) / BN) * ((rows + MB - 1) / MB) * n;
   int s = 1;
-  while (s < 8 && tiles * s * 2 <= sm_count() && (in_dim / BK) % (s * 2) == 0) s *= 2;
+  while (s < 8 && tiles * s * 2 <= 3 * sm_count() && (in_dim / BK) % (s * 2) == 0) s *= 2;
   return s;
 }
 
-// out[part][r][o] = sum over part's share of k of x[r][k] * weight[o][k] (+ bias[o] in part 0):
-// the same kernel with its accumulators written out (fp32) instead of reduced to an argmax.  The
-// reader adds the `splits` parts up (a fixed order: the result does not depend on scheduling).
-cudaError_t launch_rows_linear(const void* x, int64_t ld_x, const void* weight, int64_t ld_weight, const void* bias,
-                               int rows, int in_dim, int out_dim, float* out, int64_t ld_out, int splits,
-                               int64_t split_stride, int32_t* status, unsigned* tickets, cudaStream_t stream) {
-  return launch_rows_times_weights(x, ld_x, weight, ld_weight, rows, in_dim, out_dim, nullptr, out, ld_out, bias,
-                                   splits, split_stride, status, tickets, stream);
+// out[i][part][r][o] = sum over part's share of k of x[i][r][k] * weight[i][o][k] (+ bias[i][o] in
+// part 0) for n products of one shape (n <= 3) in one launch: the same kernel with its
+// accumulators written out (fp32) instead of reduced to an argmax.  The reader adds the `splits`
+// parts up (a fixed order: the result does not depend on scheduling).  status gets one word per
+// product.
+cudaError_t launch_rows_linear(int n, const void* const* x, int64_t ld_x, const void* const* weight,
+                               int64_t ld_weight, const void* const* bias, int rows, int in_dim, int out_dim,
+                               float* const* out, int64_t ld_out, int splits, int64_t split_stride, int32_t* status,
+                               unsigned* tickets, cudaStream_t stream) {
+  if (n < 1 || n > kMaxProb) return cudaErrorInvalidValue;
+  Product pr[kMaxProb];
+  for (int i = 0; i < n; ++i) pr[i] = Product{x[i], weight[i], bias[i], out[i]};
+  return launch_rows_times_weights(n, pr, ld_x, ld_weight, rows, in_dim, out_dim, nullptr, ld_out, splits,
+                                   split_stride, status, tickets, stream);
 }
 
 }  // namespace clv
