@@ -204,7 +204,8 @@ clv_status clv_accept_walk_commit(const clv_shape* shape, const clv_kv_cache* ca
  * without any probability mass).  Arithmetic: fp32 with hardware exp2; a decision whose uniform
  * lies within rounding distance of its threshold (relative 1e-5) may fall either way.
  * workspace: as returned by clv_workspace_bytes for this shape (with vocab set), initialised.
- * Errors: CLV_ERR_NULL, CLV_ERR_SHAPE (also temperature <= 0), CLV_ERR_ALIGN, CLV_ERR_WORKSPACE.
+ * Errors: CLV_ERR_NULL, CLV_ERR_SHAPE (also temperature <= 0), CLV_ERR_ALIGN, CLV_ERR_WORKSPACE,
+ * CLV_ERR_UNSUPPORTED (vocab above 1048576, or too many rows).
  */
 clv_status clv_accept_sample(const clv_shape* shape,
                              const void* logits, /* bf16 [B*N, ld] */

@@ -9,12 +9,13 @@
 // none) the next token is the first v, in vocabulary order and not struck, whose running sum of p
 // exceeds u[N] * (what is left).  The uniforms are the caller's.
 //
-// Two launches.  (1) One pass over all logits (an HBM stream like the argmax): every block
-// reduces a piece of a row to (maximum, sum of exponentials relative to it) with an online
-// update, in base-2 units.  (2) One block per sequence walks the tree: per level it combines the
-// pieces of the current row, fetches the logits of all children's tokens at once (one round trip
-// to memory), and one thread runs the accept chain; the final draw sums 256 slices of the row,
-// locates the slice by a running sum and then scans that slice with the whole block.
+// Two launches.  (1) One pass over all logits (an HBM stream like the argmax): every warp
+// reduces a slice of 4096 consecutive logits of a row to (maximum, sum of exponentials relative
+// to it) with an online update, in base-2 units.  (2) One block per sequence walks the tree: per
+// level it combines the slices of the current row, fetches the logits of all children's tokens
+// at once (one round trip to memory), and one thread runs the accept chain; the final draw
+// locates the slice by a running sum over the slices' weights (the weights of struck tokens
+// taken out) and then scans that one slice with the whole block, 16 logits per thread.
 #include <limits.h>
 #include <math.h>
 
@@ -26,6 +27,9 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kPiece = 32768;   // logits per block of the statistics pass (64 KB)
 constexpr int kUnroll = 8;
+constexpr int kSlice = kPiece / (kThreads / 32);   // 4096 logits per warp: the unit of the running sums
+constexpr int kPerThread = kSlice / kThreads;       // 16: what a thread scans of the chosen slice
+static_assert(kSlice == 4096 && kPerThread == 16, "a slice is scanned in one round of the block");
 
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {
   uint4 r;
@@ -67,12 +71,37 @@ __device__ __forceinline__ void stat_take8(Stat& st, const uint4& w, float k) {
   }
 }
 
+// A batch of kUnroll vectors at once: one maximum and at most one rescale for the 64 values, then
+// their exponentials into four running sums (no long chain of dependent additions).
+__device__ __forceinline__ void stat_take_batch(Stat& st, const uint4 (&w)[kUnroll], float k) {
+  float mx = -INFINITY;
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    const uint32_t r[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) mx = fmaxf(mx, fmaxf(bf16_lo(r[j]) * k, bf16_hi(r[j]) * k));   // NaN operands are dropped
+  }
+  if (!(mx > -INFINITY)) return;   // nothing but -inf (or NaN): no mass
+  if (mx > st.m) { st.s *= ex2(st.m - mx); st.m = mx; }
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    const uint32_t r[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = bf16_lo(r[j]) * k, b = bf16_hi(r[j]) * k;
+      acc[j] += ((a == a) ? ex2(a - st.m) : 0.f) + ((b == b) ? ex2(b - st.m) : 0.f);   // a NaN logit carries no mass
+    }
+  }
+  st.s += (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
 struct StatParams {
   const uint16_t* logits;
   int64_t ld;
   int vocab, pieces;
   float k;           // log2(e) / T
-  float2* partial;   // [rows][pieces]
+  float2* partial;   // [rows][pieces * 8]: one (maximum, sum) per slice
 };
 
 __global__ void __launch_bounds__(kThreads) softmax_stats_kernel(StatParams p) {
@@ -83,21 +112,22 @@ __global__ void __launch_bounds__(kThreads) softmax_stats_kernel(StatParams p) {
   const uint16_t* base = p.logits + (int64_t)row * p.ld;
   const int nvec = (end - begin) >> 3;
   const uint4* vp = reinterpret_cast<const uint4*>(base + begin);
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   cudaGridDependencySynchronize();
+  // warp w takes the vectors [512 w, 512 (w + 1)) of the piece: 4096 consecutive logits
   Stat st = {-INFINITY, 0.f};
-  int i = tid;
-  for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
+  const int lim = min(nvec, (warp + 1) * (kSlice / 8));
+  int i = warp * (kSlice / 8) + lane;
+  for (; i + (kUnroll - 1) * 32 < lim; i += kUnroll * 32) {
     uint4 w[kUnroll];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) w[u] = ld_stream16(vp + i + u * kThreads);
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) stat_take8(st, w[u], p.k);
+    for (int u = 0; u < kUnroll; ++u) w[u] = ld_stream16(vp + i + u * 32);
+    stat_take_batch(st, w, p.k);
   }
-  for (; i < nvec; i += kThreads) stat_take8(st, ld_stream16(vp + i), p.k);
-  {  // ragged end of the row: at most 7 scalars
-    const int t0 = begin + 8 * nvec + tid;
-    if (t0 < end) {
+  for (; i < lim; i += 32) stat_take8(st, ld_stream16(vp + i), p.k);
+  {  // ragged end of the row: at most 7 scalars, taken by the warp whose slice holds them
+    const int t0 = begin + 8 * nvec + lane;
+    if (t0 < end && (t0 - begin) / kSlice == warp) {
       const float x = __uint_as_float((uint32_t)base[t0] << 16) * p.k;
       if (x > -INFINITY) { Stat one = {x, 1.f}; stat_merge(st, one); }
     }
@@ -107,12 +137,7 @@ __global__ void __launch_bounds__(kThreads) softmax_stats_kernel(StatParams p) {
     Stat other = {__shfl_xor_sync(0xFFFFFFFFu, st.m, o), __shfl_xor_sync(0xFFFFFFFFu, st.s, o)};
     stat_merge(st, other);
   }
-  __shared__ float sm[kThreads / 32], ss[kThreads / 32];
-  if ((tid & 31) == 0) { sm[tid >> 5] = st.m; ss[tid >> 5] = st.s; }
-  __syncthreads();
-  if (tid != 0) return;
-  for (int w = 1; w < kThreads / 32; ++w) { Stat other = {sm[w], ss[w]}; stat_merge(st, other); }
-  p.partial[(int64_t)row * p.pieces + piece] = make_float2(st.m, st.s);
+  if (lane == 0) p.partial[((int64_t)row * p.pieces + piece) * (kThreads / 32) + warp] = make_float2(st.m, st.s);
 }
 
 struct WalkParams {
@@ -137,6 +162,7 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
   __shared__ float s_m, s_S, s_before, s_target;
   __shared__ int s_found, s_bad, s_pick, s_lastv;
   const int b = blockIdx.x, tid = threadIdx.x, N = p.N;
+  const int n_sl = p.pieces * (kPiece / kSlice);   // slices of a row
   const int64_t o = (int64_t)b * N;
   cudaGridDependencySynchronize();
   if (tid == 0) s_bad = (p.path_cap < 1) ? 1 : 0;
@@ -156,8 +182,8 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
     // ---- the current row's maximum and sum from its pieces
     if (tid < 32) {
       Stat a = {-INFINITY, 0.f};
-      for (int i = tid; i < p.pieces; i += 32) {
-        const float2 v = p.partial[(o + cur) * p.pieces + i];
+      for (int i = tid; i < n_sl; i += 32) {
+        const float2 v = p.partial[(o + cur) * n_sl + i];
         Stat other = {v.x, v.y};
         stat_merge(a, other);
       }
@@ -210,36 +236,19 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
   }
   if (!bad) {
     // ---- draw the next token from what is left of row `cur`: all of its children were rejected,
-    //      their tokens are struck.  256 slices of the row, each a multiple of 8 logits.
+    //      their tokens are struck.  The slices' weights come from the statistics pass.
     const float m = s_m;
     const uint16_t* row = p.logits + (o + cur) * p.ld;
-    const int per = ((p.vocab + kThreads - 1) / kThreads + 7) & ~7;
-    const int v0 = min(p.vocab, tid * per), v1 = min(p.vocab, v0 + per);
     auto weight = [&](int v) -> float {
       const float l = __uint_as_float((uint32_t)row[v] << 16) * p.k;
       return (l == l && m > -INFINITY) ? ex2(l - m) : 0.f;
     };
-    // the slice's sum with 16-byte reads, four in flight (v0 is a multiple of 8, rows are 16-byte
-    // aligned); the weights of struck tokens inside the slice are taken out again afterwards
-    float sum = 0.f;
-    {
-      int v = v0;
-      for (; v + 32 <= v1; v += 32) {
-        uint4 w[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) w[q] = *reinterpret_cast<const uint4*>(row + v + 8 * q);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float x[8] = {bf16_lo(w[q].x), bf16_hi(w[q].x), bf16_lo(w[q].y), bf16_hi(w[q].y),
-                              bf16_lo(w[q].z), bf16_hi(w[q].z), bf16_lo(w[q].w), bf16_hi(w[q].w)};
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float l = x[j] * p.k;
-            sum += (l == l && m > -INFINITY) ? ex2(l - m) : 0.f;
-          }
-        }
-      }
-      for (; v < v1; ++v) sum += weight(v);
+    // what is left, slice by slice (the first pass's sums minus the struck weights differ from a
+    // fresh sum by rounding only); thread 0 walks the slices in vocabulary order
+    for (int j = tid; j < n_sl; j += kThreads) {
+      const float2 sl = p.partial[(o + cur) * n_sl + j];
+      float sum = (sl.x > -INFINITY && m > -INFINITY) ? sl.y * ex2(sl.x - m) : 0.f;
+      const int v0 = j * kSlice, v1 = min(p.vocab, v0 + kSlice);
       for (int c = cur + 1; c < N; ++c) {
         if (sp[c] != cur || st[c] < v0 || st[c] >= v1) continue;
         bool repeat = false;   // a token carried by two siblings is struck once
@@ -247,18 +256,17 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
         if (!repeat) sum -= weight(st[c]);
       }
       sum = fmaxf(sum, 0.f);
+      if (j < kThreads) s_slice[j] = sum;
     }
-    s_slice[tid] = sum;
     __syncthreads();
     if (tid == 0) {
-      // what is left, by the sums of this pass (the first pass's sum minus the rejected weights
-      // differs from it by rounding only)
+      const int n_here = n_sl;   // at most one slice per thread: larger vocabularies are refused by the host
       float total = 0.f;
-      for (int j = 0; j < kThreads; ++j) total += s_slice[j];
+      for (int j = 0; j < n_here; ++j) total += s_slice[j];
       const float target = su[N] * total;
       float run = 0.f;
       int pick = -1, last = -1;
-      for (int j = 0; j < kThreads; ++j) {
+      for (int j = 0; j < n_here; ++j) {
         if (s_slice[j] > 0.f) last = j;
         if (pick < 0 && s_slice[j] > 0.f && run + s_slice[j] > target) { pick = j; s_before = run; }
         if (pick < 0) run += s_slice[j];
@@ -275,40 +283,60 @@ __global__ void __launch_bounds__(kThreads) sample_walk_kernel(WalkParams p) {
     __syncthreads();
     const int pick = s_pick;
     if (pick >= 0) {
-      // ---- the whole block walks the chosen slice, 256 elements at a time: weights, a running sum
-      //      across the block (warp scans + the warps' totals), the first element past the target
+      // ---- the whole block scans the chosen slice in one round: a thread takes 16 consecutive
+      //      logits (two 16-byte reads), strikes the children's tokens among them, adds them up;
+      //      a running sum across the block (warp scan + the warps' totals) gives every thread
+      //      its start, and the first element whose running sum exceeds the target wins
       const float target = s_target;
-      const int q0 = min(p.vocab, pick * per), q1 = min(p.vocab, q0 + per);
+      const int q0 = pick * kSlice, q1 = min(p.vocab, q0 + kSlice);
       const int lane = tid & 31, warp = tid >> 5;
-      float before = s_before;
-      for (int base = q0; base < q1; base += kThreads) {
-        const int v = base + tid;
-        float e = 0.f;
-        if (v < q1) {
-          bool hit = false;
-          for (int c = cur + 1; c < N; ++c) hit |= (sp[c] == cur && st[c] == v);
-          e = hit ? 0.f : weight(v);
-        }
-        float incl = e;
+      const int v_base = q0 + tid * kPerThread;
+      float e[kPerThread];
+      {
+        uint4 w[2];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const float up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-          if (lane >= off) incl += up;
+        for (int h = 0; h < 2; ++h)   // past the row's end: the last vector again (cut by index below)
+          w[h] = ld_stream16(row + min(v_base + 8 * h, (q1 - 1) & ~7));
+        uint32_t struck = 0;
+        for (int c = cur + 1; c < N; ++c)
+          if (sp[c] == cur && st[c] >= v_base && st[c] < v_base + kPerThread) struck |= 1u << (st[c] - v_base);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float x[8] = {bf16_lo(w[h].x), bf16_hi(w[h].x), bf16_lo(w[h].y), bf16_hi(w[h].y),
+                              bf16_lo(w[h].z), bf16_hi(w[h].z), bf16_lo(w[h].w), bf16_hi(w[h].w)};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float l = x[j] * p.k;
+            const bool in = (v_base + 8 * h + j < q1) && !((struck >> (8 * h + j)) & 1u) && l == l && m > -INFINITY;
+            e[8 * h + j] = in ? ex2(l - m) : 0.f;
+          }
         }
-        if (lane == 31) s_slice[warp] = incl;
-        __syncthreads();
-        float wbase = before;
-        for (int w = 0; w < warp; ++w) wbase += s_slice[w];
-        float round_total = 0.f;
-        for (int w = 0; w < kThreads / 32; ++w) round_total += s_slice[w];
-        if (e > 0.f) {
-          atomicMax(&s_lastv, v);
-          if (wbase + incl > target) atomicMin(&s_found, v);
-        }
-        __syncthreads();
-        if (s_found != INT_MAX) break;   // same verdict in every thread
-        before += round_total;
       }
+      float mine = 0.f;
+#pragma unroll
+      for (int j = 0; j < kPerThread; ++j) mine += e[j];
+      float incl = mine;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const float up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+      }
+      if (lane == 31) s_slice[warp] = incl;
+      __syncthreads();
+      float run = s_before + (incl - mine);   // the running sum before this thread's first element
+      for (int w = 0; w < warp; ++w) run += s_slice[w];
+      int first = INT_MAX, lastv = -1;
+#pragma unroll
+      for (int j = 0; j < kPerThread; ++j) {
+        run += e[j];
+        if (e[j] > 0.f) {
+          lastv = v_base + j;
+          if (first == INT_MAX && run > target) first = v_base + j;
+        }
+      }
+      if (lastv >= 0) atomicMax(&s_lastv, lastv);
+      if (first != INT_MAX) atomicMin(&s_found, first);
+      __syncthreads();
       if (tid == 0) p.next_token[b] = (s_found != INT_MAX) ? s_found : s_lastv;
     } else if (tid == 0) {
       p.next_token[b] = -1;   // a row without any mass
@@ -329,7 +357,11 @@ int sample_pieces(int vocab) { return (vocab + kPiece - 1) / kPiece; }
 
 }  // namespace
 
-size_t sample_scratch_bytes(int rows, int vocab) { return sizeof(float2) * (size_t)rows * sample_pieces(vocab); }
+int sample_max_vocab() { return kThreads * kSlice; }   // one slice per thread of the walk's block
+
+size_t sample_scratch_bytes(int rows, int vocab) {
+  return sizeof(float2) * (size_t)rows * sample_pieces(vocab) * (kPiece / kSlice);
+}
 
 cudaError_t launch_accept_sample(const clv_shape& s, const void* logits, int64_t ld, const int32_t* parent,
                                  const int32_t* tokens, const float* uniforms, float temperature,

@@ -237,7 +237,7 @@ clv_status clv_accept_sample(const clv_shape* shape, const void* logits, int64_t
   if (!(temperature > 0.0f) || !(temperature < INFINITY)) return CLV_ERR_SHAPE;
   if (!aligned16(logits) || (ld % 8) != 0) return CLV_ERR_ALIGN;
   const int64_t rows = (int64_t)shape->batch * shape->n_nodes;
-  if (rows > INT32_MAX / 64) return CLV_ERR_UNSUPPORTED;
+  if (rows > INT32_MAX / 64 || shape->vocab > sample_max_vocab()) return CLV_ERR_UNSUPPORTED;
   const size_t need = kWsFixedBytes + sample_scratch_bytes((int)rows, shape->vocab);
   if (!workspace || workspace_bytes < need) return CLV_ERR_WORKSPACE;
   if (!aligned16(workspace)) return CLV_ERR_ALIGN;

@@ -41,6 +41,7 @@ cudaError_t launch_argmax_static(const void* logits, int64_t ld, int rows, int v
                                  cudaStream_t stream);
 
 // ---- stochastic acceptance (temperature > 0): statistics pass over the logits + per-sequence walk
+int sample_max_vocab();
 size_t sample_scratch_bytes(int rows, int vocab);
 cudaError_t launch_accept_sample(const clv_shape& s, const void* logits, int64_t ld, const int32_t* parent,
                                  const int32_t* tokens, const float* uniforms, float temperature,

@@ -92,7 +92,8 @@ def compare(oracle, got, lg, vocab, parent, tokens, u, temperature, path_cap, mi
 
 
 @pytest.mark.parametrize("temperature", [1.0, 0.6, 1.7])
-@pytest.mark.parametrize("vocab,n_nodes", [(64, 9), (1000, 20), (4099, 33), (32000, 64), (128256, 64)])
+@pytest.mark.parametrize("vocab,n_nodes", [(64, 9), (1000, 20), (4099, 33), (8192, 10), (32000, 64), (32771, 12),
+                                           (128256, 64)])   # around the edges of the 4096-logit slices and 32768-logit pieces
 def test_sample_random_trees(clv, oracle, vocab, n_nodes, temperature):
     B = 6 if vocab > 100000 else 24
     cfg = W.small_config(batch=B, n_nodes=n_nodes, vocab=vocab, seed=W.BASE_SEED + vocab + n_nodes)
