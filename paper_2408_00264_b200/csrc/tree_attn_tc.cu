@@ -67,6 +67,7 @@ struct Params {
   int B, N, Hq, Hkv, G;
   int paged, cap_tokens, n_pages, max_pages;
   int longest_first;  // hand out sequences in order of decreasing context length
+  int pair_boxes;     // the 4-D tensor maps exist: a whole 128-key tile of a contiguous cache is one copy
   int tiles;       // row tiles per (sequence, kv head); each is worked by one cluster
   int splits;      // blocks along the key axis = cluster size
   float scale_log2;
@@ -154,7 +155,8 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                     const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
-                    const __grid_constant__ CUtensorMap tm_vt, const Params p) {
+                    const __grid_constant__ CUtensorMap tm_vt, const __grid_constant__ CUtensorMap tm_kc2,
+                    const __grid_constant__ CUtensorMap tm_vc2, const Params p) {
   constexpr int KST = Cfg::KST, VST = Cfg::VST;
   constexpr uint32_t kStage = Cfg::kStage;
   constexpr uint32_t kHalf = kStage / 2;    // a stage holds [64-wide half of d][128 keys][64 d]
@@ -211,6 +213,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (tid == 64) {
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc);
     tma_prefetch_desc(&tm_kt); tma_prefetch_desc(&tm_vt);
+    if (p.pair_boxes) { tma_prefetch_desc(&tm_kc2); tma_prefetch_desc(&tm_vc2); }
   }
   cudaGridDependencySynchronize();
 
@@ -232,18 +235,105 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     b = s_seq;
   }
 
-  // ---- per-sequence checks ------------------------------------------------------------------
+  // ---- the sequence's length, this block's range of the key axis ------------------------------
+  // The key axis is cut in 64-key pieces: p_cache pieces of context, then the tree's own pieces.
+  // A split takes a contiguous range of pieces and walks it in tiles of two pieces; the last tile
+  // of a range may hold one piece only.
   const int L = p.ctx_len[b];
-  bool bad = false;
-  for (int i = tid; i < N; i += kThreads) {
+  const bool len_bad = (L < 0) || (p.paged ? ((L + PG - 1) / PG > p.max_pages) : (L > p.cap_tokens));
+  const int p_cache = (!len_bad && L > 0) ? (L + PG - 1) / PG : 0;  // 64-key pieces (pages) of the context
+  const int p_total = p_cache + (N + PG - 1) / PG;
+  const int pc_begin = (int)((unsigned)split * (unsigned)p_total / (unsigned)p.splits);
+  const int pc_end = (int)((unsigned)(split + 1) * (unsigned)p_total / (unsigned)p.splits);
+  const int T = (pc_end - pc_begin + PPT - 1) / PPT;   // tiles of this block
+
+  // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = smem_base;
+  const uint32_t sK = sQ + kQTile;           // ring of KST K stages
+  const uint32_t sV = sK + KST * kStage;     // ring of VST V stages
+  uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
+
+  volatile int* abort_flag = &s_abort;
+  const long long wlim = p.wait_limit;
+
+  // ---- the producer's two steps (whole warp 0): the copies of K tile kt / V tile vt.  Lane j
+  //      caches the pool page of context piece (base + j) for each ring (paged cache).
+  int issued_k = 0, issued_v = 0;  // bookkeeping for the drain
+  int pk_page = 0, pk_base = -64, pv_page = 0, pv_base = -64;
+  auto issue_tile = [&](int t, bool is_k, int& page, int& page_base) {
+    const int g0 = pc_begin + t * PPT;
+    if (p.paged && g0 < p_cache && g0 + PPT > page_base + 32) {
+      page_base = g0;
+      const int pc = g0 + lane;
+      page = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
+    }
+    int row0[PPT];
+    bool is_tree[PPT];
+#pragma unroll
+    for (int j = 0; j < PPT; ++j) {
+      const int g = g0 + j;
+      int pg = __shfl_sync(0xFFFFFFFFu, page, (g - page_base) & 31);
+      is_tree[j] = g >= p_cache;
+      if (g >= pc_end) row0[j] = -1;     // the range ended inside this tile
+      else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
+      else if (p.paged) {
+        if (pg < 0 || pg >= p.n_pages) pg = 0;   // the reporter flags the sequence; any page will do
+        row0[j] = pg * PG;
+      } else row0[j] = b * p.cap_tokens + g * PG;
+    }
+    if (lane == 0) {
+      const int st = is_k ? t % KST : t % VST;
+      const uint32_t full = is_k ? bar(B_KF + st) : bar(B_VF + st);
+      const uint32_t stage = (is_k ? sK : sV) + (uint32_t)st * kStage;
+      if (p.pair_boxes && row0[0] >= 0 && !is_tree[1] && row0[1] == row0[0] + PG) {
+        // both pieces are neighbours in the cache: the whole tile, both halves of d, in one copy
+        mbar_expect_tx(full, kStage);
+        tma_load_4d(stage, is_k ? &tm_kc2 : &tm_vc2, 0, row0[0], 0, kvh, full);
+      } else {
+        int n_pieces = 0;
+#pragma unroll
+        for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
+        mbar_expect_tx(full, (uint32_t)n_pieces * 2u * kPiece);  // 0 bytes: a plain arrival
+#pragma unroll
+        for (int j = 0; j < PPT; ++j) {
+          if (row0[j] < 0) continue;
+          const CUtensorMap* m = is_tree[j] ? (is_k ? &tm_kt : &tm_vt) : (is_k ? &tm_kc : &tm_vc);
+          const uint32_t dst = stage + (uint32_t)j * kPiece;
+          tma_load_3d(dst, m, 0, kvh, row0[j], full);
+          tma_load_3d(dst + kHalf, m, 64, kvh, row0[j], full);
+        }
+      }
+    }
+    if (is_k) issued_k = t + 1;
+    else issued_v = t + 1;
+  };
+  // The Q tile and the first tiles of both rings go out before the block's first barrier: they
+  // need the sequence's length only (a bad length reads the tree's own rows, which exist; the
+  // block then waits for these copies before it leaves).
+  int kt0 = 0, vt0 = 0;
+  if (warp == 0 && T > 0) {
+    if (lane == 0) {
+      mbar_expect_tx(bar(B_Q), (uint32_t)(RT * HD * 2));   // the boxes hold RT rows
+      const int node0 = b * N + tile_idx * (BM / G);
+      tma_load_3d(sQ, &tm_q, 0, kvh * G, node0, bar(B_Q));
+      tma_load_3d(sQ + kQTile / 2, &tm_q, 64, kvh * G, node0, bar(B_Q));
+    }
+    const int nk = min(T, KST), nv = min(T, VST);
+    while (kt0 < nk || vt0 < nv) {
+      if (kt0 < nk) { issue_tile(kt0, true, pk_page, pk_base); ++kt0; }
+      if (vt0 < nv) { issue_tile(vt0, false, pv_page, pv_base); ++vt0; }
+    }
+  }
+
+  // ---- per-sequence checks (the threads of warps 2 and up) ----------------------------------
+  bool bad = len_bad;
+  for (int i = tid - 64; i < N; i += kThreads - 64) {
+    if (i < 0) continue;
     const int par = p.parent[(int64_t)b * N + i];
     s_parent[i] = par;
     bad |= (par < -1 || par >= i);
   }
-  bad |= (L < 0);
-  const int p_cache = L > 0 ? (L + PG - 1) / PG : 0;  // 64-key pieces (pages) of the context
-  if (p.paged) bad |= (p_cache > p.max_pages);
-  else bad |= (L > p.cap_tokens);
   tc_fence_before();
   const int seq_bad = __syncthreads_or(bad ? 1 : 0);  // same verdict in every block of the sequence
   tc_fence_after();
@@ -265,34 +355,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     p.status[b] = (bits & 1u) ? CLV_ERR_TREE : (bits & 2u) ? CLV_ERR_TIMEOUT : CLV_OK;
   };
   auto release_tmem = [&]() { tmem_dealloc(tmem, kTmemCols); };   // warp 1
-  if (seq_bad) {  // the whole cluster leaves together; nothing has been issued yet
+  if (seq_bad) {  // the whole cluster leaves together, once the copies that are under way have landed
+    if (tid == 0) {
+      for (int i = 0; i < kt0; ++i) mbar_drain(bar(B_KF + i), 0);
+      for (int i = 0; i < vt0; ++i) mbar_drain(bar(B_VF + i), 0);
+      if (T > 0) mbar_drain(bar(B_Q), 0);
+    }
     if (warp == 1) release_tmem();
     if (tid == 0) publish(report(1u));
     return;
   }
 
-  // ---- this block's range of the key axis -----------------------------------------------------
-  // The key axis is cut in 64-key pieces: p_cache pieces of context, then the tree's own pieces.
-  // A split takes a contiguous range of pieces and walks it in tiles of two pieces; the last tile
-  // of a range may hold one piece only.
-  const int p_total = p_cache + (N + PG - 1) / PG;
-  const int pc_begin = (int)((int64_t)split * p_total / p.splits);
-  const int pc_end = (int)((int64_t)(split + 1) * p_total / p.splits);
-  const int T = (pc_end - pc_begin + PPT - 1) / PPT;   // tiles of this block
-
-  // ---- shared memory carve-up (1024-byte aligned tiles for the 128-byte swizzle) ------------
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = smem_base;
-  const uint32_t sK = sQ + kQTile;           // ring of KST K stages
-  const uint32_t sV = sK + KST * kStage;     // ring of VST V stages
-  uint8_t* const sV_gen = smem_raw + (sV - smem_u32(smem_raw));
-
-  volatile int* abort_flag = &s_abort;
-  const long long wlim = p.wait_limit;
   auto tmem_S = [&](int buf) { return tmem + (uint32_t)(buf * BN); };   // P overwrites columns 0-31 and 64-95
   const uint32_t tmem_O = tmem + (uint32_t)(NSB * BN);
-
-  int issued_k = 0, issued_v = 0;  // producer bookkeeping for the drain
 
   // per-thread state of the softmax threads (warps 2..9); declared here because the epilogue runs
   // after block-wide synchronisation points that all roles must reach together
@@ -310,59 +385,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (warp == 0) {
     // =========================== TMA producer ===============================================
-    // K and V advance independently: whichever ring has a free buffer gets its next tile.  Lane j
-    // caches the pool page of context piece (base + j) for each ring (paged cache).
-    int kt = 0, vt = 0;
-    int pk_page = 0, pk_base = -64, pv_page = 0, pv_base = -64;
+    // K and V advance independently: whichever ring has a free buffer gets its next tile.
+    int kt = kt0, vt = vt0;
     long long t_idle = clock64();
     bool ok = true;
     while (ok && (kt < T || vt < T)) {
       bool progress = false;
-      // ---- K of tile kt: this block's piece(s)
       if (kt < T) {
         const int st = kt % KST;
         int ready = 1;
         if (kt >= KST && lane == 0) ready = mbar_test(bar(B_SF + st), ((kt / KST) - 1) & 1) ? 1 : 0;
         ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
         if (ready) {
-          const int g0 = pc_begin + kt * PPT;
-          if (p.paged && g0 < p_cache && g0 + PPT > pk_base + 32) {
-            pk_base = g0;
-            const int pc = g0 + lane;
-            pk_page = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
-          }
-          int row0[PPT];
-          bool is_tree[PPT];
-#pragma unroll
-          for (int j = 0; j < PPT; ++j) {
-            const int g = g0 + j;
-            int pg = __shfl_sync(0xFFFFFFFFu, pk_page, (g - pk_base) & 31);
-            is_tree[j] = g >= p_cache;
-            if (g >= pc_end) row0[j] = -1;     // the range ended inside this tile
-            else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
-            else if (p.paged) { if (pg < 0 || pg >= p.n_pages) pg = 0; row0[j] = pg * PG; }
-            else row0[j] = b * p.cap_tokens + g * PG;
-          }
-          if (lane == 0) {
-            int n_pieces = 0;
-#pragma unroll
-            for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
-            mbar_expect_tx(bar(B_KF + st), (uint32_t)n_pieces * 2u * kPiece);  // 0 bytes: a plain arrival
-#pragma unroll
-            for (int j = 0; j < PPT; ++j) {
-              if (row0[j] < 0) continue;
-              const CUtensorMap* mk = is_tree[j] ? &tm_kt : &tm_kc;
-              const uint32_t dst = sK + st * kStage + (uint32_t)j * kPiece;
-              tma_load_3d(dst, mk, 0, kvh, row0[j], bar(B_KF + st));
-              tma_load_3d(dst + kHalf, mk, 64, kvh, row0[j], bar(B_KF + st));
-            }
-          }
+          issue_tile(kt, true, pk_page, pk_base);
           ++kt;
-          issued_k = kt;
           progress = true;
         }
       }
-      // ---- V of tile vt
       if (vt < T) {
         const int st = vt % VST;
         int ready = 1;
@@ -370,42 +409,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           ready = mbar_test(bar(B_VE + st), ((vt / VST) - 1) & 1) ? 1 : 0;
         ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
         if (ready) {
-          const int g0 = pc_begin + vt * PPT;
-          if (p.paged && g0 < p_cache && g0 + PPT > pv_base + 32) {
-            pv_base = g0;
-            const int pc = g0 + lane;
-            pv_page = (pc < p_cache) ? p.block_table[(int64_t)b * p.max_pages + pc] : 0;
-          }
-          int row0[PPT];
-          bool is_tree[PPT];
-#pragma unroll
-          for (int j = 0; j < PPT; ++j) {
-            const int g = g0 + j;
-            int pg = __shfl_sync(0xFFFFFFFFu, pv_page, (g - pv_base) & 31);
-            is_tree[j] = g >= p_cache;
-            if (g >= pc_end) row0[j] = -1;
-            else if (is_tree[j]) row0[j] = b * N + (g - p_cache) * PG;
-            else if (p.paged) {
-              if (pg < 0 || pg >= p.n_pages) pg = 0;   // the reporter flags the sequence; any page will do
-              row0[j] = pg * PG;
-            } else row0[j] = b * p.cap_tokens + g * PG;
-          }
-          if (lane == 0) {
-            int n_pieces = 0;
-#pragma unroll
-            for (int j = 0; j < PPT; ++j) n_pieces += row0[j] >= 0;
-            mbar_expect_tx(bar(B_VF + st), (uint32_t)n_pieces * 2u * kPiece);
-#pragma unroll
-            for (int j = 0; j < PPT; ++j) {
-              if (row0[j] < 0) continue;
-              const CUtensorMap* mv = is_tree[j] ? &tm_vt : &tm_vc;
-              const uint32_t dst = sV + st * kStage + (uint32_t)j * kPiece;
-              tma_load_3d(dst, mv, 0, kvh, row0[j], bar(B_VF + st));
-              tma_load_3d(dst + kHalf, mv, 64, kvh, row0[j], bar(B_VF + st));
-            }
-          }
+          issue_tile(vt, false, pv_page, pv_base);
           ++vt;
-          issued_v = vt;
           progress = true;
         }
       }
@@ -469,12 +474,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   } else {
     // =========================== softmax threads ==============================================
-    if (warp == 2 && T > 0 && lane == 0) {  // the Q tile: issued here so that the producer starts with K/V
-      mbar_expect_tx(bar(B_Q), (uint32_t)(RT * HD * 2));   // the boxes hold RT rows
-      const int node0 = b * N + tile_idx * (BM / G);
-      tma_load_3d(sQ, &tm_q, 0, kvh * G, node0, bar(B_Q));
-      tma_load_3d(sQ + kQTile / 2, &tm_q, 64, kvh * G, node0, bar(B_Q));
-    }
     // ancestor bitsets (row i of the tree's topology matrix), built while the first tiles are on
     // their way; the 256 threads meet at a named barrier of their own
     for (int i = tid - 64; i < N; i += kSoftmaxThreads) {
@@ -855,6 +854,21 @@ bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t heads, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same tensor seen as [rows][heads][2 halves of d][64]: a box of 64 x box_rows x 2 x 1 in the
+// order (d, row, half, head) lands in shared memory as [half][row][64], the layout of a K or V
+// stage, so a tile of 128 neighbouring rows is one copy instead of four.
+bool make_map_halves(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t heads, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {64, rows, 2, heads};
+  const cuuint64_t strides[3] = {(cuuint64_t)HD * 2 * heads, 128, (cuuint64_t)HD * 2};
+  const cuuint32_t box[4] = {64, box_rows, 2, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int row_tiles(const clv_shape& s) {
   const int G = s.n_q_heads / s.n_kv_heads;
   return (s.n_nodes + BM / G - 1) / (BM / G);   // row tiles of BM / G whole nodes
@@ -899,7 +913,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
                                 (int)Cfg::kSmem);
   });
   if (e0 != cudaSuccess) return e0;
-  alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt;
+  alignas(64) CUtensorMap tm_q, tm_kc, tm_vc, tm_kt, tm_vt, tm_kc2, tm_vc2;
   const uint64_t cache_rows = c.paged ? (uint64_t)c.n_pages * CLV_PAGE_SIZE : (uint64_t)s.batch * c.cap_tokens;
   const uint64_t tree_rows = (uint64_t)s.batch * s.n_nodes;
   if (!make_map(&tm_q, q, tree_rows, s.n_q_heads, G, BM / G) ||
@@ -908,8 +922,13 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
       !make_map(&tm_kt, k_tree, tree_rows, s.n_kv_heads, 1, PG) ||
       !make_map(&tm_vt, v_tree, tree_rows, s.n_kv_heads, 1, PG))
     return cudaErrorInvalidValue;
+  // whole-tile copies: only if the driver accepts the 4-D view (else the piece-wise copies do it all)
+  const bool pair_boxes = make_map_halves(&tm_kc2, c.k, cache_rows, s.n_kv_heads, BN) &&
+                          make_map_halves(&tm_vc2, c.v, cache_rows, s.n_kv_heads, BN);
+  if (!pair_boxes) { tm_kc2 = tm_kc; tm_vc2 = tm_vc; }
 
   Params p;
+  p.pair_boxes = pair_boxes ? 1 : 0;
   p.block_table = c.block_table;
   p.parent = parent;
   p.ctx_len = ctx_len;
@@ -941,7 +960,7 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, p);
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, tm_q, tm_kc, tm_vc, tm_kt, tm_vt, tm_kc2, tm_vc2, p);
 }
 
 }  // namespace clv
