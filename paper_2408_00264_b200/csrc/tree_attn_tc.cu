@@ -106,19 +106,41 @@ __device__ __forceinline__ void named_barrier(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// The same loads from this block's own shared memory (volatile asm too, so that they join the batch).
+__device__ __forceinline__ float4 smem_ld16(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint2 smem_ld8u(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+
 // Final combination of NSRC accumulators per output row, for the rows [first_row, first_row +
 // per_rank) of the tile that this block finalises.  The staged accumulators are fp16 (each row
-// scaled by a power of two of its own, which the weight undoes), 256 bytes per row.  One warp takes
-// 16 / NSRC rows at a time (16 remote 8-byte loads in flight per lane); lane j owns output
-// columns 4j .. 4j+3.  w[] holds the normalised weights divided by the rows' scales; source q of
-// a row lives in cluster rank q.
+// scaled by a power of two of its own, which the weight undoes), 256 bytes per row; source q of a
+// row lives in cluster rank q (this block's own share is read locally).  One warp takes 16 / NSRC
+// rows at a time: lane i < 16 fetches the (maximum, sum, scale) of one (row, source) pair and
+// every lane 16 8-byte pieces of the rows, all in flight together (one round trip through
+// distributed shared memory); the normalised weights then come from shuffles.  Lane j owns output
+// columns 4j .. 4j+3.
 template <int NSRC>
-__device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int first_row, int per_rank, int rot,
-                                           int warp, int lane, int tile_row0,
-                                           int RT, int rows_total, int G, int64_t seq_row0, int Hq, int head0,
-                                           uint16_t* out) {
+__device__ __forceinline__ void merge_rows(uint32_t sO_addr, uint32_t ml_addr, int my_rank, int first_row,
+                                           int per_rank, int warp, int lane, int tile_row0, int RT, int rows_total,
+                                           int G, int64_t seq_row0, int Hq, int head0, uint16_t* out, float* lse) {
   constexpr int RB = 16 / NSRC;
+  const float kLn2 = 0.6931471805599453f;
+  const int rot = my_rank + 1;   // first source read: the next rank's (every block starts at a different peer)
   for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
+    const int mu_ = (lane & 15) / NSRC, mj = (lane & 15) % NSRC;   // this lane's (row, source) pair
+    float4 ml;
+    {
+      const int trow = first_row + min(k0 + mu_, per_rank - 1);
+      const uint32_t a = ml_addr + (uint32_t)trow * 16u;
+      ml = (mj == my_rank) ? smem_ld16(a) : dsmem_ld16(cluster_map(a, (uint32_t)mj));
+    }
     uint2 x[RB * NSRC];
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
@@ -126,24 +148,41 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, const float* w, int
       const uint32_t off = (uint32_t)(trow * (HD * 2) + (((lane >> 1) ^ (trow & 15)) << 4) + ((lane & 1) << 3));
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
-        const int q = (j + rot) & (NSRC - 1);  // every block starts at a different peer
-        x[u * NSRC + j] = dsmem_ld8u(cluster_map(sO_addr + off, (uint32_t)q));
+        const int q = (j + rot) & (NSRC - 1);
+        x[u * NSRC + j] = (q == my_rank) ? smem_ld8u(sO_addr + off) : dsmem_ld8u(cluster_map(sO_addr + off, (uint32_t)q));
+      }
+    }
+    // weights: the NSRC lanes of a row sit side by side
+    float mmax = ml.x;
+#pragma unroll
+    for (int o = 1; o < NSRC; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
+    const float mu = (mmax == -INFINITY) ? 0.f : mmax;
+    const float wgt = (ml.y > 0.f) ? ex2(ml.x - mu) : 0.f;
+    float lsum = wgt * ml.y;
+#pragma unroll
+    for (int o = 1; o < NSRC; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+    const float wn = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
+    if (lse != nullptr && lane < 16 && mj == 0 && k0 + mu_ < per_rank) {
+      const int trow = first_row + k0 + mu_;
+      const int rg = tile_row0 + trow;
+      if (trow < RT && rg < rows_total) {
+        const int onode = rg / G, ogq = rg - onode * G;
+        lse[(seq_row0 + onode) * Hq + head0 + ogq] = (mmax + log2f(lsum)) * kLn2;
       }
     }
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
-      if (k0 + u >= per_rank) continue;
-      const int k = k0 + u;
-      const int trow = first_row + k;
-      const int rg = tile_row0 + trow;
-      if (trow >= RT || rg >= rows_total) continue;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int j = 0; j < NSRC; ++j) {
-        const float wq = w[k * NSRC + ((j + rot) & (NSRC - 1))];
+        const float wq = __shfl_sync(0xFFFFFFFFu, wn, u * NSRC + ((j + rot) & (NSRC - 1)));
         const float2 lo = half2_bits_to_float2(x[u * NSRC + j].x), hi = half2_bits_to_float2(x[u * NSRC + j].y);
         acc.x += wq * lo.x; acc.y += wq * lo.y; acc.z += wq * hi.x; acc.w += wq * hi.y;
       }
+      const int k = k0 + u;
+      const int trow = first_row + k;
+      const int rg = tile_row0 + trow;
+      if (k >= per_rank || trow >= RT || rg >= rows_total) continue;
       const int onode = rg / G, ogq = rg - onode * G;
       uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
       *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
@@ -176,7 +215,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ float s_xch[2][BM];   // values exchanged between the two threads of a row
   __shared__ float s_xch2[2][BM];
   __shared__ float4 s_ml[BM];      // (reference maximum, row sum, 1 / staging scale, -) for the merge
-  __shared__ float s_w[BM];        // merge: normalised weight of every (row of this rank, source)
   __shared__ int s_seq;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -802,35 +840,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     //      [j, j+1) * 128 / splits of the tile; source q of a row lives in cluster rank q ----
     const int per_rank = BM / p.splits;
     const int first_row = split * per_rank;
-    // (a) thread (k, q) fetches the (maximum, sum, scale) of source q of row k; the n_src lanes of
-    //     a row sit side by side in one warp, so the normalised weights come from shuffles.
-    if (tid < BM) {
-      const int k = tid / n_src, q = tid - k * n_src;
-      const int trow = first_row + k;
-      const float4 ml = dsmem_ld16(cluster_map(smem_u32(&s_ml[trow]), (uint32_t)q));
-      float mmax = ml.x;
-      for (int o = 1; o < n_src; o <<= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xFFFFFFFFu, mmax, o));
-      const float mu = (mmax == -INFINITY) ? 0.f : mmax;
-      const float wgt = (ml.y > 0.f) ? ex2(ml.x - mu) : 0.f;
-      float lsum = wgt * ml.y;
-      for (int o = 1; o < n_src; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
-      s_w[tid] = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
-      const int rg = tile_idx * RT + trow;
-      if (q == 0 && p.lse != nullptr && trow < RT && rg < rows_total) {
-        const int onode = rg / G, ogq = rg - onode * G;
-        p.lse[((int64_t)b * N + onode) * p.Hq + kvh * G + ogq] = (mmax + log2f(lsum)) * kLn2;
-      }
-    }
-    __syncthreads();
-    // (b) weighted sums, rows spread over the warps
     {
-      const uint32_t sO_addr = smem_u32(sO);
-      const int rot = split + 1;  // first source read: the next split's
+      const uint32_t sO_addr = smem_u32(sO), ml_addr = smem_u32(&s_ml[0]);
       const int64_t seq_row0 = (int64_t)b * N;
+      const int tr0 = tile_idx * RT, h0 = kvh * G;
       switch (n_src) {
-        case 2: merge_rows<2>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-        case 4: merge_rows<4>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
-        default: merge_rows<8>(sO_addr, s_w, first_row, per_rank, rot, warp, lane, tile_idx * RT, RT, rows_total, G, seq_row0, p.Hq, kvh * G, p.out); break;
+        case 2: merge_rows<2>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, tr0, RT, rows_total, G, seq_row0, p.Hq, h0, p.out, p.lse); break;
+        case 4: merge_rows<4>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, tr0, RT, rows_total, G, seq_row0, p.Hq, h0, p.out, p.lse); break;
+        default: merge_rows<8>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, tr0, RT, rows_total, G, seq_row0, p.Hq, h0, p.out, p.lse); break;
       }
     }
   }
