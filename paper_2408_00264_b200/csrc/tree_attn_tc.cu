@@ -128,8 +128,8 @@ __device__ __forceinline__ uint2 smem_ld8u(uint32_t addr) {
 // columns 4j .. 4j+3.
 template <int NSRC>
 __device__ __forceinline__ void merge_rows(uint32_t sO_addr, uint32_t ml_addr, int my_rank, int first_row,
-                                           int per_rank, int warp, int lane, int tile_row0, int RT, int rows_total,
-                                           int G, int64_t seq_row0, int Hq, int head0, uint16_t* out, float* lse) {
+                                           int per_rank, int warp, int lane, const long long* row_off,
+                                           uint16_t* out, float* lse) {
   constexpr int RB = 16 / NSRC;
   const float kLn2 = 0.6931471805599453f;
   const int rot = my_rank + 1;   // first source read: the next rank's (every block starts at a different peer)
@@ -163,12 +163,8 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, uint32_t ml_addr, i
     for (int o = 1; o < NSRC; o <<= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
     const float wn = wgt * (lsum > 0.f ? 1.f / lsum : 0.f) * ml.z;  // the staged row is 1 / ml.z times O
     if (lse != nullptr && lane < 16 && mj == 0 && k0 + mu_ < per_rank) {
-      const int trow = first_row + k0 + mu_;
-      const int rg = tile_row0 + trow;
-      if (trow < RT && rg < rows_total) {
-        const int onode = rg / G, ogq = rg - onode * G;
-        lse[(seq_row0 + onode) * Hq + head0 + ogq] = (mmax + log2f(lsum)) * kLn2;
-      }
+      const long long o = row_off[first_row + k0 + mu_];   // where the row's output starts, -1 for an idle row
+      if (o >= 0) lse[o / HD] = (mmax + log2f(lsum)) * kLn2;
     }
 #pragma unroll
     for (int u = 0; u < RB; ++u) {
@@ -179,13 +175,10 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, uint32_t ml_addr, i
         const float2 lo = half2_bits_to_float2(x[u * NSRC + j].x), hi = half2_bits_to_float2(x[u * NSRC + j].y);
         acc.x += wq * lo.x; acc.y += wq * lo.y; acc.z += wq * hi.x; acc.w += wq * hi.y;
       }
-      const int k = k0 + u;
-      const int trow = first_row + k;
-      const int rg = tile_row0 + trow;
-      if (k >= per_rank || trow >= RT || rg >= rows_total) continue;
-      const int onode = rg / G, ogq = rg - onode * G;
-      uint16_t* dst = out + ((seq_row0 + onode) * Hq + head0 + ogq) * HD + lane * 4;
-      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+      if (k0 + u >= per_rank) continue;
+      const long long o = row_off[first_row + k0 + u];
+      if (o < 0) continue;
+      *reinterpret_cast<uint2*>(out + o + lane * 4) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
     }
   }
 }
@@ -216,6 +209,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ float s_xch2[2][BM];
   __shared__ float4 s_ml[BM];      // (reference maximum, row sum, 1 / staging scale, -) for the merge
   __shared__ int s_seq;
+  __shared__ long long s_rowoff[BM];   // per row of the tile: element offset of its output row, -1 for an idle row
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int CS = p.splits;                            // cluster size
@@ -420,6 +414,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
   const int pair_bar = 2 + quarter;              // named barrier of the two warps that share rows
   float m_ref = -INFINITY, l_run = 0.f;
+  if (warp >= 2 && ch == 0)   // read by the merge, after several block-wide barriers
+    s_rowoff[row] = row_valid ? (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD : -1ll;
 
   if (warp == 0) {
     // =========================== TMA producer ===============================================
@@ -842,12 +838,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int first_row = split * per_rank;
     {
       const uint32_t sO_addr = smem_u32(sO), ml_addr = smem_u32(&s_ml[0]);
-      const int64_t seq_row0 = (int64_t)b * N;
-      const int tr0 = tile_idx * RT, h0 = kvh * G;
       switch (n_src) {
-        case 2: merge_rows<2>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, tr0, RT, rows_total, G, seq_row0, p.Hq, h0, p.out, p.lse); break;
-        case 4: merge_rows<4>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, tr0, RT, rows_total, G, seq_row0, p.Hq, h0, p.out, p.lse); break;
-        default: merge_rows<8>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, tr0, RT, rows_total, G, seq_row0, p.Hq, h0, p.out, p.lse); break;
+        case 2: merge_rows<2>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, s_rowoff, p.out, p.lse); break;
+        case 4: merge_rows<4>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, s_rowoff, p.out, p.lse); break;
+        default: merge_rows<8>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, s_rowoff, p.out, p.lse); break;
       }
     }
   }
