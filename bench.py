@@ -393,10 +393,10 @@ ATTN_BOUND = {"C1": "hbm", "C2": "hbm", "C3": "hbm", "C4": "hbm", "C5": "tensor"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from ncu captures of the library whose
 # clv_version() is the first element; a different library version reports null instead
 NCU_TRAFFIC = {
-    (110, "C1", "tree_attn"): 8.88e6, (110, "C2", "tree_attn"): 35.2e6, (110, "C3", "tree_attn"): 73.0e6,
-    (110, "C4", "tree_attn"): 521.2e6, (110, "C5", "tree_attn"): 1090.3e6,
-    (110, "C1", "accept_argmax"): 1.04e6, (110, "C2", "accept_argmax"): 4.11e6, (110, "C3", "accept_argmax"): 66.3e6,
-    (110, "C4", "accept_argmax"): 263.2e6, (110, "C5", "accept_argmax"): 263.3e6,
+    (111, "C1", "tree_attn"): 8.88e6, (111, "C2", "tree_attn"): 35.2e6, (111, "C3", "tree_attn"): 72.7e6,
+    (111, "C4", "tree_attn"): 521.0e6, (111, "C5", "tree_attn"): 1089.0e6,
+    (111, "C1", "accept_argmax"): 1.04e6, (111, "C2", "accept_argmax"): 4.11e6, (111, "C3", "accept_argmax"): 65.7e6,
+    (111, "C4", "accept_argmax"): 263.0e6, (111, "C5", "accept_argmax"): 263.0e6,
 }
 MIN_TIMED_MS = 200.0   # the --steps loop is repeated until this much has been timed
 

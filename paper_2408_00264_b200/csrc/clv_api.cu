@@ -520,6 +520,6 @@ int clv_last_cuda_error(void) { return g_last_cuda_error; }
 void clv_test_set_wait_limit(int64_t sm_cycles) {
   g_wait_limit.store(sm_cycles > 0 ? (long long)sm_cycles : 2000000000ll, std::memory_order_relaxed);
 }
-int clv_version(void) { return 110; }
+int clv_version(void) { return 111; }
 
 }  // extern "C"
