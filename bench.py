@@ -726,13 +726,19 @@ def main(argv=None):
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer timing (profiling runs)")
     ap.add_argument("--no-other-workloads", dest="all_workloads", action="store_false",
                     help="time only --workload (by default a single-GPU run also times the other four)")
-    ap.add_argument("--only", default=None, choices=["draft_head_step"],
-                    help="profiling aid: time just this call (batch 4, hidden 4096, vocabulary 128256), print its "
+    ap.add_argument("--only", default=None, choices=["draft_head_step", "accept_sample"],
+                    help="profiling aid: time just this call (C3's batch, hidden size and vocabulary), print its "
                          "figures and exit")
     args = ap.parse_args(argv)
     if args.only == "draft_head_step":
         import torch
         print(json.dumps({"draft_head_step": time_draft_head(4, 4096, 32, 128256, torch.device("cuda:0"))}))
+        return
+    if args.only == "accept_sample":
+        import torch
+        from paper_2408_00264_b200 import workloads as W
+        w = W.generate(W.CONFIGS["C3"])
+        print(json.dumps({"accept_sample": time_accept_sample(w, torch.device("cuda:0"))}))
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         if args.impl == "reference":   # the CPU arm runs on rank 0 alone
