@@ -54,7 +54,8 @@ def run_gpu(clv, h, e, wts, k_top):
                                          (130, 128, 4, 1000, 4), (8, 4096, 32, 128256, 8),
                                          (4, 64, 4, 9000, 32),      # the widest one-pass selection, two levels
                                          (2, 64, 2, 3000, 40),      # beyond it: one pass per proposal
-                                         (70, 192, 48, 2049, 2)])   # head size 4; one entry in the second slice
+                                         (70, 192, 48, 2049, 2),    # head size 4; one entry in the second slice
+                                         (1, 64, 1, 100, 3), (256, 64, 2, 300, 3)])   # fewest and most rows
 def test_draft_head_step(clv, oracle, R, H, nh, V, k):
     h, e, wts = W.make_draft_head(R, H, nh, V, seed=R + H + V)
     p, ids, vals, logits = oracle.draft_head_step(h, e, wts, k)
