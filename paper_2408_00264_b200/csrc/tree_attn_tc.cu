@@ -43,10 +43,7 @@ constexpr int BM = 128;                // rows per block
 constexpr int BN = 128;                // keys per tile
 constexpr int PPT = BN / PG;           // pieces per tile
 constexpr int NSB = 3;                 // score buffers (= depth of the K ring)
-constexpr int kThreads = 384;          // three warpgroups: producer + issuer (+ two idle warps), and two of softmax warps
-constexpr int kFirstSoftmaxWarp = 4;
-constexpr int kRegsLow = 56, kRegsHigh = 224, kRegsLaunch = 168;   // per thread: first warpgroup / softmax warpgroups / at launch
-static_assert(128 * kRegsLow + 256 * kRegsHigh <= kThreads * kRegsLaunch, "the register split fits what the block is launched with");
+constexpr int kThreads = 320;
 constexpr int kSoftmaxThreads = 256;
 constexpr uint32_t kQTile = BM * HD * 2;      // 32 KB: two [128 rows][64 d] swizzled halves
 constexpr uint32_t kPiece = PG * 64 * 2;       // 8 KB: [64 keys][64 d] swizzled, one TMA box
@@ -105,17 +102,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t u) {
   return __half22float2(*reinterpret_cast<const __half2*>(&u));
 }
-// A warpgroup (four warps) hands registers back to the block's pool or takes some from it; every
-// warp of the warpgroup executes the same one.  The counts must add up to no more than what the
-// block was launched with (an increase waits until the pool has enough).
-template <int kRegs>
-__device__ __forceinline__ void regs_release_to() {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
-}
-template <int kRegs>
-__device__ __forceinline__ void regs_grow_to() {
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
-}
 __device__ __forceinline__ void named_barrier(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -147,7 +133,7 @@ __device__ __forceinline__ void merge_rows(uint32_t sO_addr, uint32_t ml_addr, i
   constexpr int RB = 16 / NSRC;
   const float kLn2 = 0.6931471805599453f;
   const int rot = my_rank + 1;   // first source read: the next rank's (every block starts at a different peer)
-  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kSoftmaxThreads / 32)) {
+  for (int k0 = warp * RB; k0 < per_rank; k0 += RB * (kThreads / 32)) {
     const int mu_ = (lane & 15) / NSRC, mj = (lane & 15) % NSRC;   // this lane's (row, source) pair
     float4 ml;
     {
@@ -374,7 +360,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   // ---- per-sequence checks (the threads of warps 2 and up) ----------------------------------
   bool bad = len_bad;
-  for (int i = tid - 32 * kFirstSoftmaxWarp; i < N; i += kSoftmaxThreads) {
+  for (int i = tid - 64; i < N; i += kThreads - 64) {
     if (i < 0) continue;
     const int par = p.parent[(int64_t)b * N + i];
     s_parent[i] = par;
@@ -417,7 +403,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   // per-thread state of the softmax threads (warps 2..9); declared here because the epilogue runs
   // after block-wide synchronisation points that all roles must reach together
-  const int sw = warp >= kFirstSoftmaxWarp ? warp - kFirstSoftmaxWarp : 0;
+  const int sw = warp >= 2 ? warp - 2 : 0;
   const int ch = sw >> 2;                        // which 64-key piece of every tile (= column half)
   const int quarter = warp & 3;                  // TMEM lanes this warp may touch
   const int row = quarter * 32 + lane;           // row inside the 128-row tile
@@ -428,11 +414,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
   const int pair_bar = 2 + quarter;              // named barrier of the two warps that share rows
   float m_ref = -INFINITY, l_run = 0.f;
-  if (warp >= kFirstSoftmaxWarp && ch == 0)   // read by the merge, after several block-wide barriers
+  if (warp >= 2 && ch == 0)   // read by the merge, after several block-wide barriers
     s_rowoff[row] = row_valid ? (((int64_t)b * N + node) * p.Hq + kvh * G + gq) * HD : -1ll;
 
-  if (warp < kFirstSoftmaxWarp) {
-  regs_release_to<kRegsLow>();   // the softmax warpgroups take what is freed
   if (warp == 0) {
     // =========================== TMA producer ===============================================
     // K and V advance independently: whichever ring has a free buffer gets its next tile.
@@ -522,46 +506,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (t + NSB < T) ok = issue_qk(t + NSB);
       }
     }
-  }
-  __syncwarp();
-    // ---- the first warpgroup's way out: the barriers of the tail below in the same order, and none
-    //      of the softmax threads' state (this path runs on few registers)
-    if (*abort_flag) {
-      if (warp == 0 && lane == 0) {
-        // TMA copies that were issued land on their own; wait for the newest phase of each stage
-        for (int i = max(0, issued_k - KST); i < issued_k; ++i) mbar_drain(bar(B_KF + i % KST), (i / KST) & 1);
-        for (int i = max(0, issued_v - VST); i < issued_v; ++i) mbar_drain(bar(B_VF + i % VST), (i / VST) & 1);
-        if (T > 0) mbar_drain(bar(B_Q), 0);
-      }
-      if (warp == 1 && lane == 0) {
-        umma_commit(bar(B_DR));
-        mbar_drain(bar(B_DR), 0);  // completes when every MMA issued so far has finished
-      }
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    // the ticket is taken here and looked at when the block leaves, so that its round trip is
-    // hidden behind the epilogue (no wait can run out after this point)
-    unsigned my_ticket = 0;
-    if (tid == 0) my_ticket = report(*abort_flag != 0 ? 2u : 0u);
-    tc_fence_before();
-    __syncthreads();
-    if (CS > 1) {
-      cg::cluster_group cl = cg::this_cluster();
-      cl.sync();
-      cl.sync();
-    }
-    if (warp == 1) release_tmem();
-    if (tid == 0) publish(my_ticket);
-    return;
-  }
-  regs_grow_to<kRegsHigh>();
-  {
+  } else {
     // =========================== softmax threads ==============================================
     // ancestor bitsets (row i of the tree's topology matrix), built while the first tiles are on
     // their way; the 256 threads meet at a named barrier of their own
-    for (int i = tid - 32 * kFirstSoftmaxWarp; i < N; i += kSoftmaxThreads) {
+    for (int i = tid - 64; i < N; i += kSoftmaxThreads) {
       uint32_t w[4] = {0, 0, 0, 0};
       int j = i;
       for (int hop = 0; hop < N && j >= 0; ++hop) {
@@ -570,7 +519,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       s_anc[i][0] = w[0]; s_anc[i][1] = w[1]; s_anc[i][2] = w[2]; s_anc[i][3] = w[3];
     }
-    if (reporter && warp == kFirstSoftmaxWarp) {  // one warp per sequence reports: block table of the context
+    if (reporter && warp == 2) {  // one warp per sequence reports: block table of the context
       bool pbad = false;
       if (p.paged) {
         for (int pg = lane; pg < p_cache; pg += 32) {
@@ -737,7 +686,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         wait_all(bar(B_VF + vst), (t / VST) & 1);
         if (!fail) {
           uint8_t* vt = sV_gen + vst * kStage;
-          const int me = tid - 32 * kFirstSoftmaxWarp;   // 0 .. 255 among the softmax threads
+          const int me = tid - 64;   // 0 .. 255 among the softmax threads
           constexpr int kHalves = 2;   // halves of the head dimension
 #pragma unroll
           for (int j = 0; j < PPT; ++j) {
@@ -767,10 +716,26 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   // ---- every role meets here: all MMAs and copies of this block are complete -----------------
   __syncwarp();
+  if (*abort_flag) {
+    if (warp == 0 && lane == 0) {
+      // TMA copies that were issued land on their own; wait for the newest phase of each stage
+      for (int i = max(0, issued_k - KST); i < issued_k; ++i) mbar_drain(bar(B_KF + i % KST), (i / KST) & 1);
+      for (int i = max(0, issued_v - VST); i < issued_v; ++i) mbar_drain(bar(B_VF + i % VST), (i / VST) & 1);
+    }
+    if (warp == 2 && lane == 0 && T > 0) mbar_drain(bar(B_Q), 0);
+    if (warp == 1 && lane == 0) {
+      umma_commit(bar(B_DR));
+      mbar_drain(bar(B_DR), 0);  // completes when every MMA issued so far has finished
+    }
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const bool aborted = *abort_flag != 0;
+  // the ticket is taken here and looked at when the block leaves, so that its round trip is hidden
+  // behind the epilogue (no wait can run out after this point)
+  unsigned my_ticket = 0;
+  if (tid == 0) my_ticket = report(aborted ? 2u : 0u);
   const int n_src = p.splits;   // accumulators that cover one output row
   const float kLn2 = 0.6931471805599453f;
   // staging area for the merge: O as fp16 [128 rows][128], every row scaled by a power of two that
@@ -781,7 +746,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // The area reuses the tile memory, which nothing reads any more.
   uint8_t* const sO = smem_raw + (sQ - smem_u32(smem_raw));
 
-  if (!aborted && warp >= kFirstSoftmaxWarp) {
+  if (!aborted && warp >= 2) {
     // the row's two threads add up their sums (and, for staging, agree on the row's scale)
     float amax = 0.f;
     if (n_src > 1 && T > 0) {
@@ -858,7 +823,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
   tc_fence_before();
   __syncthreads();
-  if (CS == 1) return;  // a block that is its own cluster
+  if (CS == 1) {  // a block that is its own cluster
+    if (warp == 1) release_tmem();
+    if (tid == 0) publish(my_ticket);
+    return;
+  }
 
   cg::cluster_group cluster = cg::this_cluster();
   cluster.sync();  // every block's staging area is complete and its MMAs are done (also reached by an aborted block)
@@ -869,17 +838,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int first_row = split * per_rank;
     {
       const uint32_t sO_addr = smem_u32(sO), ml_addr = smem_u32(&s_ml[0]);
-      const int mw = warp - kFirstSoftmaxWarp;   // the softmax warps do the merge
-      if (mw >= 0) {
-        switch (n_src) {
-          case 2: merge_rows<2>(sO_addr, ml_addr, split, first_row, per_rank, mw, lane, s_rowoff, p.out, p.lse); break;
-          case 4: merge_rows<4>(sO_addr, ml_addr, split, first_row, per_rank, mw, lane, s_rowoff, p.out, p.lse); break;
-          default: merge_rows<8>(sO_addr, ml_addr, split, first_row, per_rank, mw, lane, s_rowoff, p.out, p.lse); break;
-        }
+      switch (n_src) {
+        case 2: merge_rows<2>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, s_rowoff, p.out, p.lse); break;
+        case 4: merge_rows<4>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, s_rowoff, p.out, p.lse); break;
+        default: merge_rows<8>(sO_addr, ml_addr, split, first_row, per_rank, warp, lane, s_rowoff, p.out, p.lse); break;
       }
     }
   }
   cluster.sync();  // no block may leave while a peer still reads its shared memory
+  if (warp == 1) release_tmem();
+  if (tid == 0) publish(my_ticket);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -952,12 +920,6 @@ cudaError_t launch_tree_attn_tc(const AttnPlan& plan, const clv_shape& s, const 
   const int G = s.n_q_heads / s.n_kv_heads;
   static OncePerDevice once;
   cudaError_t e0 = run_once_per_device(once, [] {
-    // the kernel moves registers between its warpgroups: that must fit what a block is launched with
-    cudaFuncAttributes fa;
-    cudaError_t e = cudaFuncGetAttributes(&fa, tree_attn_tc_kernel);
-    if (e != cudaSuccess) return e;
-    if (fa.numRegs * kThreads < 128 * kRegsLow + 256 * kRegsHigh || fa.numRegs < kRegsLaunch)
-      return cudaErrorLaunchOutOfResources;
     return cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)Cfg::kSmem);
   });
