@@ -6,7 +6,8 @@ receives input and output tensors, or on a latency path that must not hit cudaMa
 synchronisation.  `clv_accept_argmax_noalloc` keeps its counters and partial results in a fixed
 array inside the library instead of a workspace.  This file checks, through the C ABI, that it
 returns exactly what `clv_accept_argmax` returns, twice in a row (the array keeps the previous
-call's contents), and that it refuses problems beyond its fixed capacity.
+call's contents), that it refuses problems beyond its fixed capacity, that a call leaves the free
+device memory unchanged and that a call can be recorded in a CUDA graph and replayed.
 
 The file name sorts last on purpose, so a run that stops at the first failure has already
 executed every other test.
@@ -88,3 +89,25 @@ def test_noalloc_allocates_nothing(clv):
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
     assert free1 == free0
+
+
+def test_noalloc_call_can_be_captured_in_a_graph(clv, oracle):
+    # after the first call on the device (which looks up the array's address) a call is a clearing
+    # of the counters and a launch on the caller's stream: both can be recorded and replayed
+    vocab, rows = 5000, 24
+    lg, ld = _logits(rows, vocab, seed=9)
+    d = torch.from_numpy(lg.view(np.int16)).cuda()
+    shape = clv.make_shape(1, rows, 1, 1, vocab, 1)
+    ids = torch.full((1, rows), -7, dtype=torch.int32, device="cuda")
+    clv.clv_accept_argmax_noalloc(shape, d, ld, ids)      # warm-up, outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        clv.clv_accept_argmax_noalloc(shape, d, ld, ids)
+    for seed in (10, 11):                                  # new data in the same buffer, replayed twice
+        lg2, _ = _logits(rows, vocab, seed=seed)
+        d.copy_(torch.from_numpy(lg2.view(np.int16)))
+        ids.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(ids.cpu().numpy().reshape(-1), oracle.argmax(lg2, vocab))
